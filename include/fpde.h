@@ -1,0 +1,173 @@
+/*
+ * fpde.h -- C ABI of the fused finite-difference PDE-residual operator library (libfpde.so).
+ *
+ * The library evaluates, on a regular Cartesian (space or space-time) grid, the discrete PDE
+ * residuals of grid-aligned physical fields in one fused forward pass, and maps the upstream
+ * sensitivities dL/dres back to dL/dfield with a hand-derived discrete adjoint in gather form.
+ * It is the method of the paper's Section 2 ("Kernel design and discrete analytic adjoints"):
+ * fused forward stencil (Section 2.1), analytic discrete-adjoint backward (Section 2.2,
+ * Eq. 1, Appendix A.2) and boundary-gradient correction (Section 2.3, Appendix A.4).
+ *
+ * General rules (all entry points)
+ *   - Plain C types only.  Nothing throws or aborts; every call returns an fpde_status.
+ *   - Arrays are fp32, row-major, axis 0 slowest, last axis contiguous, all of the FULL grid
+ *     shape.  Space-time grids keep t as the last (contiguous) axis.
+ *   - "device" pointers are CUDA device memory owned by the caller, 16-byte aligned, not
+ *     overlapping; "host" pointers are ordinary host memory read during the call only.
+ *   - The library allocates no device memory and keeps no state between calls.  Work is queued
+ *     on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and the
+ *     call returns without waiting for it.
+ *   - On any status other than FPDE_OK nothing has been launched.  FPDE_ERR_CUDA reports a
+ *     launch the CUDA runtime rejected.
+ *   - With no CUDA device the entry points still load and validate, and a launch attempt
+ *     returns FPDE_ERR_CUDA: there is no CPU fallback.
+ */
+#ifndef FPDE_H
+#define FPDE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FPDE_OK = 0,
+    FPDE_ERR_BAD_OP = 1,       /* operator id out of range                                   */
+    FPDE_ERR_NULL = 2,         /* a required pointer (or array entry) is NULL                */
+    FPDE_ERR_NDIM = 3,         /* ndim does not match the operator                           */
+    FPDE_ERR_SHAPE = 4,        /* an extent is too small, too large, or breaks the x4 rule   */
+    FPDE_ERR_ALIGN = 5,        /* a device pointer is not 16-byte aligned                    */
+    FPDE_ERR_SPACING = 6,      /* a spacing is not finite and positive                       */
+    FPDE_ERR_COEFF_COUNT = 7,  /* ncoeffs does not match the operator                        */
+    FPDE_ERR_BC = 8,           /* boundary kinds not supported by the operator               */
+    FPDE_ERR_WORKSPACE = 9,    /* workspace NULL, misaligned or smaller than required        */
+    FPDE_ERR_CUDA = 10         /* the CUDA runtime reported an error                         */
+} fpde_status;
+
+/*
+ * Operators.  Fields (differentiated inputs), sources (read-only inputs without gradient),
+ * residuals and coefficients, in the order the arrays are passed:
+ *
+ *  FPDE_OP_BURGERS_1D_T     (x,t) array.  fields [u]; residuals [r]; coeffs [nu].
+ *        r = D_t u + u D_x u - nu D_xx u at every node; centred second-order differences
+ *        inside, second-order one-sided differences on the first/last node of each axis.
+ *        bc = (ONE_SIDED, ONE_SIDED).
+ *  FPDE_OP_POISSON_2D       (x,y) array.  fields [u]; sources [f]; residuals [r]; no coeffs.
+ *        r = -(d_xx u + d_yy u) - f, five-point Laplacian, rows where it fits.
+ *        bc = (INTERIOR, INTERIOR).
+ *  FPDE_OP_GRAYSCOTT_2D     (x,y) array.  fields [u,v]; residuals [r_u,r_v];
+ *        coeffs [D_u, D_v, F, k].  r_u = D_u Lap u - u v^2 + F (1-u),
+ *        r_v = D_v Lap v + u v^2 - (F+k) v.  bc = (PERIODIC, PERIODIC).
+ *  FPDE_OP_HELMHOLTZ_3D_O4  (x,y,z) array.  fields [u]; sources [f]; residuals [r];
+ *        coeffs [k] (wavenumber).  r = Lap4 u + k^2 u - f with the fourth-order 13-point
+ *        Laplacian (-1,16,-30,16,-1)/(12 h^2) per axis.  bc = (INTERIOR x3): rows at indices
+ *        2..n-3; the two outer layers are data and receive gradient.
+ *  FPDE_OP_NS_3D_T          (x,y,z,t) array.  fields [u,v,w,p];
+ *        residuals [mom_x, mom_y, mom_z, continuity]; coeffs [nu].
+ *        mom_q = d_t q + u d_x q + v d_y q + w d_z q + d_{a_q} p - nu Lap q, continuity =
+ *        d_x u + d_y v + d_z w (Section 2.1's residuals extended by t, w and z), centred
+ *        differences.  bc = (PERIODIC x3, INTERIOR): rows at t-index 1..n_t-2.
+ *
+ * Shape rules: the contiguous extent must be a multiple of 4 (float4 path) except for
+ * BURGERS_1D_T; PERIODIC / INTERIOR axes need n >= 2*radius+1, ONE_SIDED axes n >= 4; the
+ * total number of nodes must stay below 2^31.
+ */
+typedef enum {
+    FPDE_OP_BURGERS_1D_T = 0,
+    FPDE_OP_POISSON_2D = 1,
+    FPDE_OP_GRAYSCOTT_2D = 2,
+    FPDE_OP_HELMHOLTZ_3D_O4 = 3,
+    FPDE_OP_NS_3D_T = 4,
+    FPDE_OP_COUNT = 5
+} fpde_op;
+
+/* Boundary kind of one array axis (Appendix A.4 names the three causes of boundary terms:
+ * prescribed values, one-sided formulas, omitted neighbours). */
+typedef enum {
+    FPDE_BC_PERIODIC = 0,   /* rows at every node, wrap-around neighbours                       */
+    FPDE_BC_INTERIOR = 1,   /* rows only where the full stencil fits; the outer `radius` layers */
+                            /* are ordinary input data (e.g. Dirichlet values) and do receive   */
+                            /* gradient from the rows that read them                            */
+    FPDE_BC_ONE_SIDED = 2   /* rows at every node, second-order one-sided formulas at the edges */
+} fpde_bc;
+
+typedef struct {
+    int ndim, nfields, nsources, nresiduals, ncoeffs, radius;
+    int bc[4];              /* the boundary kinds the operator accepts, per axis */
+} fpde_op_info_t;
+
+/* Describe an operator (host only).  FPDE_ERR_BAD_OP / FPDE_ERR_NULL on bad arguments. */
+int fpde_op_info(int op, fpde_op_info_t* out);
+
+/* Static, never-NULL description of a status code. */
+const char* fpde_strerror(int status);
+
+/* Number of nodes that carry a residual row (N_r, the divisor of each mean square); 0 if the
+ * operator / shape is invalid.  Host only. */
+int64_t fpde_row_count(int op, int ndim, const int64_t* shape);
+
+/* Bytes of device scratch fpde_fwd needs for this operator and grid (loss partial sums); 0 if
+ * the operator / shape is invalid.  fpde_bwd needs none.  Host only. */
+size_t fpde_workspace_bytes(int op, int ndim, const int64_t* shape);
+
+/*
+ * Fused forward residual + loss (Section 2.1; loss = mean square residual, summed over the
+ * residual fields, which the paper evaluates outside its operator and this library fuses).
+ *
+ *   fields     host array of nfields   device pointers, read only
+ *   sources    host array of nsources  device pointers, read only (may be NULL if nsources = 0)
+ *   residuals  host array of nresiduals device pointers, overwritten: r_e at every node that
+ *              carries a row, exactly 0.0f elsewhere
+ *   loss_out   device, nresiduals+1 doubles, overwritten with L_0..L_{E-1} and their sum, where
+ *              L_e = (1/N_r) sum over rows r_e^2.  The sum is taken in a fixed order: repeated
+ *              calls give bit-identical results.  NULL skips the loss (workspace unused).
+ *   ndim, shape, spacing, coeffs, ncoeffs, bc   host; see the operator list
+ *   workspace  device scratch of at least fpde_workspace_bytes() bytes, contents arbitrary
+ *              before and after; calls sharing a workspace must not overlap on the GPU
+ *   stream     cudaStream_t
+ */
+int fpde_fwd(int op,
+             const float* const* fields,
+             const float* const* sources,
+             float* const* residuals,
+             double* loss_out,
+             int ndim, const int64_t* shape,
+             const double* spacing,
+             const double* coeffs, int ncoeffs,
+             const int* bc,
+             void* workspace, size_t workspace_bytes,
+             void* stream);
+
+/*
+ * Discrete adjoint in gather form with boundary-gradient correction (Sections 2.2 and 2.3):
+ * gfields[f] = sum_e J_{e,f}^T G_e with G_e = gscale[e] * gres[e] on the rows of residual e
+ * and 0 elsewhere (entries of gres at nodes without a row are ignored).
+ *
+ *   fields     as in fpde_fwd (the Jacobian of a nonlinear operator depends on them)
+ *   gres       host array of nresiduals device pointers: upstream dL/dr_e, read only.  Passing
+ *              the residual arrays fpde_fwd wrote, with gscale[e] = 2/N_r, yields the gradient
+ *              of the fused loss.
+ *   gscale     host, nresiduals doubles; NULL means all 1
+ *   gfields    host array of nfields device pointers, OVERWRITTEN (not accumulated) at every
+ *              node, boundary layers included
+ *   workspace  unused by the current kernels; may be NULL with workspace_bytes = 0
+ * No atomics are used: every output element is written by exactly one thread.
+ */
+int fpde_bwd(int op,
+             const float* const* fields,
+             const float* const* gres,
+             const double* gscale,
+             float* const* gfields,
+             int ndim, const int64_t* shape,
+             const double* spacing,
+             const double* coeffs, int ncoeffs,
+             const int* bc,
+             void* workspace, size_t workspace_bytes,
+             void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FPDE_H */

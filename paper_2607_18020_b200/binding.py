@@ -1,0 +1,187 @@
+"""ctypes binding of libfpde.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path (residuals, loss, adjoint, boundary correction) runs in the library's
+CUDA kernels; this module turns torch tensors into device pointers and host scalars into C
+arrays.  There is no fallback: if the shared library is missing or a call is refused, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+from . import workloads as _w
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfpde.so")
+
+# numeric ids of include/fpde.h
+OP_IDS = {_w.BURGERS_1D_T: 0, _w.POISSON_2D: 1, _w.GRAYSCOTT_2D: 2, _w.HELMHOLTZ_3D_O4: 3, _w.NS_3D_T: 4}
+BC_IDS = {_w.PERIODIC: 0, _w.INTERIOR: 1, _w.ONE_SIDED: 2}
+FPDE_OK = 0
+
+
+class FpdeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: status %d (%s)" % (where, status, strerror(status)))
+
+
+class OpInfo(ctypes.Structure):
+    _fields_ = [("ndim", ctypes.c_int), ("nfields", ctypes.c_int), ("nsources", ctypes.c_int),
+                ("nresiduals", ctypes.c_int), ("ncoeffs", ctypes.c_int), ("radius", ctypes.c_int),
+                ("bc", ctypes.c_int * 4)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libfpde.so is missing (%s): build it with "
+                               "`python -m paper_2607_18020_b200.build`; there is no fallback path" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vpp = ctypes.POINTER(ctypes.c_void_p)
+        L.fpde_op_info.restype = ctypes.c_int
+        L.fpde_op_info.argtypes = [ctypes.c_int, ctypes.POINTER(OpInfo)]
+        L.fpde_strerror.restype = ctypes.c_char_p
+        L.fpde_strerror.argtypes = [ctypes.c_int]
+        L.fpde_row_count.restype = ctypes.c_int64
+        L.fpde_row_count.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_workspace_bytes.restype = ctypes.c_size_t
+        L.fpde_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_fwd.restype = ctypes.c_int
+        L.fpde_fwd.argtypes = [ctypes.c_int, vpp, vpp, vpp, ctypes.c_void_p, ctypes.c_int,
+                               ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                               ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                               ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fpde_bwd.restype = ctypes.c_int
+        L.fpde_bwd.argtypes = [ctypes.c_int, vpp, vpp, ctypes.POINTER(ctypes.c_double), vpp, ctypes.c_int,
+                               ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                               ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                               ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _opid(op) -> int:
+    return OP_IDS[op] if isinstance(op, str) else int(op)
+
+
+def _ptr_array(ptrs: Sequence[Optional[int]]):
+    arr = (ctypes.c_void_p * max(1, len(ptrs)))()
+    for i, p in enumerate(ptrs):
+        arr[i] = p
+    return ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p))
+
+
+def _dev_ptrs(tensors) -> List[int]:
+    out = []
+    for t in tensors:
+        if hasattr(t, "data_ptr"):
+            out.append(t.data_ptr())
+        else:
+            out.append(int(t) if t is not None else None)
+    return out
+
+
+def _i64(v):
+    return (ctypes.c_int64 * max(1, len(v)))(*[int(x) for x in v])
+
+
+def _f64(v):
+    return (ctypes.c_double * max(1, len(v)))(*[float(x) for x in v])
+
+
+def _bcs(bc):
+    return (ctypes.c_int * max(1, len(bc)))(*[BC_IDS[b] if isinstance(b, str) else int(b) for b in bc])
+
+
+def strerror(status: int) -> str:
+    return lib().fpde_strerror(int(status)).decode()
+
+
+def op_info(op) -> OpInfo:
+    info = OpInfo()
+    st = lib().fpde_op_info(_opid(op), ctypes.byref(info))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_op_info")
+    return info
+
+
+def row_count(op, shape) -> int:
+    return int(lib().fpde_row_count(_opid(op), len(shape), _i64(shape)))
+
+
+def workspace_bytes(op, shape) -> int:
+    return int(lib().fpde_workspace_bytes(_opid(op), len(shape), _i64(shape)))
+
+
+def fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace,
+               workspace_bytes_, stream, ndim=None, ncoeffs=None) -> int:
+    """Raw call: returns the status code (used by the error-path tests)."""
+    return lib().fpde_fwd(_opid(op),
+                          _ptr_array(_dev_ptrs(fields)) if fields is not None else None,
+                          _ptr_array(_dev_ptrs(sources)) if sources is not None else None,
+                          _ptr_array(_dev_ptrs(residuals)) if residuals is not None else None,
+                          _dev_ptrs([loss_out])[0] if loss_out is not None else None,
+                          len(shape) if ndim is None else ndim,
+                          _i64(shape) if shape is not None else None,
+                          _f64(spacing) if spacing is not None else None,
+                          _f64(coeffs) if coeffs is not None else None,
+                          len(coeffs) if ncoeffs is None else ncoeffs,
+                          _bcs(bc) if bc is not None else None,
+                          _dev_ptrs([workspace])[0] if workspace is not None else None,
+                          int(workspace_bytes_), stream)
+
+
+def bwd_status(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace,
+               workspace_bytes_, stream, ndim=None, ncoeffs=None) -> int:
+    return lib().fpde_bwd(_opid(op),
+                          _ptr_array(_dev_ptrs(fields)) if fields is not None else None,
+                          _ptr_array(_dev_ptrs(gres)) if gres is not None else None,
+                          _f64(gscale) if gscale is not None else None,
+                          _ptr_array(_dev_ptrs(gfields)) if gfields is not None else None,
+                          len(shape) if ndim is None else ndim,
+                          _i64(shape) if shape is not None else None,
+                          _f64(spacing) if spacing is not None else None,
+                          _f64(coeffs) if coeffs is not None else None,
+                          len(coeffs) if ncoeffs is None else ncoeffs,
+                          _bcs(bc) if bc is not None else None,
+                          _dev_ptrs([workspace])[0] if workspace is not None else None,
+                          int(workspace_bytes_), stream)
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if hasattr(stream, "cuda_stream"):
+        return stream.cuda_stream
+    return int(stream)
+
+
+def fpde_fwd(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, stream=None):
+    """Queue the fused forward residual + loss on `stream` (default: torch's current stream).
+
+    fields / sources / residuals: sequences of fp32 CUDA tensors of the grid shape;
+    loss_out: fp64 CUDA tensor with nresiduals+1 entries, or None; workspace: a CUDA tensor of at
+    least workspace_bytes(op, shape) bytes (uint8 or any dtype)."""
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    st = fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, wsb,
+                    _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_fwd")
+
+
+def fpde_bwd(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace=None, stream=None):
+    """Queue the gather-form adjoint (with its boundary correction) on `stream`."""
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    st = bwd_status(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace, wsb,
+                    _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_bwd")

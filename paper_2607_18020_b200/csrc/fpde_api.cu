@@ -1,0 +1,253 @@
+// C ABI of libfpde.so: operator registry, argument validation, conversion of host scalars to
+// kernel parameters, dispatch to the per-operator launchers, and the final loss reduction.
+// See include/fpde.h for the contract of every entry point.
+#include "../../include/fpde.h"
+#include "fpde_common.cuh"
+#include "fpde_internal.h"
+
+#include <cmath>
+#include <cstring>
+
+namespace fpde {
+
+int lap2d_items(const int* n);
+int star3d_items(const int* n);
+int ns_items(const int* n);
+int burgers_items(const int* n);
+
+struct OpEntry {
+    int ndim, nf, ns, ne, nc, radius;
+    int bc[MAX_D];
+    bool x4;                // contiguous extent must be a multiple of 4
+};
+
+static const OpEntry REGISTRY[FPDE_OP_COUNT] = {
+    /* BURGERS_1D_T    */ {2, 1, 0, 1, 1, 1, {FPDE_BC_ONE_SIDED, FPDE_BC_ONE_SIDED, 0, 0}, false},
+    /* POISSON_2D      */ {2, 1, 1, 1, 0, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0, 0}, true},
+    /* GRAYSCOTT_2D    */ {2, 2, 0, 2, 4, 1, {FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, 0, 0}, true},
+    /* HELMHOLTZ_3D_O4 */ {3, 1, 1, 1, 1, 2, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0}, true},
+    /* NS_3D_T         */ {4, 4, 0, 4, 1, 1, {FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_INTERIOR}, true},
+};
+
+static int check_shape(int op, int ndim, const int64_t* shape, int* n_out, int64_t* total, int64_t* rows) {
+    if (op < 0 || op >= FPDE_OP_COUNT) return FPDE_ERR_BAD_OP;
+    if (!shape) return FPDE_ERR_NULL;
+    const OpEntry& e = REGISTRY[op];
+    if (ndim != e.ndim) return FPDE_ERR_NDIM;
+    int64_t N = 1, R = 1;
+    for (int a = 0; a < ndim; ++a) {
+        const int64_t n = shape[a];
+        const int64_t need = e.bc[a] == FPDE_BC_ONE_SIDED ? 4 : 2 * e.radius + 1;
+        if (n < need || n > (int64_t)1 << 30) return FPDE_ERR_SHAPE;
+        N *= n;
+        if (N >= (int64_t)1 << 31) return FPDE_ERR_SHAPE;
+        R *= e.bc[a] == FPDE_BC_INTERIOR ? n - 2 * e.radius : n;
+        if (n_out) n_out[a] = (int)n;
+    }
+    if (e.x4 && shape[ndim - 1] % 4 != 0) return FPDE_ERR_SHAPE;
+    if (total) *total = N;
+    if (rows) *rows = R;
+    return FPDE_OK;
+}
+
+static size_t workspace_need(int op, const int* n) {
+    int items = 0;
+    switch (op) {
+    case FPDE_OP_BURGERS_1D_T: items = burgers_items(n); break;
+    case FPDE_OP_POISSON_2D:
+    case FPDE_OP_GRAYSCOTT_2D: items = lap2d_items(n); break;
+    case FPDE_OP_HELMHOLTZ_3D_O4: items = star3d_items(n); break;
+    case FPDE_OP_NS_3D_T: items = ns_items(n); break;
+    }
+    return (size_t)items * REGISTRY[op].ne * sizeof(float);
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Common validation of the arguments fwd and bwd share; fills the Problem.
+static int validate(int op, const float* const* fields, int ndim, const int64_t* shape,
+                    const double* spacing, const double* coeffs, int ncoeffs, const int* bc,
+                    Problem& q) {
+    int st = check_shape(op, ndim, shape, q.n, nullptr, &q.rows);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!fields || !spacing || !bc) return FPDE_ERR_NULL;
+    if (ncoeffs != e.nc) return FPDE_ERR_COEFF_COUNT;
+    if (e.nc > 0 && !coeffs) return FPDE_ERR_NULL;
+    for (int a = 0; a < ndim; ++a) {
+        if (!(spacing[a] > 0.0) || !std::isfinite(spacing[a])) return FPDE_ERR_SPACING;
+        if (bc[a] != e.bc[a]) return FPDE_ERR_BC;
+        q.h[a] = spacing[a];
+    }
+    for (int c = 0; c < e.nc; ++c) {
+        if (!std::isfinite(coeffs[c])) return FPDE_ERR_SPACING;
+        q.coef[c] = coeffs[c];
+    }
+    for (int f = 0; f < e.nf; ++f) {
+        if (!fields[f]) return FPDE_ERR_NULL;
+        if (!aligned16(fields[f])) return FPDE_ERR_ALIGN;
+        q.in[f] = fields[f];
+    }
+    q.op = op; q.ndim = ndim;
+    return FPDE_OK;
+}
+
+// Fixed-order final sum: thread t adds partials t, t+256, ... in fp64, then a shared-memory
+// tree of fixed shape.  One block, so no inter-block ordering exists to vary.
+__global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restrict__ partials, int nitems,
+                                                            int nres, double inv_rows,
+                                                            double* __restrict__ loss_out) {
+    __shared__ double sm[256];
+    double total = 0.0;
+    for (int e = 0; e < nres; ++e) {
+        double s = 0.0;
+        for (int i = threadIdx.x; i < nitems; i += 256) s += (double)partials[(size_t)e * nitems + i];
+        sm[threadIdx.x] = s;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if ((int)threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+            __syncthreads();
+        }
+        const double le = sm[0] * inv_rows;
+        if (threadIdx.x == 0) loss_out[e] = le;
+        total += le;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) loss_out[nres] = total;
+}
+
+cudaError_t launch_loss_finalize(const float* partials, int nitems, int nres, int64_t rows,
+                                 double* loss_out, cudaStream_t stream) {
+    loss_finalize_kernel<<<1, 256, 0, stream>>>(partials, nitems, nres, 1.0 / (double)rows, loss_out);
+    return cudaGetLastError();
+}
+
+}  // namespace fpde
+
+using namespace fpde;
+
+extern "C" {
+
+int fpde_op_info(int op, fpde_op_info_t* out) {
+    if (op < 0 || op >= FPDE_OP_COUNT) return FPDE_ERR_BAD_OP;
+    if (!out) return FPDE_ERR_NULL;
+    const OpEntry& e = REGISTRY[op];
+    out->ndim = e.ndim; out->nfields = e.nf; out->nsources = e.ns; out->nresiduals = e.ne;
+    out->ncoeffs = e.nc; out->radius = e.radius;
+    for (int a = 0; a < 4; ++a) out->bc[a] = a < e.ndim ? e.bc[a] : 0;
+    return FPDE_OK;
+}
+
+const char* fpde_strerror(int status) {
+    switch (status) {
+    case FPDE_OK: return "ok";
+    case FPDE_ERR_BAD_OP: return "operator id out of range";
+    case FPDE_ERR_NULL: return "a required pointer is NULL";
+    case FPDE_ERR_NDIM: return "ndim does not match the operator";
+    case FPDE_ERR_SHAPE: return "grid extent too small, too large, or contiguous extent not a multiple of 4";
+    case FPDE_ERR_ALIGN: return "device pointer not 16-byte aligned";
+    case FPDE_ERR_SPACING: return "spacing or coefficient not finite / not positive";
+    case FPDE_ERR_COEFF_COUNT: return "ncoeffs does not match the operator";
+    case FPDE_ERR_BC: return "boundary kinds not supported by the operator";
+    case FPDE_ERR_WORKSPACE: return "workspace NULL, misaligned or too small";
+    case FPDE_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+    }
+}
+
+int64_t fpde_row_count(int op, int ndim, const int64_t* shape) {
+    int64_t rows = 0;
+    if (check_shape(op, ndim, shape, nullptr, nullptr, &rows) != FPDE_OK) return 0;
+    return rows;
+}
+
+size_t fpde_workspace_bytes(int op, int ndim, const int64_t* shape) {
+    int n[MAX_D] = {0, 0, 0, 0};
+    if (check_shape(op, ndim, shape, n, nullptr, nullptr) != FPDE_OK) return 0;
+    // rounded up generously so that tile-shape tuning never outgrows a caller's allocation
+    const size_t need = workspace_need(op, n);
+    return ((need + 255) / 256) * 256 + 4096;
+}
+
+int fpde_fwd(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+             double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+             const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+             void* stream) {
+    Problem q;
+    std::memset(&q, 0, sizeof(q));
+    int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!residuals) return FPDE_ERR_NULL;
+    if (e.ns > 0 && !sources) return FPDE_ERR_NULL;
+    for (int s = 0; s < e.ns; ++s) {
+        if (!sources[s]) return FPDE_ERR_NULL;
+        if (!aligned16(sources[s])) return FPDE_ERR_ALIGN;
+        q.aux[s] = sources[s];
+    }
+    for (int r = 0; r < e.ne; ++r) {
+        if (!residuals[r]) return FPDE_ERR_NULL;
+        if (!aligned16(residuals[r])) return FPDE_ERR_ALIGN;
+        q.out[r] = residuals[r];
+    }
+    if (loss_out) {
+        if (!aligned16(loss_out)) return FPDE_ERR_ALIGN;
+        if (!workspace || !aligned16(workspace) || workspace_bytes < workspace_need(op, q.n))
+            return FPDE_ERR_WORKSPACE;
+        q.partials = static_cast<float*>(workspace);
+        q.loss_out = loss_out;
+    }
+    q.stream = static_cast<cudaStream_t>(stream);
+    cudaError_t ce = cudaSuccess;
+    int items = 0;
+    switch (op) {
+    case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_fwd(q); items = burgers_items(q.n); break;
+    case FPDE_OP_POISSON_2D:
+    case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_fwd(q); items = lap2d_items(q.n); break;
+    case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q); items = star3d_items(q.n); break;
+    case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n); break;
+    }
+    if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+    if (loss_out) {
+        ce = launch_loss_finalize(q.partials, items, e.ne, q.rows, loss_out, q.stream);
+        if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+    }
+    return FPDE_OK;
+}
+
+int fpde_bwd(int op, const float* const* fields, const float* const* gres, const double* gscale,
+             float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
+             const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+             void* stream) {
+    (void)workspace; (void)workspace_bytes;
+    Problem q;
+    std::memset(&q, 0, sizeof(q));
+    int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!gres || !gfields) return FPDE_ERR_NULL;
+    for (int r = 0; r < e.ne; ++r) {
+        if (!gres[r]) return FPDE_ERR_NULL;
+        if (!aligned16(gres[r])) return FPDE_ERR_ALIGN;
+        q.aux[r] = gres[r];
+        q.gscale[r] = gscale ? gscale[r] : 1.0;
+        if (!std::isfinite(q.gscale[r])) return FPDE_ERR_SPACING;
+    }
+    for (int f = 0; f < e.nf; ++f) {
+        if (!gfields[f]) return FPDE_ERR_NULL;
+        if (!aligned16(gfields[f])) return FPDE_ERR_ALIGN;
+        q.out[f] = gfields[f];
+    }
+    q.stream = static_cast<cudaStream_t>(stream);
+    cudaError_t ce = cudaSuccess;
+    switch (op) {
+    case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_bwd(q); break;
+    case FPDE_OP_POISSON_2D:
+    case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_bwd(q); break;
+    case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_bwd(q); break;
+    case FPDE_OP_NS_3D_T: ce = launch_ns_bwd(q); break;
+    }
+    return ce == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
+}
+
+}  // extern "C"

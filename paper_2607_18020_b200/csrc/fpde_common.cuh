@@ -1,0 +1,100 @@
+// Device-side helpers shared by the operator kernels: 128-bit loads/stores, lane-neighbour
+// exchange along the contiguous axis, and the deterministic loss reduction
+// (per-thread fp32 -> warp shuffle tree -> shared-memory block tree -> one partial per CTA).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fpde {
+
+constexpr unsigned FULL_MASK = 0xffffffffu;
+constexpr int MAX_RES = 4;        // most residual fields of any operator
+
+__device__ __forceinline__ float4 ld4(const float* p) {
+    return __ldg(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st4(float* p, float4 v) {
+    *reinterpret_cast<float4*>(p) = v;
+}
+__device__ __forceinline__ float4 f4zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ float4 f4scale(float4 a, float s) {
+    return make_float4(a.x * s, a.y * s, a.z * s, a.w * s);
+}
+__device__ __forceinline__ float f4get(const float4& a, int k) {
+    return k == 0 ? a.x : k == 1 ? a.y : k == 2 ? a.z : a.w;
+}
+__device__ __forceinline__ float sq4(float4 a) {
+    return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+}
+
+// Values one and two elements to the left / right of a thread's float4 along the contiguous
+// axis.  Inside a warp they come from the neighbouring lane's registers; the first and last
+// lane (and the first / last float4 of a row) fetch them from global memory, wrapped around
+// the row when `periodic`, else 0 outside the row.  `row` points at element 0 of the row,
+// `c4` is this thread's float4 index, `nc4` the row length in float4.  All 32 lanes must call
+// this (lanes with c4 >= nc4 pass cur = 0 and get unspecified values).  `cur` is the value
+// the thread holds in registers (already scaled / masked by the caller); values fetched from
+// global memory are multiplied by `scale` to match.
+struct LR2 { float l1, l2, r1, r2; };
+
+template <int R>
+__device__ __forceinline__ LR2 lane_neighbours(const float* __restrict__ row, int c4, int nc4,
+                                               float4 cur, bool periodic, float scale) {
+    LR2 o;
+    const int lane = threadIdx.x & 31;
+    o.l1 = __shfl_up_sync(FULL_MASK, cur.w, 1);
+    o.r1 = __shfl_down_sync(FULL_MASK, cur.x, 1);
+    if (R >= 2) {
+        o.l2 = __shfl_up_sync(FULL_MASK, cur.z, 1);
+        o.r2 = __shfl_down_sync(FULL_MASK, cur.y, 1);
+    } else {
+        o.l2 = 0.f; o.r2 = 0.f;
+    }
+    if (c4 < nc4) {
+        const int n = nc4 * 4;
+        if (lane == 0 || c4 == 0) {
+            int j1 = 4 * c4 - 1, j2 = 4 * c4 - 2;
+            if (periodic) { if (j1 < 0) j1 += n; if (j2 < 0) j2 += n; }
+            o.l1 = j1 >= 0 ? scale * __ldg(row + j1) : 0.f;
+            if (R >= 2) o.l2 = j2 >= 0 ? scale * __ldg(row + j2) : 0.f;
+        }
+        if (lane == 31 || c4 == nc4 - 1) {
+            int j1 = 4 * c4 + 4, j2 = 4 * c4 + 5;
+            if (periodic) { if (j1 >= n) j1 -= n; if (j2 >= n) j2 -= n; }
+            o.r1 = j1 < n ? scale * __ldg(row + j1) : 0.f;
+            if (R >= 2) o.r2 = j2 < n ? scale * __ldg(row + j2) : 0.f;
+        }
+    }
+    return o;
+}
+
+// Deterministic block reduction of NE per-thread partial sums; thread 0 writes
+// partials[e * stride + slot].  The shuffle tree and the shared-memory tree have a fixed shape,
+// so the result depends only on the data, never on scheduling.
+template <int NE>
+__device__ __forceinline__ void block_reduce_store(const float (&acc)[NE], float* __restrict__ partials,
+                                                   int stride, int slot) {
+    __shared__ float red[NE][32];
+    const int tid = threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z);
+    const int nthreads = blockDim.x * blockDim.y * blockDim.z;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = (nthreads + 31) >> 5;
+#pragma unroll
+    for (int e = 0; e < NE; ++e) {
+        float v = acc[e];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(FULL_MASK, v, o);
+        if (lane == 0) red[e][warp] = v;
+    }
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+            float v = lane < nwarps ? red[e][lane] : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(FULL_MASK, v, o);
+            if (lane == 0) partials[(size_t)e * stride + slot] = v;
+        }
+    }
+}
+
+}  // namespace fpde

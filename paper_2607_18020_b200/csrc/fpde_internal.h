@@ -1,0 +1,48 @@
+// Host-side internal interface between the C-ABI layer (validation, registry) and the
+// per-operator launchers.  Not installed; the public interface is include/fpde.h.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace fpde {
+
+constexpr int MAX_F = 4;   // most fields / residuals of any operator
+constexpr int MAX_D = 4;   // most array axes
+
+// A validated problem, as the launchers see it.
+struct Problem {
+    int op;
+    int ndim;
+    int n[MAX_D];            // extents, memory order
+    double h[MAX_D];         // spacings
+    double coef[8];          // operator coefficients
+    const float* in[MAX_F];  // fwd: fields            bwd: fields
+    const float* aux[MAX_F]; // fwd: sources           bwd: upstream dL/dr_e
+    float* out[MAX_F];       // fwd: residuals         bwd: field gradients
+    double gscale[MAX_F];    // bwd only
+    float* partials;         // fwd: loss partial sums (NULL = no loss)
+    double* loss_out;        // fwd: device, E+1 doubles
+    int64_t rows;            // N_r
+    cudaStream_t stream;
+};
+
+// Number of loss partial sums (= work items) per residual field the forward kernel of this
+// operator produces for this grid.  Fixed by the grid alone, so the reduction order is too.
+int fwd_items(int op, const int* n);
+
+// Launchers: return cudaGetLastError() after queuing the kernels.
+cudaError_t launch_burgers_fwd(const Problem& p);
+cudaError_t launch_burgers_bwd(const Problem& p);
+cudaError_t launch_lap2d_fwd(const Problem& p);     // Poisson 2-D and Gray-Scott
+cudaError_t launch_lap2d_bwd(const Problem& p);
+cudaError_t launch_helmholtz_fwd(const Problem& p);
+cudaError_t launch_helmholtz_bwd(const Problem& p);
+cudaError_t launch_ns_fwd(const Problem& p);
+cudaError_t launch_ns_bwd(const Problem& p);
+
+// Final, fixed-order fp64 sum of the per-item partials: loss_out[e] = sum/N_r, loss_out[E] = total.
+cudaError_t launch_loss_finalize(const float* partials, int nitems, int nres, int64_t rows,
+                                 double* loss_out, cudaStream_t stream);
+
+}  // namespace fpde

@@ -1,0 +1,111 @@
+"""Host-side checks that need no GPU: the shared library builds, loads, exports every symbol the
+public header declares, and rejects bad arguments with the documented status codes."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2607_18020_b200 import binding as B
+from paper_2607_18020_b200 import build as fbuild
+from paper_2607_18020_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    fbuild.build()
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            txt = open(os.path.join(ROOT, "include", fn)).read()
+            txt = re.sub(r"/\*.*?\*/", "", txt, flags=re.S)
+            names |= set(re.findall(r"\b(fpde_[a-z0-9_]+)\s*\(", txt))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(B.LIB_PATH)
+    names = _declared_symbols()
+    assert {"fpde_fwd", "fpde_bwd", "fpde_op_info", "fpde_strerror", "fpde_workspace_bytes", "fpde_row_count"} <= names
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_registry():
+    expect = {W.BURGERS_1D_T: (2, 1, 0, 1, 1, 1), W.POISSON_2D: (2, 1, 1, 1, 0, 1), W.GRAYSCOTT_2D: (2, 2, 0, 2, 4, 1),
+              W.HELMHOLTZ_3D_O4: (3, 1, 1, 1, 1, 2), W.NS_3D_T: (4, 4, 0, 4, 1, 1)}
+    for op, e in expect.items():
+        i = B.op_info(op)
+        assert (i.ndim, i.nfields, i.nsources, i.nresiduals, i.ncoeffs, i.radius) == e
+        cfg = next(c for c in W.CONFIGS.values() if c["op"] == op)
+        assert [B.BC_IDS[b] for b in cfg["bc"]] == list(i.bc)[:i.ndim]
+        assert len(W.OP_META[op]["fields"]) == i.nfields and len(W.DEFAULT_COEFFS[op]) == i.ncoeffs
+    with pytest.raises(B.FpdeError):
+        B.op_info(99)
+    assert "unknown" in B.strerror(1234)
+
+
+def test_row_counts_and_workspace():
+    assert B.row_count(W.BURGERS_1D_T, (256, 128)) == 256 * 128
+    assert B.row_count(W.POISSON_2D, (1024, 1024)) == 1022 * 1022
+    assert B.row_count(W.GRAYSCOTT_2D, (4096, 4096)) == 4096 * 4096
+    assert B.row_count(W.HELMHOLTZ_3D_O4, (256, 256, 256)) == 252 ** 3
+    assert B.row_count(W.NS_3D_T, (128, 128, 128, 16)) == 128 ** 3 * 14
+    assert B.row_count(W.POISSON_2D, (1024, 1023)) == 0          # x4 rule
+    for name in W.CONFIG_ORDER:
+        c = W.CONFIGS[name]
+        assert 0 < B.workspace_bytes(c["op"], c["shape"]) < (64 << 20)
+    assert B.workspace_bytes(W.NS_3D_T, (2, 8, 8, 8)) == 0
+
+
+def test_argument_validation_without_a_gpu():
+    """Every check that precedes a launch; pointers are fake (never dereferenced on the host)."""
+    P = 0x1000
+    ok = dict(op=W.POISSON_2D, fields=[P], sources=[P], residuals=[P], loss_out=None, shape=(16, 16),
+              spacing=(0.1, 0.1), coeffs=(), bc=(W.INTERIOR, W.INTERIOR), workspace=None, workspace_bytes_=0,
+              stream=None)
+    def call(**kw):
+        a = dict(ok); a.update(kw)
+        return B.fwd_status(**a)
+    assert call(op=17) == 1
+    assert call(fields=None) == 2
+    assert call(fields=[None]) == 2
+    assert call(sources=None) == 2
+    assert call(residuals=[None]) == 2
+    assert call(ndim=3) == 3
+    assert call(shape=(2, 16)) == 4
+    assert call(shape=(16, 18)) == 4
+    assert call(shape=(1 << 16, 1 << 16)) == 4
+    assert call(fields=[P + 4]) == 5
+    assert call(spacing=(0.1, 0.0)) == 6
+    assert call(spacing=(float("nan"), 0.1)) == 6
+    assert call(coeffs=(1.0,)) == 7
+    assert call(bc=(W.PERIODIC, W.INTERIOR)) == 8
+    assert call(loss_out=P, workspace=None) == 9
+    assert call(loss_out=P, workspace=P, workspace_bytes_=2) == 9
+    assert call(op=W.HELMHOLTZ_3D_O4, shape=(4, 8, 8), spacing=(.1, .1, .1), coeffs=(1.0,), bc=(W.INTERIOR,) * 3) == 4
+    assert call(op=W.BURGERS_1D_T, shape=(3, 8), coeffs=(0.1,), bc=(W.ONE_SIDED,) * 2, sources=None) == 4
+    okb = dict(op=W.GRAYSCOTT_2D, fields=[P, P], gres=[P, P], gscale=None, gfields=[P, P], shape=(8, 8),
+               spacing=(0.1, 0.1), coeffs=(1, 1, 1, 1), bc=(W.PERIODIC, W.PERIODIC), workspace=None,
+               workspace_bytes_=0, stream=None)
+    def callb(**kw):
+        a = dict(okb); a.update(kw)
+        return B.bwd_status(**a)
+    assert callb(gres=None) == 2
+    assert callb(gfields=[P, None]) == 2
+    assert callb(gres=[P, P + 8]) == 5
+    assert callb(gscale=(1.0, float("inf"))) == 6
+    assert callb(coeffs=(1, 1, 1)) == 7
+    assert callb(bc=(W.PERIODIC, W.ONE_SIDED)) == 8
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    monkeypatch.setattr(B, "_lib", None)
+    with pytest.raises(RuntimeError, match="no fallback"):
+        B.lib()

@@ -1,0 +1,137 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded fp32 inputs.  Tolerances: relative L2 <= 1e-5 and infinity-norm-relative <= 1e-4 per
+output array, |dL|/L <= 1e-5; zero-pattern (nodes without a row) exact."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2607_18020_b200 import binding as B
+from paper_2607_18020_b200 import workloads as W
+
+from gpu_util import LOSS_TOL, assert_close, run_bwd, run_fwd, to_dev
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+# (config name, shape or None for the full configuration)
+MEDIUM = [
+    ("burgers_256x128", None),
+    ("burgers_256x128", (37, 23)),
+    ("poisson_1024", None),
+    ("poisson_1024", (203, 300)),          # several row chunks and column blocks, ragged tails
+    ("grayscott_4096", (1000, 1032)),
+    ("helmholtz_256", (70, 45, 136)),
+    ("ns_tgv_128x16", (36, 21, 20, 16)),
+]
+TINY = [
+    ("burgers_256x128", (4, 4)),
+    ("burgers_256x128", (5, 9)),
+    ("poisson_1024", (3, 4)),
+    ("poisson_1024", (36, 40)),
+    ("grayscott_4096", (3, 4)),
+    ("grayscott_4096", (17, 12)),
+    ("helmholtz_256", (5, 5, 8)),
+    ("helmholtz_256", (12, 20, 24)),
+    ("ns_tgv_128x16", (3, 3, 3, 4)),
+    ("ns_tgv_128x16", (8, 12, 16, 8)),
+    ("ns_tgv_128x16", (5, 6, 7, 12)),
+]
+FULL = [
+    ("grayscott_4096", None),
+    ("helmholtz_256", None),
+    ("ns_tgv_128x16", None),
+]
+
+
+def _check_case(w, tag):
+    R_ref, loss_ref, g_ref, rows = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    assert rows == B.row_count(w.op, w.shape)
+    fields, sources, res, loss = run_fwd(torch, w)
+    for e, (r, rr) in enumerate(zip(res, R_ref)):
+        got = r.view.cpu().numpy()
+        assert_close(got, rr, "%s residual %d" % (tag, e))
+        assert np.array_equal(got == 0, rr == 0) or np.all(got[rr == 0] == 0), "%s: row-less nodes must be 0" % tag
+    L = loss.cpu().numpy()
+    assert np.all(np.abs(L - loss_ref) <= LOSS_TOL * np.abs(loss_ref) + 1e-300), (tag, L, loss_ref)
+    # gradient of the fused loss: upstream = the residual arrays the forward wrote, scale 2/N_r
+    grads = run_bwd(torch, w, fields, [r.view for r in res], [2.0 / rows] * len(res))
+    for f, (g, gr) in enumerate(zip(grads, g_ref)):
+        assert_close(g.view.cpu().numpy(), gr, "%s gradient %d" % (tag, f))
+
+
+@pytest.mark.parametrize("name,shape", MEDIUM)
+def test_config_fields(name, shape):
+    _check_case(W.make(name, seed=42, shape=shape), "%s%s" % (name, shape or ""))
+
+
+@pytest.mark.parametrize("name,shape", TINY)
+@pytest.mark.parametrize("seed", [42, 43, 44, 45, 46])
+def test_randn_fields_tiny(name, shape, seed):
+    _check_case(W.make(name, seed=seed, shape=shape, kind="randn"), "%s%s randn seed %d" % (name, shape, seed))
+
+
+@pytest.mark.parametrize("name,shape", MEDIUM[1:])
+def test_adjoint_alone_random_upstream(name, shape):
+    """The adjoint on arbitrary upstream arrays (not a residual): non-zero entries at nodes
+    without a row must be ignored, and gscale applied."""
+    w = W.make(name, seed=44, shape=shape, kind="randn")
+    G = W.random_sensitivities(w, seed=7)
+    gscale = [0.5 + 0.25 * e for e in range(len(G))]
+    ref = oracle.bwd(w.op, w.fields, [s * g.astype(np.float64) for s, g in zip(gscale, G)], w.shape, w.spacing, w.coeffs)
+    fields = to_dev(torch, w.fields)
+    grads = run_bwd(torch, w, fields, to_dev(torch, G), gscale)
+    for f, (g, gr) in enumerate(zip(grads, ref)):
+        assert_close(g.view.cpu().numpy(), gr, "%s adjoint %d" % (name, f))
+
+
+def test_unequal_spacing():
+    for name, shape, h in [("poisson_1024", (20, 24), (0.3, 0.07)), ("helmholtz_256", (9, 10, 12), (0.2, 0.15, 0.11)),
+                           ("ns_tgv_128x16", (5, 6, 7, 8), (0.3, 0.2, 0.25, 0.1)), ("grayscott_4096", (9, 8), (0.01, 0.02)),
+                           ("burgers_256x128", (11, 7), (0.05, 0.02))]:
+        _check_case(W.make(name, seed=45, shape=shape, kind="randn", spacing=h), name + " unequal spacing")
+
+
+@pytest.mark.parametrize("name,shape", FULL)
+def test_full_size_configs(name, shape):
+    """BASELINE's full sizes in the launch configuration the bench times; the C oracle is fast
+    enough to check every element."""
+    _check_case(W.make(name, seed=42), name + " full size")
+
+
+def test_loss_is_bitwise_reproducible():
+    w = W.make("ns_tgv_128x16", seed=42, shape=(32, 32, 32, 16))
+    fields = to_dev(torch, w.fields)
+    res = [torch.empty(w.shape, dtype=torch.float32, device="cuda") for _ in range(4)]
+    ws = torch.empty(B.workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+    seen = set()
+    for _ in range(20):
+        loss = torch.zeros(5, dtype=torch.float64, device="cuda")
+        B.fpde_fwd(w.op, fields, [], res, loss, w.shape, w.spacing, w.coeffs, w.bc, ws)
+        torch.cuda.synchronize()
+        seen.add(loss.cpu().numpy().tobytes())
+    assert len(seen) == 1
+
+
+def test_loss_can_be_skipped_and_stream_is_honoured():
+    w = W.make("grayscott_4096", seed=42, shape=(64, 64))
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        fields, sources, res, loss = run_fwd(torch, w, with_loss=False, stream=s)
+    R_ref, _, _ = oracle.fwd(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    assert loss is None
+    for r, rr in zip(res, R_ref):
+        assert_close(r.view.cpu().numpy(), rr, "no-loss forward")
+
+
+def test_invalid_arguments_launch_nothing():
+    w = W.make("poisson_1024", seed=42, shape=(16, 16))
+    fields = to_dev(torch, w.fields); sources = to_dev(torch, w.sources)
+    out = torch.full(w.shape, 3.0, dtype=torch.float32, device="cuda")
+    loss = torch.full((2,), -1.0, dtype=torch.float64, device="cuda")
+    ws = torch.empty(B.workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+    st = B.fwd_status(w.op, fields, sources, [out], loss, w.shape, w.spacing, w.coeffs, w.bc, ws, 8, None)
+    assert st == 9      # workspace too small
+    st = B.fwd_status(w.op, fields, sources, [out.view(-1)[1:].data_ptr()], None, w.shape, w.spacing, w.coeffs, w.bc, None, 0, None)
+    assert st == 5      # misaligned
+    torch.cuda.synchronize()
+    assert bool((out == 3.0).all()) and bool((loss == -1.0).all())
