@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the fused finite-difference PDE-residual hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl fpde|reference]
+
+One "step" = one fused forward (all residual fields + loss) plus one adjoint (gradient of that
+loss, boundary correction included) over one synthetic grid, through the C ABI.  The default
+workload is the 3-D unsteady Navier-Stokes (Taylor-Green) configuration, 128^3 x 16 space-time
+points, four fields: the paper's headline operator and the largest configuration; its 2.5 GB of
+per-step traffic is far beyond L2, so back-to-back steps need no cache flush.
+
+Prints ONE JSON line (rank 0).  `value` is grid points per second over all GPUs (replicas: the
+path has no exchange step, so N GPUs run N independent grids, weak scaling).
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2607_18020_b200 import workloads as W
+
+METRIC = "grid-points/s for fused fwd+bwd residual loss"
+UNIT = "grid-points/s"
+DEFAULT_WORKLOAD = "ns_tgv_128x16"
+
+# Algorithmic bytes per grid point (fp32, every array touched once): forward reads fields and
+# sources and writes residuals; the adjoint reads the upstream arrays plus the fields its
+# Jacobian needs and writes one gradient per field.
+ALGO_BYTES = {                      # op: (fwd, bwd)
+    W.BURGERS_1D_T: (8, 12),
+    W.POISSON_2D: (12, 8),
+    W.GRAYSCOTT_2D: (16, 24),
+    W.HELMHOLTZ_3D_O4: (12, 8),
+    W.NS_3D_T: (32, 44),
+}
+KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
+    W.BURGERS_1D_T: ("burgers_fwd_kernel", "burgers_bwd_kernel"),
+    W.POISSON_2D: ("lap2d_kernel<PoissonFwd>", "lap2d_kernel<PoissonBwd>"),
+    W.GRAYSCOTT_2D: ("lap2d_kernel<GrayScottFwd>", "lap2d_kernel<GrayScottBwd>"),
+    W.HELMHOLTZ_3D_O4: ("star3d_kernel<fwd>", "star3d_kernel<bwd>"),
+    W.NS_3D_T: ("ns_fwd_kernel", "ns_bwd_kernel"),
+}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; None where no capture has been taken yet.
+NCU_TRAFFIC_BYTES = {
+}
+FALLBACK_HBM_GBS = 6650.0
+LAUNCHES_PER_STEP = 3               # forward kernel, loss finalise, adjoint kernel
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# clocks: sampled through NVML (read-only) while the timed region runs
+# ------------------------------------------------------------------------------------------
+_REASONS = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+            0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+
+class ClockSampler:
+    def __init__(self, torch, device_index: int, period_s: float = 0.004):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            p = torch.cuda.get_device_properties(device_index)
+            bus = "%08x:%02x:%02x.0" % (p.pci_domain_id, p.pci_bus_id, p.pci_device_id)
+            self._h = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+            self._nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as exc:      # NVML unavailable: report that instead of numbers
+            self.error = repr(exc)
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in _REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self):
+        if self._h is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "error": getattr(self, "error", "nvml unavailable")}
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+def oracle_sample(name: str, planes: int, seed: int = 42):
+    """A bounded sample of a workload: its first `planes` slices along the slowest axis, taken
+    as a grid of its own (same spacings, same recipe)."""
+    cfg = W.CONFIGS[name]
+    shape = list(cfg["shape"])
+    planes = max(5, min(shape[0], planes))
+    full = W.make(name, seed=seed, shape=[planes] + shape[1:], spacing=_spacing_of(name))
+    return full
+
+
+def _spacing_of(name):
+    cfg = W.CONFIGS[name]
+    hs = []
+    for n, (lo, hi), b in zip(cfg["shape"], cfg["domain"], cfg["bc"]):
+        hs.append((hi - lo) / n if b == W.PERIODIC else (hi - lo) / (n - 1))
+    return tuple(hs)
+
+
+def time_oracle(w, reps: int):
+    import oracle
+    best = float("inf")
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+        best = min(best, time.perf_counter() - t0)
+    return best
+
+
+def cpu_baseline(name: str):
+    """The oracle as it stands (single thread), fwd + bwd, on a sample of about 10-30 s of work."""
+    cfg_shape = W.CONFIGS[name]["shape"]
+    per_plane = int(np.prod(cfg_shape[1:]))
+    planes = max(5, min(cfg_shape[0], int(8.0e6 // per_plane) or 1))
+    w = oracle_sample(name, planes)
+    t = time_oracle(w, 3)
+    return {"value": w.npoints / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "first %d of %d slices along axis 0 of %s (%d points), fp64 fwd+bwd incl. loss, best of 3"
+                      % (w.shape[0], cfg_shape[0], name, w.npoints),
+            "seconds": t}
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle on a bounded sample, one sample pass per step."""
+    if rank != 0:
+        return
+    name = args.workload
+    cfg_shape = W.CONFIGS[name]["shape"]
+    per_plane = int(np.prod(cfg_shape[1:]))
+    # keep the whole run near two minutes whatever K and W are (the oracle does ~2.5e6 points/s)
+    budget_points = 120.0 * 2.5e6 / max(1, args.steps + args.warmup)
+    planes = max(5, min(cfg_shape[0], int(budget_points // per_plane)))
+    w = oracle_sample(name, planes)
+    import oracle
+    for _ in range(args.warmup):
+        oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    dt = time.perf_counter() - t0
+    value = w.npoints * args.steps / dt
+    sample = "first %d of %d slices along axis 0 (%d points per step)" % (w.shape[0], cfg_shape[0], w.npoints)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": name, "shape": list(w.shape), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------------------------------
+# GPU legs
+# ------------------------------------------------------------------------------------------
+class DeviceProblem:
+    def __init__(self, torch, B, w):
+        self.w, self.B, self.torch = w, B, torch
+        self.fields = [torch.from_numpy(f).cuda() for f in w.fields]
+        self.sources = [torch.from_numpy(s).cuda() for s in w.sources]
+        ne = len(W.OP_META[w.op]["residuals"])
+        self.res = [torch.empty(w.shape, dtype=torch.float32, device="cuda") for _ in range(ne)]
+        self.grads = [torch.empty(w.shape, dtype=torch.float32, device="cuda") for _ in w.fields]
+        self.loss = torch.zeros(ne + 1, dtype=torch.float64, device="cuda")
+        self.ws = torch.empty(B.workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+        self.gscale = [2.0 / B.row_count(w.op, w.shape)] * ne
+
+    def fwd(self):
+        w = self.w
+        self.B.fpde_fwd(w.op, self.fields, self.sources, self.res, self.loss, w.shape, w.spacing, w.coeffs, w.bc, self.ws)
+
+    def bwd(self):
+        w = self.w
+        self.B.fpde_bwd(w.op, self.fields, self.res, self.gscale, self.grads, w.shape, w.spacing, w.coeffs, w.bc)
+
+
+def timed_steps(torch, prob, steps, warmup, barrier, flush=None):
+    """K back-to-back steps between two events; inner events give per-call durations."""
+    for _ in range(warmup):
+        prob.fwd(); prob.bwd()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    barrier(); torch.cuda.synchronize()
+    for k in range(steps):
+        if flush is not None:
+            flush.fill_(k)
+        ev[k][0].record(); prob.fwd(); ev[k][1].record(); prob.bwd(); ev[k][2].record()
+    torch.cuda.synchronize(); barrier()
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    return total_ms, fwd_ms, bwd_ms
+
+
+def e2e_steps(torch, B, w, steps, warmup, barrier):
+    """The same step from pinned HOST buffers through fpde_loss_grad_host: per step, H2D of every
+    field/source, forward, adjoint, D2H of every gradient and of the loss, then a stream sync (the
+    caller reads the loss)."""
+    hf = [torch.from_numpy(f).pin_memory() for f in w.fields]
+    hs = [torch.from_numpy(s).pin_memory() for s in w.sources]
+    hg = [torch.empty(w.shape, dtype=torch.float32).pin_memory() for _ in w.fields]
+    ne = len(W.OP_META[w.op]["residuals"])
+    hl = torch.zeros(ne + 1, dtype=torch.float64).pin_memory()
+    arena = torch.empty(B.host_arena_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.fpde_loss_grad_host(w.op, hf, hs, hg, hl, w.shape, w.spacing, w.coeffs, w.bc, arena)
+        stream.synchronize()
+        return float(hl[-1])
+
+    for _ in range(warmup):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        loss = step()
+    e1.record()
+    torch.cuda.synchronize(); barrier()
+    nbytes = w.npoints * 4
+    return e0.elapsed_time(e1), nbytes * (len(hf) + len(hs)), nbytes * len(hg) + 8 * (ne + 1), loss
+
+
+def config_line(torch, B, name, steps, warmup, peak):
+    """Secondary figures for one configuration: per-call medians with an L2 flush (a 256 MiB
+    write) before every step, so small grids are measured cold like large ones."""
+    w = W.make(name, seed=42)
+    prob = DeviceProblem(torch, B, w)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    _, f_ms, b_ms = timed_steps(torch, prob, steps, warmup, lambda: None, flush=flush)
+    fm, bm = statistics.median(f_ms), statistics.median(b_ms)
+    fb, bb = ALGO_BYTES[w.op]
+    N = w.npoints
+    out = {"shape": list(w.shape), "points": N, "ms_fwd": fm, "ms_bwd": bm,
+           "points_per_s": N / ((fm + bm) * 1e-3),
+           "gbs_fwd": fb * N / (fm * 1e-3) / 1e9, "gbs_bwd": bb * N / (bm * 1e-3) / 1e9,
+           "gbs_pair": (fb + bb) * N / ((fm + bm) * 1e-3) / 1e9}
+    out["frac_pair"] = out["gbs_pair"] / peak
+    del prob, flush
+    torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(W.CONFIG_ORDER))
+    ap.add_argument("--impl", default="fpde", choices=["fpde", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip per-config figures and the CPU baseline")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--shape", default=None, help="override the grid extents, e.g. 64,128,128,16 (profiling runs)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "fpde" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    from paper_2607_18020_b200 import binding as B
+    B.lib()                                   # fail loudly if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peak, peak_src = measured_peak()
+    shape = [int(x) for x in args.shape.split(",")] if args.shape else None
+    w = W.make(args.workload, seed=42 + rank, shape=shape,
+               spacing=_spacing_of(args.workload) if shape else None)
+    prob = DeviceProblem(torch, B, w)
+    N = w.npoints
+
+    sampler = ClockSampler(torch, local_rank)
+    sampler.start()
+    total_ms, fwd_ms, bwd_ms = timed_steps(torch, prob, args.steps, args.warmup, barrier)
+    sampler.stop()
+    total_ms = max_over_ranks(total_ms)
+    value = world * N * args.steps / (total_ms * 1e-3)
+
+    e2e_k = max(1, min(args.steps, 20))
+    if args.no_e2e:
+        e2e_ms, h2d, d2h = float("nan"), 0, 0
+    else:
+        e2e_ms, h2d, d2h, _ = e2e_steps(torch, B, w, e2e_k, 3, barrier)
+    e2e_ms = max_over_ranks(e2e_ms)
+    e2e_value = world * N * e2e_k / (e2e_ms * 1e-3)
+
+    fb, bb = ALGO_BYTES[w.op]
+    f_avg, b_avg = sum(fwd_ms) / len(fwd_ms), sum(bwd_ms) / len(bwd_ms)
+    dom = 1 if b_avg >= f_avg else 0
+    dom_bytes = (fb, bb)[dom] * N
+    dom_ms = (f_avg, b_avg)[dom]
+    dom_name = KERNEL_NAMES[w.op][dom]
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_src,
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom_name)),
+                "algorithmic_bytes": dom_bytes, "avg_ms": dom_ms,
+                "other_kernel": {"kernel": KERNEL_NAMES[w.op][1 - dom], "avg_ms": (f_avg, b_avg)[1 - dom],
+                                 "note": "forward figure includes the one-block loss finalise launch",
+                                 "achieved": (fb, bb)[1 - dom] * N / ((f_avg, b_avg)[1 - dom] * 1e-3) / 1e9},
+                "pair_achieved": (fb + bb) * N * args.steps / (total_ms * 1e-3) / 1e9,
+                "pair_frac": (fb + bb) * N * args.steps / (total_ms * 1e-3) / 1e9 / peak}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "operator": w.op, "shape": list(w.shape), "points": N,
+                   "fields": len(w.fields), "parallelism": "replicas x%d (no exchange step)" % world,
+                   "l2": "per-step traffic %.0f MB >> L2, no flush needed" % ((fb + bb) * N / 1e6)
+                         if (fb + bb) * N > (256 << 20) else "working set fits L2: warm-cache number"},
+        "clocks": sampler.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_k, "ms_per_step": e2e_ms / e2e_k,
+                "what": "fpde_loss_grad_host from pinned host buffers: H2D fields, fwd, bwd, D2H gradients + loss, sync"},
+        "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        "roofline": roofline,
+        "loss": float(prob.loss[-1].item()),
+    }
+    if world == 1 and not args.no_extras:
+        del prob
+        torch.cuda.empty_cache()
+        line["per_config"] = {name: config_line(torch, B, name, 30, 5, peak) for name in W.CONFIG_ORDER}
+        line["cpu_baseline"] = cpu_baseline(args.workload)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -167,6 +167,35 @@ int fpde_bwd(int op,
              void* workspace, size_t workspace_bytes,
              void* stream);
 
+/*
+ * Loss gradient from HOST buffers in one call: copies the fields (and sources) to the device,
+ * runs fpde_fwd, then fpde_bwd with the upstream sensitivities of the mean-square loss,
+ * G_e = (2/N_r) r_e (Section 2.2: the operator receives G = dL/dres from the loss), and copies
+ * dL/dfield and the loss vector back.  Everything is queued on `stream`; the host buffers may be
+ * read / written until the stream has been synchronised (use page-locked memory for the copies to
+ * run asynchronously).
+ *
+ *   h_fields   host array of nfields  HOST pointers, N floats each, read only
+ *   h_sources  host array of nsources HOST pointers (may be NULL if nsources = 0)
+ *   h_gfields  host array of nfields  HOST pointers, N floats each, overwritten with dL/dfield
+ *   h_loss     HOST, nresiduals+1 doubles, overwritten with L_0..L_{E-1} and their sum
+ *   d_arena    DEVICE scratch of at least fpde_host_arena_bytes() bytes, 256-byte aligned, owned
+ *              by the caller (staging for fields, sources, residuals, gradients, loss, workspace)
+ * Same status codes as fpde_fwd / fpde_bwd; FPDE_ERR_WORKSPACE if the arena is too small.
+ */
+size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape);
+int fpde_loss_grad_host(int op,
+                        const float* const* h_fields,
+                        const float* const* h_sources,
+                        float* const* h_gfields,
+                        double* h_loss,
+                        int ndim, const int64_t* shape,
+                        const double* spacing,
+                        const double* coeffs, int ncoeffs,
+                        const int* bc,
+                        void* d_arena, size_t arena_bytes,
+                        void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -64,6 +64,14 @@ def lib():
                                ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fpde_host_arena_bytes.restype = ctypes.c_size_t
+        L.fpde_host_arena_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_loss_grad_host.restype = ctypes.c_int
+        L.fpde_loss_grad_host.argtypes = [ctypes.c_int, vpp, vpp, vpp, ctypes.c_void_p, ctypes.c_int,
+                                          ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                          ctypes.POINTER(ctypes.c_double), ctypes.c_int,
+                                          ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_size_t,
+                                          ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -185,3 +193,29 @@ def fpde_bwd(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, work
                     _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_bwd")
+
+
+def host_arena_bytes(op, shape) -> int:
+    return int(lib().fpde_host_arena_bytes(_opid(op), len(shape), _i64(shape)))
+
+
+def loss_grad_host_status(op, h_fields, h_sources, h_gfields, h_loss, shape, spacing, coeffs, bc, arena,
+                          arena_bytes, stream) -> int:
+    return lib().fpde_loss_grad_host(_opid(op),
+                                     _ptr_array(_dev_ptrs(h_fields)) if h_fields is not None else None,
+                                     _ptr_array(_dev_ptrs(h_sources)) if h_sources is not None else None,
+                                     _ptr_array(_dev_ptrs(h_gfields)) if h_gfields is not None else None,
+                                     _dev_ptrs([h_loss])[0] if h_loss is not None else None,
+                                     len(shape), _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                                     _dev_ptrs([arena])[0] if arena is not None else None, int(arena_bytes), stream)
+
+
+def fpde_loss_grad_host(op, h_fields, h_sources, h_gfields, h_loss, shape, spacing, coeffs, bc, arena, stream=None):
+    """Loss and dL/dfield from HOST tensors (pinned CPU tensors recommended): H2D copies, forward,
+    adjoint and D2H copies are queued on `stream`; synchronise it before reading the results.
+    `arena` is a CUDA tensor of at least host_arena_bytes(op, shape) bytes."""
+    ab = arena.numel() * arena.element_size()
+    st = loss_grad_host_status(op, h_fields, h_sources, h_gfields, h_loss, shape, spacing, coeffs, bc, arena, ab,
+                               _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_loss_grad_host")

@@ -250,4 +250,65 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
     return ce == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
 }
 
+static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+
+size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape) {
+    int64_t N = 0;
+    if (check_shape(op, ndim, shape, nullptr, &N, nullptr) != FPDE_OK) return 0;
+    const OpEntry& e = REGISTRY[op];
+    const size_t arr = round256((size_t)N * sizeof(float));
+    return arr * (size_t)(2 * e.nf + e.ns + e.ne) + round256((e.ne + 1) * sizeof(double))
+         + fpde_workspace_bytes(op, ndim, shape);
+}
+
+int fpde_loss_grad_host(int op, const float* const* h_fields, const float* const* h_sources,
+                        float* const* h_gfields, double* h_loss, int ndim, const int64_t* shape,
+                        const double* spacing, const double* coeffs, int ncoeffs, const int* bc,
+                        void* d_arena, size_t arena_bytes, void* stream) {
+    int64_t N = 0, rows = 0;
+    int st = check_shape(op, ndim, shape, nullptr, &N, &rows);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!h_fields || !h_gfields || !h_loss || (e.ns > 0 && !h_sources)) return FPDE_ERR_NULL;
+    for (int f = 0; f < e.nf; ++f) if (!h_fields[f] || !h_gfields[f]) return FPDE_ERR_NULL;
+    for (int s = 0; s < e.ns; ++s) if (!h_sources[s]) return FPDE_ERR_NULL;
+    if (!d_arena || (reinterpret_cast<uintptr_t>(d_arena) & 255u) != 0 ||
+        arena_bytes < fpde_host_arena_bytes(op, ndim, shape))
+        return FPDE_ERR_WORKSPACE;
+    // validate the remaining host arguments before the first copy is queued
+    if (!spacing || !bc) return FPDE_ERR_NULL;
+    if (ncoeffs != e.nc) return FPDE_ERR_COEFF_COUNT;
+    if (e.nc > 0 && !coeffs) return FPDE_ERR_NULL;
+    for (int a = 0; a < ndim; ++a) {
+        if (!(spacing[a] > 0.0) || !std::isfinite(spacing[a])) return FPDE_ERR_SPACING;
+        if (bc[a] != e.bc[a]) return FPDE_ERR_BC;
+    }
+    const size_t bytes = (size_t)N * sizeof(float), arr = round256(bytes);
+    char* base = static_cast<char*>(d_arena);
+    float* d_f[MAX_F]; float* d_s[MAX_F]; float* d_r[MAX_F]; float* d_g[MAX_F];
+    for (int f = 0; f < e.nf; ++f) { d_f[f] = reinterpret_cast<float*>(base); base += arr; }
+    for (int s = 0; s < e.ns; ++s) { d_s[s] = reinterpret_cast<float*>(base); base += arr; }
+    for (int r = 0; r < e.ne; ++r) { d_r[r] = reinterpret_cast<float*>(base); base += arr; }
+    for (int f = 0; f < e.nf; ++f) { d_g[f] = reinterpret_cast<float*>(base); base += arr; }
+    double* d_loss = reinterpret_cast<double*>(base); base += round256((e.ne + 1) * sizeof(double));
+    void* d_ws = base;
+    const size_t ws_bytes = fpde_workspace_bytes(op, ndim, shape);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    for (int f = 0; f < e.nf; ++f)
+        if (cudaMemcpyAsync(d_f[f], h_fields[f], bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FPDE_ERR_CUDA;
+    for (int s = 0; s < e.ns; ++s)
+        if (cudaMemcpyAsync(d_s[s], h_sources[s], bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FPDE_ERR_CUDA;
+    st = fpde_fwd(op, d_f, d_s, d_r, d_loss, ndim, shape, spacing, coeffs, ncoeffs, bc, d_ws, ws_bytes, stream);
+    if (st != FPDE_OK) return st;
+    double gscale[MAX_F];
+    for (int r = 0; r < e.ne; ++r) gscale[r] = 2.0 / (double)rows;
+    st = fpde_bwd(op, d_f, d_r, gscale, d_g, ndim, shape, spacing, coeffs, ncoeffs, bc, nullptr, 0, stream);
+    if (st != FPDE_OK) return st;
+    for (int f = 0; f < e.nf; ++f)
+        if (cudaMemcpyAsync(h_gfields[f], d_g[f], bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return FPDE_ERR_CUDA;
+    if (cudaMemcpyAsync(h_loss, d_loss, (e.ne + 1) * sizeof(double), cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+        return FPDE_ERR_CUDA;
+    return FPDE_OK;
+}
+
 }  // extern "C"

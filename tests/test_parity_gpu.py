@@ -129,9 +129,27 @@ def test_invalid_arguments_launch_nothing():
     out = torch.full(w.shape, 3.0, dtype=torch.float32, device="cuda")
     loss = torch.full((2,), -1.0, dtype=torch.float64, device="cuda")
     ws = torch.empty(B.workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
-    st = B.fwd_status(w.op, fields, sources, [out], loss, w.shape, w.spacing, w.coeffs, w.bc, ws, 8, None)
+    st = B.fwd_status(w.op, fields, sources, [out], loss, w.shape, w.spacing, w.coeffs, w.bc, ws, 2, None)
     assert st == 9      # workspace too small
     st = B.fwd_status(w.op, fields, sources, [out.view(-1)[1:].data_ptr()], None, w.shape, w.spacing, w.coeffs, w.bc, None, 0, None)
     assert st == 5      # misaligned
     torch.cuda.synchronize()
     assert bool((out == 3.0).all()) and bool((loss == -1.0).all())
+
+
+def test_loss_grad_from_host_buffers():
+    """The host-buffer entry point (copies + forward + adjoint in one call) against the oracle."""
+    w = W.make("ns_tgv_128x16", seed=43, shape=(12, 10, 8, 8))
+    _, loss_ref, g_ref, rows = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    hf = [torch.from_numpy(f).pin_memory() for f in w.fields]
+    hg = [torch.empty(w.shape, dtype=torch.float32).pin_memory() for _ in w.fields]
+    hl = torch.zeros(5, dtype=torch.float64).pin_memory()
+    arena = torch.empty(B.host_arena_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+    assert arena.data_ptr() % 256 == 0
+    B.fpde_loss_grad_host(w.op, hf, [], hg, hl, w.shape, w.spacing, w.coeffs, w.bc, arena)
+    torch.cuda.synchronize()
+    assert np.all(np.abs(hl.numpy() - loss_ref) <= LOSS_TOL * np.abs(loss_ref))
+    for f, (g, gr) in enumerate(zip(hg, g_ref)):
+        assert_close(g.numpy(), gr, "host entry gradient %d" % f)
+    st = B.loss_grad_host_status(w.op, hf, [], hg, hl, w.shape, w.spacing, w.coeffs, w.bc, arena, 1024, None)
+    assert st == 9
