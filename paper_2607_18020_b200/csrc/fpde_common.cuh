@@ -27,6 +27,39 @@ __device__ __forceinline__ float sq4(float4 a) {
     return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Packed fp32x2 arithmetic (sm_100 FFMA2 / FADD2 / FMUL2): one instruction per two lanes of a
+// thread's float4, which halves the issue slots the stencil arithmetic takes.  Per component
+// the results are those of fmaf / add / mul in round-to-nearest.
+// ------------------------------------------------------------------------------------------
+struct V4 { float2 lo, hi; };           // a float4 as two register-aligned pairs
+
+__device__ __forceinline__ float2 splat2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) {            // a - b, exactly rounded once
+    return __ffma2_rn(b, make_float2(-1.f, -1.f), a);
+}
+__device__ __forceinline__ V4 ldv4(const float* p) {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    V4 v; v.lo = make_float2(t.x, t.y); v.hi = make_float2(t.z, t.w);
+    return v;
+}
+__device__ __forceinline__ void stv4(float* p, float2 lo, float2 hi) {
+    *reinterpret_cast<float4*>(p) = make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ V4 v4zero() { V4 v; v.lo = make_float2(0.f, 0.f); v.hi = v.lo; return v; }
+__device__ __forceinline__ V4 v4add(V4 a, V4 b) { V4 r; r.lo = add2(a.lo, b.lo); r.hi = add2(a.hi, b.hi); return r; }
+__device__ __forceinline__ V4 v4sub(V4 a, V4 b) { V4 r; r.lo = sub2(a.lo, b.lo); r.hi = sub2(a.hi, b.hi); return r; }
+__device__ __forceinline__ V4 v4mul(V4 a, float2 s) { V4 r; r.lo = mul2(a.lo, s); r.hi = mul2(a.hi, s); return r; }
+__device__ __forceinline__ V4 v4mulv(V4 a, V4 b) { V4 r; r.lo = mul2(a.lo, b.lo); r.hi = mul2(a.hi, b.hi); return r; }
+// a * s + c
+__device__ __forceinline__ V4 v4fma(V4 a, float2 s, V4 c) { V4 r; r.lo = fma2(a.lo, s, c.lo); r.hi = fma2(a.hi, s, c.hi); return r; }
+// a * b + c
+__device__ __forceinline__ V4 v4fmav(V4 a, V4 b, V4 c) { V4 r; r.lo = fma2(a.lo, b.lo, c.lo); r.hi = fma2(a.hi, b.hi, c.hi); return r; }
+
 // Values one and two elements to the left / right of a thread's float4 along the contiguous
 // axis.  Inside a warp they come from the neighbouring lane's registers; the first and last
 // lane (and the first / last float4 of a row) fetch them from global memory, wrapped around

@@ -10,10 +10,18 @@
 //
 // Kernel shape (both directions): a thread owns one float4 (four consecutive t of one z) of a
 // (y,row) tile and marches along x, the slowest axis, with a three-plane register window per
-// array; y+-1 and z+-1 neighbours of the current plane are read through L1, t+-1 neighbours
-// come from the adjacent lanes' registers.  Nodes at the first / last t carry no row: the
-// forward pass writes 0 there, the adjoint treats the upstream arrays as 0 there (omitted
-// neighbours, Appendix A.4), which is the boundary-gradient correction of the t axis.
+// array (rotated by unrolling, not by moves); y+-1 and z+-1 neighbours of the current plane are
+// read through L1, t+-1 neighbours come from the adjacent lanes' registers.  Arithmetic is
+// packed fp32x2.  Second differences are formed as (q[-1]-q[0]) + (q[+1]-q[0]) before scaling:
+// here the viscous term is small against the other terms and must not carry the rounding of
+// the large centre value.
+//
+// Nodes at the first / last t carry no row: the forward pass writes 0 there; in the adjoint the
+// upstream arrays count as 0 there (omitted neighbours, Appendix A.4).  Every spatial read of an
+// output node happens at the node's own t, so that rule only changes (i) the t-neighbour of the
+// nodes next to the two end planes and (ii) the end planes themselves, where only the
+// transposed d_t term survives: that is the boundary-gradient correction of this operator, and
+// it is applied as a fix-up of two lanes instead of masking every load.
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
 
@@ -24,23 +32,41 @@ namespace fpde {
 
 struct NsParams {
     const float* f[4];    // u, v, w, p
-    const float* g[4];    // adjoint: upstream G of mom_x, mom_y, mom_z, continuity
+    const float* g[4];    // adjoint: upstream arrays of mom_x, mom_y, mom_z, continuity
     float* out[4];
-    float gs[4];
     int n0, n1, n3;       // x, y extents; t extent
     int C, C4, nt4;       // row length in floats / float4, float4 per z
     int planes_per_item, ncb, nmb, nitems;
-    float ihx, ihy, ihz, iht;       // 1/(2h)
-    float ihxx, ihyy, ihzz;         // 1/h^2
-    float nu;
+    // forward constants, splatted
+    float2 ih[3];         // 1/(2 h_a)
+    float2 iht;           // 1/(2 dt)
+    float2 nv[3];         // -nu / h_a^2
+    // adjoint constants (upstream scales folded in), splatted
+    float2 a_ih[3][3];    // [q][a]  gs_q / (2 h_a)
+    float2 a_nv[3][3];    // [q][a]  -nu gs_q / h_a^2
+    float2 a_t[3];        // [q]     gs_q / (2 dt)
+    float2 l_g[3];        // [e]     gs_e
+    float2 c_ih[3];       // [a]     gs_c / (2 h_a)
     float* partials;
+    int prefetch;         // planes ahead of the window to prefetch into L2 (0 = off)
 };
 
 struct NsIndex {
-    int c4, m, zm4, zp4;       // own float4 column, y row, float4 columns of z-1 / z+1
-    bool cvalid, valid;
-    bool t_first, t_last;      // this float4 holds t = 0 (in .x) / t = n3-1 (in .w)
+    int col, rowoff;           // own column (floats) and m*C
+    int ymoff, ypoff;          // (m-1)*C, (m+1)*C wrapped
+    int zmcol, zpcol;          // columns of z-1 / z+1 (floats), wrapped over the row
+    int m, c4;
+    bool valid;
+    bool t_first, t_last;      // this float4 holds t = 0 (in lo.x) / t = n3-1 (in hi.y)
 };
+
+__device__ __forceinline__ int wrapi(int i, int n) { return i < 0 ? i + n : (i >= n ? i - n : i); }
+
+// Ask L2 for the line holding `ptr` (no register, no wait): hides most of the DRAM latency of
+// the plane the register window will pull in a few steps later.
+__device__ __forceinline__ void prefetch_l2(const float* ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 
 __device__ __forceinline__ NsIndex ns_index(const NsParams& p, int& a0, int& a1) {
     NsIndex ix;
@@ -50,11 +76,15 @@ __device__ __forceinline__ NsIndex ns_index(const NsParams& p, int& a0, int& a1)
     const int ab = item / p.nmb;
     ix.c4 = cb * blockDim.x + threadIdx.x;
     ix.m = mb * blockDim.y + threadIdx.y;
-    ix.cvalid = ix.c4 < p.C4;
-    ix.valid = ix.cvalid && ix.m < p.n1;
-    const int c4c = ix.cvalid ? ix.c4 : 0;
-    ix.zm4 = c4c - p.nt4; if (ix.zm4 < 0) ix.zm4 += p.C4;
-    ix.zp4 = c4c + p.nt4; if (ix.zp4 >= p.C4) ix.zp4 -= p.C4;
+    ix.valid = ix.c4 < p.C4 && ix.m < p.n1;
+    const int c4c = ix.c4 < p.C4 ? ix.c4 : 0;       // out-of-range threads shadow column 0 / row 0
+    const int mc = ix.m < p.n1 ? ix.m : 0;
+    ix.col = 4 * c4c;
+    ix.rowoff = mc * p.C;
+    ix.ymoff = wrapi(mc - 1, p.n1) * p.C;
+    ix.ypoff = wrapi(mc + 1, p.n1) * p.C;
+    ix.zmcol = 4 * wrapi(c4c - p.nt4, p.C4);
+    ix.zpcol = 4 * wrapi(c4c + p.nt4, p.C4);
     const int tq = c4c % p.nt4;
     ix.t_first = tq == 0;
     ix.t_last = tq == p.nt4 - 1;
@@ -63,92 +93,130 @@ __device__ __forceinline__ NsIndex ns_index(const NsParams& p, int& a0, int& a1)
     return ix;
 }
 
-__device__ __forceinline__ int wrapi(int i, int n) { return i < 0 ? i + n : (i >= n ? i - n : i); }
+// t-1 / t+1 neighbours of a float4's outer lanes: lane-1's last / lane+1's first element.  When
+// a warp boundary can fall inside a z group (TSAFE false) the outer lanes fetch them from memory.
+template <bool TSAFE>
+__device__ __forceinline__ void t_neighbours(const V4& c, const float* __restrict__ row, const NsIndex& ix,
+                                             float& l1, float& r1) {
+    l1 = __shfl_up_sync(FULL_MASK, c.hi.y, 1);
+    r1 = __shfl_down_sync(FULL_MASK, c.lo.x, 1);
+    if (!TSAFE) {
+        const int lane = threadIdx.x & 31;
+        if (lane == 0 && !ix.t_first) l1 = __ldg(row + ix.col - 1);
+        if (lane == 31 && !ix.t_last) r1 = __ldg(row + ix.col + 4);
+    }
+}
 
 // ------------------------------------------------------------------------------------------
 // forward
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) ns_fwd_kernel(const NsParams p) {
+template <bool TSAFE, int MINB>
+__global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
-    const int n0 = p.n0, n1 = p.n1;
-    const size_t C = p.C;
-    const int mrow = ix.m < n1 ? ix.m : 0;
-    const int ym = wrapi(mrow - 1, n1), yp = wrapi(mrow + 1, n1);
+    const int n0 = p.n0;
+    const int PS = p.n1 * p.C;                      // plane stride
+    const float* __restrict__ f0 = p.f[0];
+    const float* __restrict__ f1 = p.f[1];
+    const float* __restrict__ f2 = p.f[2];
+    const float* __restrict__ f3 = p.f[3];
+    const float* const fp[4] = {f0, f1, f2, f3};
 
-    auto ld = [&](const float* base, int a, int mm, int col4) -> float4 {
-        return ld4(base + ((size_t)a * n1 + mm) * C + 4 * col4);
-    };
-    const int c4 = ix.cvalid ? ix.c4 : 0;
-
-    float4 W0[4], W1[4], W2[4];     // planes x-1, x, x+1 of u,v,w,p at the own column
+    V4 A[4], B[4], Cc[4];                           // three x-planes of u,v,w,p at the own column
+    {
+        const int om = wrapi(a0 - 1, n0) * PS + ix.rowoff + ix.col;
+        const int oc = a0 * PS + ix.rowoff + ix.col;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        W0[k] = ld(p.f[k], wrapi(a0 - 1, n0), mrow, c4);
-        W1[k] = ld(p.f[k], a0, mrow, c4);
+        for (int k = 0; k < 4; ++k) { A[k] = ldv4(fp[k] + om); B[k] = ldv4(fp[k] + oc); }
     }
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float2 acc[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
 
-    for (int a = a0; a < a1; ++a) {
-        const int ap = wrapi(a + 1, n0);
-        float4 Ym[4], Yp[4], Zm[4], Zp[4];
+    // one x step: W0 = plane a-1, W1 = plane a, W2 receives plane a+1
+    auto step = [&](int a, const V4 (&W0)[4], const V4 (&W1)[4], V4 (&W2)[4]) {
+        const int pl = a * PS;
+        const int ap = wrapi(a + 1, n0) * PS;
+        if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= a1) {   // one lane per 128-byte line
+            int af = a + 1 + p.prefetch; if (af >= n0) af -= n0;
+            const int po = af * PS + ix.rowoff + ix.col;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) prefetch_l2(fp[k] + po);
+        }
+        V4 Ym[4], Yp[4], Zm[4], Zp[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            W2[k] = ld(p.f[k], ap, mrow, c4);
-            Ym[k] = ld(p.f[k], a, ym, c4);
-            Yp[k] = ld(p.f[k], a, yp, c4);
-            Zm[k] = ld(p.f[k], a, mrow, ix.zm4);
-            Zp[k] = ld(p.f[k], a, mrow, ix.zp4);
+            W2[k] = ldv4(fp[k] + ap + ix.rowoff + ix.col);
+            Ym[k] = ldv4(fp[k] + pl + ix.ymoff + ix.col);
+            Yp[k] = ldv4(fp[k] + pl + ix.ypoff + ix.col);
+            Zm[k] = ldv4(fp[k] + pl + ix.rowoff + ix.zmcol);
+            Zp[k] = ldv4(fp[k] + pl + ix.rowoff + ix.zpcol);
         }
-        LR2 lr[3];
+        float2 dtl[3], dth[3];                      // q(t+1) - q(t-1), lanes (x,y) and (z,w)
 #pragma unroll
-        for (int k = 0; k < 3; ++k)
-            lr[k] = lane_neighbours<1>(p.f[k] + ((size_t)a * n1 + mrow) * C, ix.c4, p.C4, W1[k], false, 1.f);
-
-        float o[4][4];
+        for (int k = 0; k < 3; ++k) {
+            float l1, r1;
+            t_neighbours<TSAFE>(W1[k], fp[k] + pl + ix.rowoff, ix, l1, r1);
+            const V4 c = W1[k];
+            dtl[k] = make_float2(c.lo.y - l1, c.hi.x - c.lo.x);
+            dth[k] = make_float2(c.hi.y - c.lo.y, r1 - c.hi.x);
+        }
+        float2 o[4][2];
 #pragma unroll
-        for (int comp = 0; comp < 4; ++comp) {
-            const float u = f4get(W1[0], comp), v = f4get(W1[1], comp), w = f4get(W1[2], comp);
-            float res[3];
+        for (int h = 0; h < 2; ++h) {               // the two packed halves of the float4
+            auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
+            const float2 us = mul2(H(W1[0]), p.ih[0]);   // advecting velocities, pre-scaled by 1/(2h)
+            const float2 vs = mul2(H(W1[1]), p.ih[1]);
+            const float2 ws = mul2(H(W1[2]), p.ih[2]);
+            float2 dself[3];                        // d_x u, d_y v, d_z w (raw differences)
 #pragma unroll
             for (int k = 0; k < 3; ++k) {
-                const float c = f4get(W1[k], comp);
-                const float xm = f4get(W0[k], comp), xp = f4get(W2[k], comp);
-                const float ymv = f4get(Ym[k], comp), ypv = f4get(Yp[k], comp);
-                const float zmv = f4get(Zm[k], comp), zpv = f4get(Zp[k], comp);
-                const float tm = comp == 0 ? lr[k].l1 : f4get(W1[k], comp - 1);
-                const float tp = comp == 3 ? lr[k].r1 : f4get(W1[k], comp + 1);
-                const float lap = ((xm - c) + (xp - c)) * p.ihxx + ((ymv - c) + (ypv - c)) * p.ihyy
-                                + ((zmv - c) + (zpv - c)) * p.ihzz;
-                res[k] = (tp - tm) * p.iht + u * ((xp - xm) * p.ihx) + v * ((ypv - ymv) * p.ihy)
-                       + w * ((zpv - zmv) * p.ihz) - p.nu * lap;
+                const float2 c = H(W1[k]);
+                const float2 xm = sub2(H(W0[k]), c), xp = sub2(H(W2[k]), c);
+                const float2 ym = sub2(H(Ym[k]), c), yp = sub2(H(Yp[k]), c);
+                const float2 zm = sub2(H(Zm[k]), c), zp = sub2(H(Zp[k]), c);
+                const float2 dx = sub2(xp, xm), dy = sub2(yp, ym), dz = sub2(zp, zm);
+                float2 r = mul2(add2(xm, xp), p.nv[0]);
+                r = fma2(add2(ym, yp), p.nv[1], r);
+                r = fma2(add2(zm, zp), p.nv[2], r);
+                r = fma2(us, dx, r);
+                r = fma2(vs, dy, r);
+                r = fma2(ws, dz, r);
+                r = fma2(h == 0 ? dtl[k] : dth[k], p.iht, r);
+                dself[k] = k == 0 ? dx : (k == 1 ? dy : dz);
+                o[k][h] = r;
             }
-            res[0] += (f4get(W2[3], comp) - f4get(W0[3], comp)) * p.ihx;     // d_x p
-            res[1] += (f4get(Yp[3], comp) - f4get(Ym[3], comp)) * p.ihy;     // d_y p
-            res[2] += (f4get(Zp[3], comp) - f4get(Zm[3], comp)) * p.ihz;     // d_z p
-            const float div = (f4get(W2[0], comp) - f4get(W0[0], comp)) * p.ihx
-                            + (f4get(Yp[1], comp) - f4get(Ym[1], comp)) * p.ihy
-                            + (f4get(Zp[2], comp) - f4get(Zm[2], comp)) * p.ihz;
-            o[0][comp] = res[0]; o[1][comp] = res[1]; o[2][comp] = res[2]; o[3][comp] = div;
+            o[0][h] = fma2(sub2(H(W2[3]), H(W0[3])), p.ih[0], o[0][h]);     // d_x p
+            o[1][h] = fma2(sub2(H(Yp[3]), H(Ym[3])), p.ih[1], o[1][h]);     // d_y p
+            o[2][h] = fma2(sub2(H(Zp[3]), H(Zm[3])), p.ih[2], o[2][h]);     // d_z p
+            o[3][h] = fma2(dself[2], p.ih[2], fma2(dself[1], p.ih[1], mul2(dself[0], p.ih[0])));
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {          // t = 0 and t = n3-1 carry no row
-            if (ix.t_first) o[e][0] = 0.f;
-            if (ix.t_last) o[e][3] = 0.f;
+        for (int e = 0; e < 4; ++e) {               // t = 0 and t = n3-1 carry no row
+            if (ix.t_first) o[e][0].x = 0.f;
+            if (ix.t_last) o[e][1].y = 0.f;
         }
         if (ix.valid) {
-            const size_t off = ((size_t)a * n1 + ix.m) * C + 4 * ix.c4;
+            const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float4 ov = make_float4(o[e][0], o[e][1], o[e][2], o[e][3]);
-                st4(p.out[e] + off, ov);
-                acc[e] += sq4(ov);
+                stv4(p.out[e] + off, o[e][0], o[e][1]);
+                acc[e] = fma2(o[e][0], o[e][0], fma2(o[e][1], o[e][1], acc[e]));
             }
         }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { W0[k] = W1[k]; W1[k] = W2[k]; }
+    };
+
+    for (int a = a0; a < a1; a += 3) {
+        step(a, A, B, Cc);
+        if (a + 1 < a1) step(a + 1, B, Cc, A);
+        if (a + 2 < a1) step(a + 2, Cc, A, B);
     }
-    if (p.partials != nullptr) block_reduce_store<4>(acc, p.partials, p.nitems, blockIdx.x);
+    if (p.partials != nullptr) {
+        float s[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[e] = acc[e].x + acc[e].y;
+        block_reduce_store<4>(s, p.partials, p.nitems, blockIdx.x);
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -160,110 +228,115 @@ __global__ void __launch_bounds__(256) ns_fwd_kernel(const NsParams p) {
 //          + [ G_q(P-t) - G_q(P+t) ] / (2 dt)                                  transposed d_t
 //          + [ G_c(P-a_q) - G_c(P+a_q) ] / (2 h_{a_q})                         continuity row
 //   g_p(P) = sum_q [ G_q(P-a_q) - G_q(P+a_q) ] / (2 h_{a_q})
+// G_e = gscale_e * gres_e; the scales are folded into the constants.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) ns_bwd_kernel(const NsParams p) {
+template <bool TSAFE, int MINB>
+__global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
-    const int n0 = p.n0, n1 = p.n1;
-    const size_t C = p.C;
-    const int mrow = ix.m < n1 ? ix.m : 0;
-    const int ym = wrapi(mrow - 1, n1), yp = wrapi(mrow + 1, n1);
-    const int c4 = ix.cvalid ? ix.c4 : 0;
+    const int n0 = p.n0;
+    const int PS = p.n1 * p.C;
+    // arrays 0..2: u,v,w ; 3..6: upstream of mom_x, mom_y, mom_z, continuity
+    const float* const ap[7] = {p.f[0], p.f[1], p.f[2], p.g[0], p.g[1], p.g[2], p.g[3]};
 
-    auto ldf = [&](int k, int a, int mm, int col4) -> float4 {
-        return ld4(p.f[k] + ((size_t)a * n1 + mm) * C + 4 * col4);
-    };
-    // upstream array k, scaled, zeroed at the first / last t.  z-neighbours sit at the same t.
-    auto ldg = [&](int k, int a, int mm, int col4) -> float4 {
-        float4 v = f4scale(ld4(p.g[k] + ((size_t)a * n1 + mm) * C + 4 * col4), p.gs[k]);
-        if (ix.t_first) v.x = 0.f;
-        if (ix.t_last) v.w = 0.f;
-        return v;
-    };
-
-    float4 F0[3], F1[3], F2[3];     // u,v,w at x-1, x, x+1
-    float4 G0[4], G1[4], G2[4];     // G_u,G_v,G_w,G_c at x-1, x, x+1
+    V4 A[7], B[7], Cc[7];
     {
-        const int am = wrapi(a0 - 1, n0);
+        const int om = wrapi(a0 - 1, n0) * PS + ix.rowoff + ix.col;
+        const int oc = a0 * PS + ix.rowoff + ix.col;
 #pragma unroll
-        for (int k = 0; k < 3; ++k) { F0[k] = ldf(k, am, mrow, c4); F1[k] = ldf(k, a0, mrow, c4); }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { G0[k] = ldg(k, am, mrow, c4); G1[k] = ldg(k, a0, mrow, c4); }
+        for (int k = 0; k < 7; ++k) { A[k] = ldv4(ap[k] + om); B[k] = ldv4(ap[k] + oc); }
     }
 
-    for (int a = a0; a < a1; ++a) {
-        const int ap = wrapi(a + 1, n0);
-        float4 FYm[3], FYp[3], FZm[3], FZp[3], GYm[4], GYp[4], GZm[4], GZp[4];
+    auto step = [&](int a, const V4 (&W0)[7], const V4 (&W1)[7], V4 (&W2)[7]) {
+        const int pl = a * PS;
+        const int apl = wrapi(a + 1, n0) * PS;
+        if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= a1) {
+            int af = a + 1 + p.prefetch; if (af >= n0) af -= n0;
+            const int po = af * PS + ix.rowoff + ix.col;
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            F2[k] = ldf(k, ap, mrow, c4);
-            FYm[k] = ldf(k, a, ym, c4); FYp[k] = ldf(k, a, yp, c4);
-            FZm[k] = ldf(k, a, mrow, ix.zm4); FZp[k] = ldf(k, a, mrow, ix.zp4);
+            for (int k = 0; k < 7; ++k) prefetch_l2(ap[k] + po);
         }
+        V4 Ym[7], Yp[7], Zm[7], Zp[7];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            G2[k] = ldg(k, ap, mrow, c4);
-            GYm[k] = ldg(k, a, ym, c4); GYp[k] = ldg(k, a, yp, c4);
-            GZm[k] = ldg(k, a, mrow, ix.zm4); GZp[k] = ldg(k, a, mrow, ix.zp4);
+        for (int k = 0; k < 7; ++k) {
+            W2[k] = ldv4(ap[k] + apl + ix.rowoff + ix.col);
+            Ym[k] = ldv4(ap[k] + pl + ix.ymoff + ix.col);
+            Yp[k] = ldv4(ap[k] + pl + ix.ypoff + ix.col);
+            Zm[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zmcol);
+            Zp[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zpcol);
         }
-        LR2 lr[3];
+        float2 dtl[3], dth[3];                      // G_q(t-1) - G_q(t+1) with the end planes counted as 0
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            lr[k] = lane_neighbours<1>(p.g[k] + ((size_t)a * n1 + mrow) * C, ix.c4, p.C4, G1[k], false, p.gs[k]);
-            // the neighbour across a z-group boundary is the other group's first / last t: no row
-            if (ix.t_first) lr[k].l1 = 0.f;
-            if (ix.t_last) lr[k].r1 = 0.f;
+        for (int q = 0; q < 3; ++q) {
+            float l1, r1;
+            t_neighbours<TSAFE>(W1[3 + q], ap[3 + q] + pl + ix.rowoff, ix, l1, r1);
+            const V4 c = W1[3 + q];
+            const float tm_y = ix.t_first ? 0.f : c.lo.x;       // t-1 of lane y is the end plane t = 0
+            const float tp_z = ix.t_last ? 0.f : c.hi.y;        // t+1 of lane z is the end plane t = n3-1
+            dtl[q] = make_float2(l1 - c.lo.y, tm_y - c.hi.x);
+            dth[q] = make_float2(c.lo.y - tp_z, c.hi.x - r1);
         }
-
-        float o[4][4];
+        float2 o[4][2];
 #pragma unroll
-        for (int comp = 0; comp < 4; ++comp) {
-            // centred first differences d_a e of the three velocity components
-            float dx[3], dy[3], dz[3];
+        for (int h = 0; h < 2; ++h) {
+            auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
+            // neighbours of array k along axis a: minus / plus
+            auto NM = [&](int k, int a_) -> float2 { return a_ == 0 ? H(W0[k]) : (a_ == 1 ? H(Ym[k]) : H(Zm[k])); };
+            auto NP = [&](int k, int a_) -> float2 { return a_ == 0 ? H(W2[k]) : (a_ == 1 ? H(Yp[k]) : H(Zp[k])); };
+            float2 gs[3];                            // scaled centre sensitivities
 #pragma unroll
-            for (int e = 0; e < 3; ++e) {
-                dx[e] = (f4get(F2[e], comp) - f4get(F0[e], comp)) * p.ihx;
-                dy[e] = (f4get(FYp[e], comp) - f4get(FYm[e], comp)) * p.ihy;
-                dz[e] = (f4get(FZp[e], comp) - f4get(FZm[e], comp)) * p.ihz;
+            for (int e = 0; e < 3; ++e) gs[e] = mul2(H(W1[3 + e]), p.l_g[e]);
+            float2 cm[3], ncp[3];                    // advecting velocity at P-a, minus the one at P+a
+#pragma unroll
+            for (int a_ = 0; a_ < 3; ++a_) {
+                cm[a_] = NM(a_, a_);
+                const float2 cp = NP(a_, a_);
+                ncp[a_] = make_float2(-cp.x, -cp.y);
             }
-            const float gu = f4get(G1[0], comp), gv = f4get(G1[1], comp), gw = f4get(G1[2], comp);
-            // advecting velocities at the six neighbours: u at x-+1, v at y-+1, w at z-+1
-            const float uxm = f4get(F0[0], comp), uxp = f4get(F2[0], comp);
-            const float vym = f4get(FYm[1], comp), vyp = f4get(FYp[1], comp);
-            const float wzm = f4get(FZm[2], comp), wzp = f4get(FZp[2], comp);
-            float gq[3];
+            float2 gp = make_float2(0.f, 0.f);
 #pragma unroll
             for (int q = 0; q < 3; ++q) {
-                const float c = f4get(G1[q], comp);
-                const float xm = f4get(G0[q], comp), xp = f4get(G2[q], comp);
-                const float ymv = f4get(GYm[q], comp), ypv = f4get(GYp[q], comp);
-                const float zmv = f4get(GZm[q], comp), zpv = f4get(GZp[q], comp);
-                const float tm = comp == 0 ? lr[q].l1 : f4get(G1[q], comp - 1);
-                const float tp = comp == 3 ? lr[q].r1 : f4get(G1[q], comp + 1);
-                const float adv = (xm * uxm - xp * uxp) * p.ihx + (ymv * vym - ypv * vyp) * p.ihy
-                                + (zmv * wzm - zpv * wzp) * p.ihz;
-                const float lap = ((xm - c) + (xp - c)) * p.ihxx + ((ymv - c) + (ypv - c)) * p.ihyy
-                                + ((zmv - c) + (zpv - c)) * p.ihzz;
-                gq[q] = adv - p.nu * lap + (tm - tp) * p.iht;
+                const float2 c = H(W1[3 + q]);
+                float2 r = mul2(h == 0 ? dtl[q] : dth[q], p.a_t[q]);
+#pragma unroll
+                for (int a_ = 0; a_ < 3; ++a_) {
+                    const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
+                    const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
+                    r = fma2(adv, p.a_ih[q][a_], r);
+                    const float2 dm = sub2(gm, c), dp = sub2(gpl, c);
+                    r = fma2(add2(dm, dp), p.a_nv[q][a_], r);
+                    if (a_ == q) gp = fma2(sub2(dm, dp), p.a_ih[q][q], gp);
+                }
+                // local terms and continuity row along this component's own axis
+                float2 loc = mul2(gs[0], sub2(NP(0, q), NM(0, q)));
+                loc = fma2(gs[1], sub2(NP(1, q), NM(1, q)), loc);
+                loc = fma2(gs[2], sub2(NP(2, q), NM(2, q)), loc);
+                r = fma2(loc, p.ih[q], r);
+                r = fma2(sub2(NM(6, q), NP(6, q)), p.c_ih[q], r);
+                o[q][h] = r;
             }
-            gq[0] += gu * dx[0] + gv * dx[1] + gw * dx[2] + (f4get(G0[3], comp) - f4get(G2[3], comp)) * p.ihx;
-            gq[1] += gu * dy[0] + gv * dy[1] + gw * dy[2] + (f4get(GYm[3], comp) - f4get(GYp[3], comp)) * p.ihy;
-            gq[2] += gu * dz[0] + gv * dz[1] + gw * dz[2] + (f4get(GZm[3], comp) - f4get(GZp[3], comp)) * p.ihz;
-            const float gp = (f4get(G0[0], comp) - f4get(G2[0], comp)) * p.ihx
-                           + (f4get(GYm[1], comp) - f4get(GYp[1], comp)) * p.ihy
-                           + (f4get(GZm[2], comp) - f4get(GZp[2], comp)) * p.ihz;
-            o[0][comp] = gq[0]; o[1][comp] = gq[1]; o[2][comp] = gq[2]; o[3][comp] = gp;
+            o[3][h] = gp;
         }
+        // end planes of t: only the transposed d_t term exists there, and no pressure gradient
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const V4 c = W1[3 + q];
+            if (ix.t_first) o[q][0].x = -c.lo.y * p.a_t[q].x;
+            if (ix.t_last) o[q][1].y = c.hi.x * p.a_t[q].x;
+        }
+        if (ix.t_first) o[3][0].x = 0.f;
+        if (ix.t_last) o[3][1].y = 0.f;
         if (ix.valid) {
-            const size_t off = ((size_t)a * n1 + ix.m) * C + 4 * ix.c4;
+            const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                st4(p.out[e] + off, make_float4(o[e][0], o[e][1], o[e][2], o[e][3]));
+            for (int e = 0; e < 4; ++e) stv4(p.out[e] + off, o[e][0], o[e][1]);
         }
-#pragma unroll
-        for (int k = 0; k < 3; ++k) { F0[k] = F1[k]; F1[k] = F2[k]; }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { G0[k] = G1[k]; G1[k] = G2[k]; }
+    };
+
+    for (int a = a0; a < a1; a += 3) {
+        step(a, A, B, Cc);
+        if (a + 1 < a1) step(a + 1, B, Cc, A);
+        if (a + 2 < a1) step(a + 2, Cc, A, B);
     }
 }
 
@@ -274,25 +347,26 @@ static int env_int(const char* name, int dflt) {
     return v > 0 ? v : dflt;
 }
 
+static float2 sp(double v) { return make_float2((float)v, (float)v); }
+
 static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n3 = q.n[3];
     p.C = q.n[2] * q.n[3]; p.C4 = p.C / 4; p.nt4 = q.n[3] / 4;
-    int tx = p.C4 >= 64 ? 64 : 32;
-    tx = env_int("FPDE_NS_TX", tx);
-    tx = std::max(32, std::min(256, (tx / 32) * 32));
+    int tx = env_int("FPDE_NS_TX", 32);
+    tx = std::max(32, std::min(128, (tx / 32) * 32));
     int ty = env_int("FPDE_NS_TY", 4);
-    ty = std::max(1, std::min(256 / tx, ty));
+    ty = std::max(1, std::min(128 / tx, ty));
     block = dim3(tx, ty, 1);
     p.planes_per_item = env_int("FPDE_NS_PLANES", 16);
     p.ncb = (p.C4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
-    p.ihx = (float)(0.5 / q.h[0]); p.ihy = (float)(0.5 / q.h[1]); p.ihz = (float)(0.5 / q.h[2]);
-    p.iht = (float)(0.5 / q.h[3]);
-    p.ihxx = (float)(1.0 / (q.h[0] * q.h[0])); p.ihyy = (float)(1.0 / (q.h[1] * q.h[1]));
-    p.ihzz = (float)(1.0 / (q.h[2] * q.h[2]));
-    p.nu = (float)q.coef[0];
+    const char* pf = std::getenv("FPDE_NS_PREFETCH");
+    p.prefetch = pf && *pf ? std::atoi(pf) : 3;
+    if (p.prefetch < 0 || p.prefetch >= p.n0) p.prefetch = 0;
 }
+
+static bool ns_tsafe(const NsParams& p) { return 32 % p.nt4 == 0; }
 
 int ns_items(const int* n) {
     Problem q{};
@@ -306,19 +380,42 @@ cudaError_t launch_ns_fwd(const Problem& q) {
     NsParams p{}; dim3 block;
     ns_geometry(q, p, block);
     for (int k = 0; k < 4; ++k) { p.f[k] = q.in[k]; p.out[k] = q.out[k]; }
+    const double nu = q.coef[0];
+    for (int a = 0; a < 3; ++a) {
+        p.ih[a] = sp(0.5 / q.h[a]);
+        p.nv[a] = sp(-nu / (q.h[a] * q.h[a]));
+    }
+    p.iht = sp(0.5 / q.h[3]);
     p.partials = q.partials;
-    ns_fwd_kernel<<<p.nitems, block, 0, q.stream>>>(p);
+    const int minb = env_int("FPDE_NS_MINB_F", 3);
+    if (!ns_tsafe(p)) ns_fwd_kernel<false, 3><<<p.nitems, block, 0, q.stream>>>(p);
+    else if (minb == 3) ns_fwd_kernel<true, 3><<<p.nitems, block, 0, q.stream>>>(p);
+    else ns_fwd_kernel<true, 4><<<p.nitems, block, 0, q.stream>>>(p);
     return cudaGetLastError();
 }
 
 cudaError_t launch_ns_bwd(const Problem& q) {
     NsParams p{}; dim3 block;
     ns_geometry(q, p, block);
-    for (int k = 0; k < 4; ++k) {
-        p.f[k] = q.in[k]; p.g[k] = q.aux[k]; p.out[k] = q.out[k]; p.gs[k] = (float)q.gscale[k];
+    for (int k = 0; k < 4; ++k) { p.f[k] = q.in[k]; p.g[k] = q.aux[k]; p.out[k] = q.out[k]; }
+    const double nu = q.coef[0];
+    for (int a = 0; a < 3; ++a) {
+        p.ih[a] = sp(0.5 / q.h[a]);
+        p.c_ih[a] = sp(q.gscale[3] * 0.5 / q.h[a]);
+    }
+    for (int k = 0; k < 3; ++k) {
+        p.a_t[k] = sp(q.gscale[k] * 0.5 / q.h[3]);
+        p.l_g[k] = sp(q.gscale[k]);
+        for (int a = 0; a < 3; ++a) {
+            p.a_ih[k][a] = sp(q.gscale[k] * 0.5 / q.h[a]);
+            p.a_nv[k][a] = sp(-nu * q.gscale[k] / (q.h[a] * q.h[a]));
+        }
     }
     p.partials = nullptr;
-    ns_bwd_kernel<<<p.nitems, block, 0, q.stream>>>(p);
+    const int minb = env_int("FPDE_NS_MINB_B", 2);
+    if (!ns_tsafe(p)) ns_bwd_kernel<false, 2><<<p.nitems, block, 0, q.stream>>>(p);
+    else if (minb == 3) ns_bwd_kernel<true, 3><<<p.nitems, block, 0, q.stream>>>(p);
+    else ns_bwd_kernel<true, 2><<<p.nitems, block, 0, q.stream>>>(p);
     return cudaGetLastError();
 }
 
