@@ -225,18 +225,28 @@ class DeviceProblem:
         self.B.fpde_bwd(w.op, self.fields, self.res, self.gscale, self.grads, w.shape, w.spacing, w.coeffs, w.bc)
 
 
-def timed_steps(torch, prob, steps, warmup, barrier, flush=None):
-    """K back-to-back steps between two events; inner events give per-call durations."""
+def timed_steps(torch, prob, steps, warmup, barrier, flush=None, inner_events=False):
+    """K back-to-back steps between two events.  With inner_events, every forward and adjoint call
+    is bracketed by its own events as well (per-call durations; the extra records sit between
+    launches, so this variant is used for the per-kernel figures, not for the headline)."""
     for _ in range(warmup):
         prob.fwd(); prob.bwd()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    first, last = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)] if inner_events else None
     barrier(); torch.cuda.synchronize()
+    first.record()
     for k in range(steps):
         if flush is not None:
             flush.fill_(k)
-        ev[k][0].record(); prob.fwd(); ev[k][1].record(); prob.bwd(); ev[k][2].record()
+        if inner_events:
+            ev[k][0].record(); prob.fwd(); ev[k][1].record(); prob.bwd(); ev[k][2].record()
+        else:
+            prob.fwd(); prob.bwd()
+    last.record()
     torch.cuda.synchronize(); barrier()
-    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    total_ms = first.elapsed_time(last)
+    if not inner_events:
+        return total_ms, None, None
     fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
     return total_ms, fwd_ms, bwd_ms
@@ -278,7 +288,7 @@ def config_line(torch, B, name, steps, warmup, peak):
     w = W.make(name, seed=42)
     prob = DeviceProblem(torch, B, w)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    _, f_ms, b_ms = timed_steps(torch, prob, steps, warmup, lambda: None, flush=flush)
+    _, f_ms, b_ms = timed_steps(torch, prob, steps, warmup, lambda: None, flush=flush, inner_events=True)
     fm, bm = statistics.median(f_ms), statistics.median(b_ms)
     fb, bb = ALGO_BYTES[w.op]
     N = w.npoints
@@ -343,7 +353,9 @@ def main():
 
     sampler = ClockSampler(torch, local_rank)
     sampler.start()
-    total_ms, fwd_ms, bwd_ms = timed_steps(torch, prob, args.steps, args.warmup, barrier)
+    total_ms, _, _ = timed_steps(torch, prob, args.steps, args.warmup, barrier)
+    # same K steps again with an event pair around every call: per-kernel durations for the roofline
+    _, fwd_ms, bwd_ms = timed_steps(torch, prob, args.steps, 0, barrier, inner_events=True)
     sampler.stop()
     total_ms = max_over_ranks(total_ms)
     value = world * N * args.steps / (total_ms * 1e-3)

@@ -6,6 +6,7 @@
 #include "fpde_internal.h"
 
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 
 namespace fpde {
@@ -62,6 +63,11 @@ static size_t workspace_need(int op, const int* n) {
     return (size_t)items * REGISTRY[op].ne * sizeof(float);
 }
 
+bool pdl_enabled() {
+    const char* s = std::getenv("FPDE_PDL");
+    return !(s && s[0] == '0');
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Common validation of the arguments fwd and bwd share; fills the Problem.
@@ -98,6 +104,7 @@ __global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restr
                                                             int nres, double inv_rows,
                                                             double* __restrict__ loss_out) {
     __shared__ double sm[256];
+    pdl_wait_then_trigger();
     double total = 0.0;
     for (int e = 0; e < nres; ++e) {
         double s = 0.0;
@@ -118,8 +125,8 @@ __global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restr
 
 cudaError_t launch_loss_finalize(const float* partials, int nitems, int nres, int64_t rows,
                                  double* loss_out, cudaStream_t stream) {
-    loss_finalize_kernel<<<1, 256, 0, stream>>>(partials, nitems, nres, 1.0 / (double)rows, loss_out);
-    return cudaGetLastError();
+    return launch_kernel(loss_finalize_kernel, dim3(1), dim3(256), stream, partials, nitems, nres,
+                         1.0 / (double)rows, loss_out);
 }
 
 }  // namespace fpde

@@ -8,6 +8,15 @@
 namespace fpde {
 
 constexpr unsigned FULL_MASK = 0xffffffffu;
+
+// Programmatic dependent launch: every kernel first waits until the kernel before it in the
+// stream has completed and its writes are visible (a no-op when launched without the
+// attribute), then lets the kernel after it start launching, so that launch latency and the
+// tail of one kernel overlap with the head of the next.
+__device__ __forceinline__ void pdl_wait_then_trigger() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 constexpr int MAX_RES = 4;        // most residual fields of any operator
 
 __device__ __forceinline__ float4 ld4(const float* p) {

@@ -27,6 +27,20 @@ struct Problem {
     cudaStream_t stream;
 };
 
+// Launch with programmatic stream serialisation allowed (kernels call pdl_wait_then_trigger()).
+// FPDE_PDL=0 in the environment falls back to plain stream order (for A/B measurements).
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+
 // Number of loss partial sums (= work items) per residual field the forward kernel of this
 // operator produces for this grid.  Fixed by the grid alone, so the reduction order is too.
 int fwd_items(int op, const int* n);

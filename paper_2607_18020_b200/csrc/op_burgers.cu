@@ -69,6 +69,7 @@ __device__ __forceinline__ float d2T_at(WF W, int j, int n, float ihh) {
 }
 
 __global__ void __launch_bounds__(256) burgers_fwd_kernel(const BurgersParams p) {
+    pdl_wait_then_trigger();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     const int N = p.nx * p.nt;
     float acc[1] = {0.f};
@@ -85,6 +86,7 @@ __global__ void __launch_bounds__(256) burgers_fwd_kernel(const BurgersParams p)
 }
 
 __global__ void __launch_bounds__(256) burgers_bwd_kernel(const BurgersParams p) {
+    pdl_wait_then_trigger();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     const int N = p.nx * p.nt;
     if (idx >= N) return;
@@ -115,16 +117,14 @@ cudaError_t launch_burgers_fwd(const Problem& q) {
     BurgersParams p{};
     burgers_params(q, p);
     p.u = q.in[0]; p.out = q.out[0]; p.partials = q.partials;
-    burgers_fwd_kernel<<<p.nitems, 256, 0, q.stream>>>(p);
-    return cudaGetLastError();
+    return launch_kernel(burgers_fwd_kernel, dim3(p.nitems), dim3(256), q.stream, p);
 }
 
 cudaError_t launch_burgers_bwd(const Problem& q) {
     BurgersParams p{};
     burgers_params(q, p);
     p.u = q.in[0]; p.g = q.aux[0]; p.out = q.out[0]; p.gs = (float)q.gscale[0];
-    burgers_bwd_kernel<<<p.nitems, 256, 0, q.stream>>>(p);
-    return cudaGetLastError();
+    return launch_kernel(burgers_bwd_kernel, dim3(p.nitems), dim3(256), q.stream, p);
 }
 
 }  // namespace fpde

@@ -8,9 +8,12 @@
 // 2 and 3.  Forward and adjoint are therefore two instances of one 2.5-D engine:
 //
 //   a thread owns one float4 of a (y,z) tile and marches along x, the slowest axis, holding the
-//   five x-planes of its own column in registers; the y+-1, y+-2 neighbours of the current plane
-//   are read through L1 (other threads of the same block loaded those lines two steps earlier);
-//   z neighbours come from the adjacent lanes' registers.
+//   five x-planes of its own column in registers (rotated by unrolling); the y+-1, y+-2
+//   neighbours of the current plane are read through L1 (other threads of the same block loaded
+//   those lines two steps earlier); z neighbours come from the adjacent lanes' registers.  The
+//   plane the window will need three steps later is prefetched into L2.  Arithmetic is packed
+//   fp32x2; the star is evaluated as  sum_a w_a (16 (q[-1]+q[+1]) - (q[-2]+q[+2])) + K q  with
+//   K = k^2 - 30 sum_a w_a.
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
 
@@ -20,96 +23,123 @@
 namespace fpde {
 
 struct Star3dParams {
-    const float* hin;     // read with halo 2 (u forward, upstream G in the adjoint)
+    const float* hin;     // read with halo 2 (u forward, upstream array in the adjoint)
     const float* cin;     // read at the centre (f forward, unused in the adjoint)
     float* out;
-    float hscale;
     int n0, n1, n2, nc4;
     int planes_per_item, ncb, nmb, nitems;
-    float w0, w1, w2;     // 1/(12 h_a^2)
-    float k2;
+    float2 w16[3];        // 16 s / (12 h_a^2), s = upstream scale (1 forward)
+    float2 nw[3];         // -s / (12 h_a^2)
+    float2 kc;            // s (k^2 - 30 sum_a 1/(12 h_a^2))
     float* partials;
+    int prefetch;
 };
 
+__device__ __forceinline__ void prefetch_l2_line(const float* ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
+
 template <bool FWD>
-__global__ void __launch_bounds__(256) star3d_kernel(const Star3dParams p) {
-    const int n0 = p.n0, n1 = p.n1, n2 = p.n2;
+__global__ void __launch_bounds__(512) star3d_kernel(const Star3dParams p) {
+    pdl_wait_then_trigger();
+    const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
     int item = blockIdx.x;
     const int cb = item % p.ncb; item /= p.ncb;
     const int mb = item % p.nmb;
     const int ab = item / p.nmb;
     const int c4 = cb * blockDim.x + threadIdx.x;
     const int m = mb * blockDim.y + threadIdx.y;
-    const bool cvalid = c4 < p.nc4;
-    const bool valid = cvalid && m < n1;
-    const bool first_col = c4 == 0, last_col = c4 == p.nc4 - 1;
+    const int lane = threadIdx.x & 31;
+    const bool valid = c4 < nc4 && m < n1;
+    const int col = c4 < nc4 ? 4 * c4 : 0;
+    const int mc = m < n1 ? m : 0;
+    const bool first_col = c4 == 0, last_col = c4 == nc4 - 1;
     const int a0 = ab * p.planes_per_item;
     const int a1 = min(a0 + p.planes_per_item, n0);
+    const int PS = n1 * n2;
     constexpr bool MASK_IN = !FWD;
+    const float* __restrict__ hin = p.hin;
 
-    // does a (plane,row) pair of the halo input read as zero?
-    auto dead = [&](int a, int mm) -> bool {
-        if (a < 0 || a >= n0 || mm < 0 || mm >= n1) return true;
-        if (MASK_IN && (a < 2 || a > n0 - 3 || mm < 2 || mm > n1 - 3)) return true;
-        return false;
-    };
-    auto load_h = [&](int a, int mm) -> float4 {
-        if (dead(a, mm) || !cvalid) return f4zero();
-        float4 v = ld4(p.hin + ((size_t)a * n1 + mm) * n2 + 4 * c4);
+    // Rows / planes outside the grid are clamped (forward: they only feed masked outputs).  In
+    // the adjoint a row or plane outside the rows of the operator reads as zero: the load is
+    // still issued at the clamped address and the value is then discarded by a select, which
+    // keeps the loads of a step independent of each other (no branches between them).
+    auto yclamp = [&](int d) -> int { return max(0, min(n1 - 1, mc + d)); };
+    auto ydead = [&](int d) -> bool { const int r = mc + d; return MASK_IN && (r < 2 || r > n1 - 3); };
+    const int ym1 = yclamp(-1), yp1 = yclamp(1), ym2 = yclamp(-2), yp2 = yclamp(2), y0 = mc;
+    const bool dm1 = ydead(-1), dp1 = ydead(1), dm2 = ydead(-2), dp2 = ydead(2), d0 = ydead(0);
+    auto load_h = [&](int a, int r, bool rdead) -> V4 {
+        const int pa = max(0, min(n0 - 1, a));
+        V4 v = ldv4(hin + pa * PS + r * n2 + col);
         if (MASK_IN) {
-            v = f4scale(v, p.hscale);
-            if (first_col) { v.x = 0.f; v.y = 0.f; }
-            if (last_col) { v.z = 0.f; v.w = 0.f; }
+            const bool dead = rdead || a < 2 || a > n0 - 3;
+            if (dead || first_col) v.lo = make_float2(0.f, 0.f);
+            if (dead || last_col) v.hi = make_float2(0.f, 0.f);
         }
         return v;
     };
+    const bool lfetch = lane == 0 && c4 > 0 && c4 < nc4;
+    const bool rfetch = lane == 31 && c4 < nc4 - 1;
 
-    float4 q0 = load_h(a0 - 2, m), q1 = load_h(a0 - 1, m), q2 = load_h(a0, m), q3 = load_h(a0 + 1, m);
-    float acc[1] = {0.f};
+    V4 Q0 = load_h(a0 - 2, y0, d0), Q1 = load_h(a0 - 1, y0, d0), Q2 = load_h(a0, y0, d0), Q3 = load_h(a0 + 1, y0, d0), Q4;
+    float2 acc = make_float2(0.f, 0.f);
 
-    for (int a = a0; a < a1; ++a) {
-        const float4 q4 = load_h(a + 2, m);
-        const float4 ym1 = load_h(a, m - 1), yp1 = load_h(a, m + 1);
-        const float4 ym2 = load_h(a, m - 2), yp2 = load_h(a, m + 2);
-        float4 src = f4zero();
-        if (FWD && valid) src = ld4(p.cin + ((size_t)a * n1 + m) * n2 + 4 * c4);
-        LR2 lr;
-        if (!dead(a, m)) {     // uniform over a warp (a warp lies inside one row)
-            lr = lane_neighbours<2>(p.hin + ((size_t)a * n1 + m) * n2, c4, p.nc4, q2, false,
-                                    MASK_IN ? p.hscale : 1.f);
-        } else {
-            lr.l1 = lr.l2 = lr.r1 = lr.r2 = 0.f;
+    // one x step: q0..q3 = planes a-2..a+1, q4 receives plane a+2
+    auto step = [&](int a, const V4& q0, const V4& q1, const V4& q2, const V4& q3, V4& q4) {
+        if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 2 + p.prefetch <= a1 + 1 && a + 2 + p.prefetch < n0) {
+            prefetch_l2_line(hin + (a + 2 + p.prefetch) * PS + mc * n2 + col);
+            if (FWD) prefetch_l2_line(p.cin + min(a + p.prefetch, n0 - 1) * PS + mc * n2 + col);
         }
-        float o[4];
-#pragma unroll
-        for (int comp = 0; comp < 4; ++comp) {
-            const float c = f4get(q2, comp);
-            const float l1 = comp == 0 ? lr.l1 : f4get(q2, comp - 1);
-            const float l2 = comp == 0 ? lr.l2 : (comp == 1 ? lr.l1 : f4get(q2, comp - 2));
-            const float r1 = comp == 3 ? lr.r1 : f4get(q2, comp + 1);
-            const float r2 = comp == 3 ? lr.r2 : (comp == 2 ? lr.r1 : f4get(q2, comp + 2));
-            const float sx = 16.f * ((f4get(q1, comp) - c) + (f4get(q3, comp) - c))
-                           - ((f4get(q0, comp) - c) + (f4get(q4, comp) - c));
-            const float sy = 16.f * ((f4get(ym1, comp) - c) + (f4get(yp1, comp) - c))
-                           - ((f4get(ym2, comp) - c) + (f4get(yp2, comp) - c));
-            const float sz = 16.f * ((l1 - c) + (r1 - c)) - ((l2 - c) + (r2 - c));
-            float v = sx * p.w0 + sy * p.w1 + sz * p.w2 + p.k2 * c;
-            if (FWD) v -= f4get(src, comp);
-            o[comp] = v;
+        q4 = load_h(a + 2, y0, d0);
+        const V4 a1v = load_h(a, ym1, dm1), b1v = load_h(a, yp1, dp1), a2v = load_h(a, ym2, dm2), b2v = load_h(a, yp2, dp2);
+        V4 src = v4zero();
+        if (FWD) src = ldv4(p.cin + a * PS + mc * n2 + col);
+        // z neighbours from the adjacent lanes; the outer lanes of a warp fetch theirs
+        float l1 = __shfl_up_sync(FULL_MASK, q2.hi.y, 1), l2 = __shfl_up_sync(FULL_MASK, q2.hi.x, 1);
+        float r1 = __shfl_down_sync(FULL_MASK, q2.lo.x, 1), r2 = __shfl_down_sync(FULL_MASK, q2.lo.y, 1);
+        {
+            const float* rp = hin + a * PS + y0 * n2 + col;      // a is a valid plane here
+            if (lfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp - 2)); l2 = t.x; l1 = t.y; }
+            if (rfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp + 4)); r1 = t.x; r2 = t.y; }
+            const bool dead = MASK_IN && (d0 || a < 2 || a > n0 - 3);
+            if (dead || first_col) { l1 = 0.f; l2 = 0.f; }
+            if (dead || last_col) { r1 = 0.f; r2 = 0.f; }
         }
-        if (FWD) {   // nodes of the two outer layers carry no row
-            if (a < 2 || a > n0 - 3 || m < 2 || m > n1 - 3) { o[0] = o[1] = o[2] = o[3] = 0.f; }
-            if (first_col) { o[0] = 0.f; o[1] = 0.f; }
-            if (last_col) { o[2] = 0.f; o[3] = 0.f; }
+        const V4 s1x = v4add(q1, q3), s2x = v4add(q0, q4);
+        const V4 s1y = v4add(a1v, b1v), s2y = v4add(a2v, b2v);
+        V4 s1z, s2z;
+        s1z.lo = make_float2(l1 + q2.lo.y, q2.lo.x + q2.hi.x);
+        s1z.hi = make_float2(q2.lo.y + q2.hi.y, q2.hi.x + r1);
+        s2z.lo = make_float2(l2 + q2.hi.x, l1 + q2.hi.y);
+        s2z.hi = make_float2(q2.lo.x + r1, q2.lo.y + r2);
+        V4 o = v4mul(q2, p.kc);
+        o = v4fma(s1x, p.w16[0], o); o = v4fma(s2x, p.nw[0], o);
+        o = v4fma(s1y, p.w16[1], o); o = v4fma(s2y, p.nw[1], o);
+        o = v4fma(s1z, p.w16[2], o); o = v4fma(s2z, p.nw[2], o);
+        if (FWD) {
+            o = v4sub(o, src);
+            // nodes of the two outer layers carry no row
+            if (a < 2 || a > n0 - 3 || m < 2 || m > n1 - 3) { o = v4zero(); }
+            if (first_col) o.lo = make_float2(0.f, 0.f);
+            if (last_col) o.hi = make_float2(0.f, 0.f);
         }
         if (valid) {
-            const float4 ov = make_float4(o[0], o[1], o[2], o[3]);
-            st4(p.out + ((size_t)a * n1 + m) * n2 + 4 * c4, ov);
-            if (FWD) acc[0] += sq4(ov);
+            stv4(p.out + a * PS + mc * n2 + col, o.lo, o.hi);
+            if (FWD) acc = fma2(o.lo, o.lo, fma2(o.hi, o.hi, acc));
         }
-        q0 = q1; q1 = q2; q2 = q3; q3 = q4;
+    };
+
+    for (int a = a0; a < a1; a += 5) {
+        step(a, Q0, Q1, Q2, Q3, Q4);
+        if (a + 1 < a1) step(a + 1, Q1, Q2, Q3, Q4, Q0);
+        if (a + 2 < a1) step(a + 2, Q2, Q3, Q4, Q0, Q1);
+        if (a + 3 < a1) step(a + 3, Q3, Q4, Q0, Q1, Q2);
+        if (a + 4 < a1) step(a + 4, Q4, Q0, Q1, Q2, Q3);
     }
-    if (FWD && p.partials != nullptr) block_reduce_store<1>(acc, p.partials, p.nitems, blockIdx.x);
+    if (FWD && p.partials != nullptr) {
+        float s[1] = {acc.x + acc.y};
+        block_reduce_store<1>(s, p.partials, p.nitems, blockIdx.x);
+    }
 }
 
 static int env_int(const char* name, int dflt) {
@@ -119,47 +149,54 @@ static int env_int(const char* name, int dflt) {
     return v > 0 ? v : dflt;
 }
 
-static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block) {
+static float2 sp(double v) { return make_float2((float)v, (float)v); }
+
+static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, double scale) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n2 = q.n[2]; p.nc4 = q.n[2] / 4;
-    int tx = p.nc4 >= 64 ? 64 : 32;
+    int tx = p.nc4 > 32 ? 64 : 32;
     tx = env_int("FPDE_STAR3D_TX", tx);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
     int ty = env_int("FPDE_STAR3D_TY", 4);
-    ty = std::max(1, std::min(256 / tx, ty));
+    ty = std::max(1, std::min(512 / tx, ty));
     block = dim3(tx, ty, 1);
     p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 32);
     p.ncb = (p.nc4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
-    p.w0 = (float)(1.0 / (12.0 * q.h[0] * q.h[0]));
-    p.w1 = (float)(1.0 / (12.0 * q.h[1] * q.h[1]));
-    p.w2 = (float)(1.0 / (12.0 * q.h[2] * q.h[2]));
-    p.k2 = (float)(q.coef[0] * q.coef[0]);
+    double wsum = 0.0;
+    for (int a = 0; a < 3; ++a) {
+        const double w = 1.0 / (12.0 * q.h[a] * q.h[a]);
+        p.w16[a] = sp(16.0 * w * scale);
+        p.nw[a] = sp(-w * scale);
+        wsum += w;
+    }
+    p.kc = sp((q.coef[0] * q.coef[0] - 30.0 * wsum) * scale);
+    const char* pf = std::getenv("FPDE_STAR3D_PREFETCH");
+    p.prefetch = pf && *pf ? std::atoi(pf) : 3;
+    if (p.prefetch < 0) p.prefetch = 0;
 }
 
 int star3d_items(const int* n) {
     Problem q{}; q.n[0] = n[0]; q.n[1] = n[1]; q.n[2] = n[2]; q.h[0] = q.h[1] = q.h[2] = 1.0;
     Star3dParams p{}; dim3 block;
-    star3d_geometry(q, p, block);
+    star3d_geometry(q, p, block, 1.0);
     return p.nitems;
 }
 
 cudaError_t launch_helmholtz_fwd(const Problem& q) {
     Star3dParams p{}; dim3 block;
-    star3d_geometry(q, p, block);
-    p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0]; p.hscale = 1.f;
+    star3d_geometry(q, p, block, 1.0);
+    p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0];
     p.partials = q.partials;
-    star3d_kernel<true><<<p.nitems, block, 0, q.stream>>>(p);
-    return cudaGetLastError();
+    return launch_kernel(star3d_kernel<true>, dim3(p.nitems), block, q.stream, p);
 }
 
 cudaError_t launch_helmholtz_bwd(const Problem& q) {
     Star3dParams p{}; dim3 block;
-    star3d_geometry(q, p, block);
-    p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0]; p.hscale = (float)q.gscale[0];
+    star3d_geometry(q, p, block, q.gscale[0]);      // the operator is linear: the scale goes into the weights
+    p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0];
     p.partials = nullptr;
-    star3d_kernel<false><<<p.nitems, block, 0, q.stream>>>(p);
-    return cudaGetLastError();
+    return launch_kernel(star3d_kernel<false>, dim3(p.nitems), block, q.stream, p);
 }
 
 }  // namespace fpde

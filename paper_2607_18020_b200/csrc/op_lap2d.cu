@@ -97,6 +97,7 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
     constexpr bool BWD = F::BWD;
     constexpr bool MASK_IN = BWD && !PERIODIC;     // upstream array is zero outside the rows
     constexpr bool MASK_OUT = !BWD && !PERIODIC;   // ring nodes carry no row
+    pdl_wait_then_trigger();
     const int n0 = p.n0, n1 = p.n1, nc4 = p.nc4;
     const int item = blockIdx.x;
     const int cb = item % p.ncb, rc = item / p.ncb;
@@ -247,8 +248,7 @@ int lap2d_items(const int* n) {
 
 template <class F, bool PERIODIC>
 static cudaError_t launch(const Lap2dParams& p, int block, cudaStream_t s) {
-    lap2d_kernel<F, PERIODIC, 4><<<p.nitems, block, 0, s>>>(p);
-    return cudaGetLastError();
+    return launch_kernel(lap2d_kernel<F, PERIODIC, 4>, dim3(p.nitems), dim3(block), s, p);
 }
 
 static float2 sp(double v) { return make_float2((float)v, (float)v); }

@@ -112,6 +112,7 @@ __device__ __forceinline__ void t_neighbours(const V4& c, const float* __restric
 // ------------------------------------------------------------------------------------------
 template <bool TSAFE, int MINB>
 __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
+    pdl_wait_then_trigger();
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
     const int n0 = p.n0;
@@ -232,6 +233,7 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
 // ------------------------------------------------------------------------------------------
 template <bool TSAFE, int MINB>
 __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
+    pdl_wait_then_trigger();
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
     const int n0 = p.n0;
@@ -388,10 +390,11 @@ cudaError_t launch_ns_fwd(const Problem& q) {
     p.iht = sp(0.5 / q.h[3]);
     p.partials = q.partials;
     const int minb = env_int("FPDE_NS_MINB_F", 3);
-    if (!ns_tsafe(p)) ns_fwd_kernel<false, 3><<<p.nitems, block, 0, q.stream>>>(p);
-    else if (minb == 3) ns_fwd_kernel<true, 3><<<p.nitems, block, 0, q.stream>>>(p);
-    else ns_fwd_kernel<true, 4><<<p.nitems, block, 0, q.stream>>>(p);
-    return cudaGetLastError();
+    cudaError_t ce;
+    if (!ns_tsafe(p)) ce = launch_kernel(ns_fwd_kernel<false, 3>, dim3(p.nitems), block, q.stream, p);
+    else if (minb == 3) ce = launch_kernel(ns_fwd_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
+    else ce = launch_kernel(ns_fwd_kernel<true, 4>, dim3(p.nitems), block, q.stream, p);
+    return ce;
 }
 
 cudaError_t launch_ns_bwd(const Problem& q) {
@@ -413,10 +416,11 @@ cudaError_t launch_ns_bwd(const Problem& q) {
     }
     p.partials = nullptr;
     const int minb = env_int("FPDE_NS_MINB_B", 2);
-    if (!ns_tsafe(p)) ns_bwd_kernel<false, 2><<<p.nitems, block, 0, q.stream>>>(p);
-    else if (minb == 3) ns_bwd_kernel<true, 3><<<p.nitems, block, 0, q.stream>>>(p);
-    else ns_bwd_kernel<true, 2><<<p.nitems, block, 0, q.stream>>>(p);
-    return cudaGetLastError();
+    cudaError_t ce;
+    if (!ns_tsafe(p)) ce = launch_kernel(ns_bwd_kernel<false, 2>, dim3(p.nitems), block, q.stream, p);
+    else if (minb == 3) ce = launch_kernel(ns_bwd_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
+    else ce = launch_kernel(ns_bwd_kernel<true, 2>, dim3(p.nitems), block, q.stream, p);
+    return ce;
 }
 
 }  // namespace fpde
