@@ -40,7 +40,7 @@ __device__ __forceinline__ void prefetch_l2_line(const float* ptr) {
 }
 
 template <bool FWD>
-__global__ void __launch_bounds__(512) star3d_kernel(const Star3dParams p) {
+__global__ void __launch_bounds__(256, 4) star3d_kernel(const Star3dParams p) {
     pdl_wait_then_trigger();
     const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
     int item = blockIdx.x;
@@ -157,9 +157,9 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     tx = env_int("FPDE_STAR3D_TX", tx);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
     int ty = env_int("FPDE_STAR3D_TY", 4);
-    ty = std::max(1, std::min(512 / tx, ty));
+    ty = std::max(1, std::min(256 / tx, ty));
     block = dim3(tx, ty, 1);
-    p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 32);
+    p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 16);
     p.ncb = (p.nc4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
@@ -172,7 +172,7 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     }
     p.kc = sp((q.coef[0] * q.coef[0] - 30.0 * wsum) * scale);
     const char* pf = std::getenv("FPDE_STAR3D_PREFETCH");
-    p.prefetch = pf && *pf ? std::atoi(pf) : 3;
+    p.prefetch = pf && *pf ? std::atoi(pf) : 2;
     if (p.prefetch < 0) p.prefetch = 0;
 }
 
