@@ -196,6 +196,41 @@ int fpde_loss_grad_host(int op,
                         void* d_arena, size_t arena_bytes,
                         void* stream);
 
+/*
+ * fpde_fwd for callers that cannot allocate device memory.  (The paper has no counterpart; this
+ * is a convenience of this library.)
+ *
+ * Who needs it: code that runs where a device allocation is forbidden or impossible -- inside a
+ * region that must not synchronise the device (cudaMalloc does), in a plug-in that is handed
+ * tensors but no allocator, or late in a job whose memory pool is already fully committed.  Such
+ * callers can supply inputs and outputs but no workspace.
+ *
+ * Same arguments and results as fpde_fwd, without `workspace`: the loss partial sums go to a
+ * fixed array that is part of the library image (FPDE_NOALLOC_SCRATCH_BYTES bytes of device
+ * memory on every GPU that loads the library, held until the process exits).  The call makes no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ *   - Grids whose forward pass needs more scratch than that (fpde_workspace_bytes() >
+ *     FPDE_NOALLOC_SCRATCH_BYTES) are refused with FPDE_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - Every call on a device shares the one array.  The kernels overwrite every slot they later
+ *     read, so nothing has to be cleared between calls, but two calls that overlap on the GPU
+ *     (different streams, no ordering) race on it: order them, or use fpde_fwd with separate
+ *     workspaces.
+ */
+#define FPDE_NOALLOC_SCRATCH_BYTES (256u * 1024u)
+int fpde_fwd_noalloc(int op,
+                     const float* const* fields,
+                     const float* const* sources,
+                     float* const* residuals,
+                     double* loss_out,
+                     int ndim, const int64_t* shape,
+                     const double* spacing,
+                     const double* coeffs, int ncoeffs,
+                     const int* bc,
+                     void* stream);
+
 #ifdef __cplusplus
 }
 #endif

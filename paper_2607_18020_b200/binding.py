@@ -72,6 +72,11 @@ def lib():
                                           ctypes.POINTER(ctypes.c_double), ctypes.c_int,
                                           ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_size_t,
                                           ctypes.c_void_p]
+        L.fpde_fwd_noalloc.restype = ctypes.c_int
+        L.fpde_fwd_noalloc.argtypes = [ctypes.c_int, vpp, vpp, vpp, ctypes.c_void_p, ctypes.c_int,
+                                       ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                       ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                                       ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -219,3 +224,26 @@ def fpde_loss_grad_host(op, h_fields, h_sources, h_gfields, h_loss, shape, spaci
                                _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_loss_grad_host")
+
+
+NOALLOC_SCRATCH_BYTES = 256 * 1024      # FPDE_NOALLOC_SCRATCH_BYTES of include/fpde.h
+
+
+def fwd_noalloc_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, stream) -> int:
+    return lib().fpde_fwd_noalloc(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(sources)),
+                                  _ptr_array(_dev_ptrs(residuals)),
+                                  _dev_ptrs([loss_out])[0] if loss_out is not None else None,
+                                  len(shape), _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                                  stream)
+
+
+def fpde_fwd_noalloc(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, stream=None):
+    """fpde_fwd for callers that cannot allocate a workspace (no allocator at hand, or a region
+    where cudaMalloc must not be called): the loss partial sums live in a fixed array inside the
+    library.  Grids needing more than NOALLOC_SCRATCH_BYTES of scratch raise FpdeError (status 9).
+    Calls on one device share that array, so keep them ordered on the GPU; make the first call on
+    a device outside stream capture."""
+    st = fwd_noalloc_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc,
+                            _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_fwd_noalloc")

@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 namespace fpde {
 
@@ -316,6 +317,51 @@ int fpde_loss_grad_host(int op, const float* const* h_fields, const float* const
     if (cudaMemcpyAsync(h_loss, d_loss, (e.ne + 1) * sizeof(double), cudaMemcpyDeviceToHost, cs) != cudaSuccess)
         return FPDE_ERR_CUDA;
     return FPDE_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// fpde_fwd_noalloc: the forward pass with its scratch in a fixed array of the library image.
+// In host code the array's name is only a handle; the device address comes from
+// cudaGetSymbolAddress, looked up once per device with that device current.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[FPDE_NOALLOC_SCRATCH_BYTES];
+
+static constexpr int NOALLOC_MAX_DEVICES = 64;
+static std::mutex g_noalloc_mutex;
+static void* g_noalloc_addr[NOALLOC_MAX_DEVICES];      // per device, filled on first use
+
+static cudaError_t noalloc_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce != cudaSuccess) return ce;
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_addr[dev] == nullptr) {
+        void* addr = nullptr;
+        ce = cudaGetSymbolAddress(&addr, g_noalloc_scratch);
+        if (ce != cudaSuccess) return ce;
+        g_noalloc_addr[dev] = addr;
+    }
+    *out = g_noalloc_addr[dev];
+    return cudaSuccess;
+}
+
+int fpde_fwd_noalloc(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+                     double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+                     const double* coeffs, int ncoeffs, const int* bc, void* stream) {
+    // refuse grids beyond the fixed scratch before touching the device
+    const size_t need = fpde_workspace_bytes(op, ndim, shape);
+    if (need == 0) {                       // invalid op / shape: let the common validation name the error
+        return fpde_fwd(op, fields, sources, residuals, nullptr, ndim, shape, spacing, coeffs, ncoeffs, bc,
+                        nullptr, 0, stream);
+    }
+    if (loss_out != nullptr && need > FPDE_NOALLOC_SCRATCH_BYTES) return FPDE_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    if (loss_out != nullptr) {
+        if (noalloc_scratch_address(&scratch) != cudaSuccess) return FPDE_ERR_CUDA;
+    }
+    return fpde_fwd(op, fields, sources, residuals, loss_out, ndim, shape, spacing, coeffs, ncoeffs, bc,
+                    scratch, scratch ? (size_t)FPDE_NOALLOC_SCRATCH_BYTES : 0, stream);
 }
 
 }  // extern "C"
