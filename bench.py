@@ -302,6 +302,21 @@ def config_line(torch, B, name, steps, warmup, peak):
     return out
 
 
+def max_over_ranks(x: float, dist, device) -> float:
+    """Slowest rank's figure (the job is as slow as its slowest replica); identity on one rank."""
+    if dist is None:
+        return x
+    import torch
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, points_per_rank: int, steps: int, slowest_ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas: all points processed / slowest time."""
+    return world * points_per_rank * steps / (slowest_ms * 1e-3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -337,13 +352,6 @@ def main():
         if dist is not None:
             dist.barrier()
 
-    def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     peak, peak_src = measured_peak()
     shape = [int(x) for x in args.shape.split(",")] if args.shape else None
     w = W.make(args.workload, seed=42 + rank, shape=shape,
@@ -357,16 +365,16 @@ def main():
     # same K steps again with an event pair around every call: per-kernel durations for the roofline
     _, fwd_ms, bwd_ms = timed_steps(torch, prob, args.steps, 0, barrier, inner_events=True)
     sampler.stop()
-    total_ms = max_over_ranks(total_ms)
-    value = world * N * args.steps / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
+    value = job_value(world, N, args.steps, total_ms)
 
     e2e_k = max(1, min(args.steps, 20))
     if args.no_e2e:
         e2e_ms, h2d, d2h = float("nan"), 0, 0
     else:
         e2e_ms, h2d, d2h, _ = e2e_steps(torch, B, w, e2e_k, 3, barrier)
-    e2e_ms = max_over_ranks(e2e_ms)
-    e2e_value = world * N * e2e_k / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
+    e2e_value = job_value(world, N, e2e_k, e2e_ms)
 
     fb, bb = ALGO_BYTES[w.op]
     f_avg, b_avg = sum(fwd_ms) / len(fwd_ms), sum(bwd_ms) / len(bwd_ms)
