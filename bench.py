@@ -55,6 +55,13 @@ KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None where no capture has been taken yet.
 NCU_TRAFFIC_BYTES = {
+    # half-size capture (64 planes) x 2: traffic is proportional to the number of planes
+    ("ns_tgv_128x16", "ns_fwd_kernel"): 2 * 516411904,
+    ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 772324352,
+    ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 231791104,
+    ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 376371968,
+    ("helmholtz_256", "star3d_kernel<fwd>"): 188598784,
+    ("helmholtz_256", "star3d_kernel<bwd>"): 98334720,
 }
 FALLBACK_HBM_GBS = 6650.0
 LAUNCHES_PER_STEP = 3               # forward kernel, loss finalise, adjoint kernel

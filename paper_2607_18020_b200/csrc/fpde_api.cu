@@ -99,34 +99,57 @@ static int validate(int op, const float* const* fields, int ndim, const int64_t*
     return FPDE_OK;
 }
 
-// Fixed-order final sum: thread t adds partials t, t+256, ... in fp64, then a shared-memory
-// tree of fixed shape.  One block, so no inter-block ordering exists to vary.
-__global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restrict__ partials, int nitems,
-                                                            int nres, double inv_rows,
-                                                            double* __restrict__ loss_out) {
-    __shared__ double sm[256];
+// Fixed-order final sum.  Thread t adds partials t, t+1024, ... (four independent loads in
+// flight, combined in a fixed order) in fp64; then a shuffle tree inside each warp and one over
+// the 32 warp sums.  One block, so no inter-block ordering exists to vary: the result depends
+// on the data only.
+__global__ void __launch_bounds__(1024) loss_finalize_kernel(const float* __restrict__ partials, int nitems,
+                                                             int nres, double inv_rows,
+                                                             double* __restrict__ loss_out) {
+    __shared__ double sm[MAX_F][32];
     pdl_wait_then_trigger();
-    double total = 0.0;
-    for (int e = 0; e < nres; ++e) {
-        double s = 0.0;
-        for (int i = threadIdx.x; i < nitems; i += 256) s += (double)partials[(size_t)e * nitems + i];
-        sm[threadIdx.x] = s;
-        __syncthreads();
-        for (int o = 128; o > 0; o >>= 1) {
-            if ((int)threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
-            __syncthreads();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double s[MAX_F];
+#pragma unroll
+    for (int e = 0; e < MAX_F; ++e) {
+        s[e] = 0.0;
+        if (e < nres) {
+            const float* p = partials + (size_t)e * nitems;
+            int i = tid;
+            for (; i + 3072 < nitems; i += 4096) {
+                const float a = p[i], b = p[i + 1024], c = p[i + 2048], d = p[i + 3072];
+                s[e] += ((double)a + (double)b) + ((double)c + (double)d);
+            }
+            for (; i < nitems; i += 1024) s[e] += (double)p[i];
         }
-        const double le = sm[0] * inv_rows;
-        if (threadIdx.x == 0) loss_out[e] = le;
-        total += le;
-        __syncthreads();
     }
-    if (threadIdx.x == 0) loss_out[nres] = total;
+#pragma unroll
+    for (int e = 0; e < MAX_F; ++e) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s[e] += __shfl_down_sync(FULL_MASK, s[e], o);
+        if (lane == 0) sm[e][warp] = s[e];
+    }
+    __syncthreads();
+    if (warp == 0) {
+        double total = 0.0;
+#pragma unroll
+        for (int e = 0; e < MAX_F; ++e) {
+            double v = sm[e][lane];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(FULL_MASK, v, o);
+            if (e < nres) {
+                const double le = v * inv_rows;
+                if (lane == 0) loss_out[e] = le;
+                total += le;
+            }
+        }
+        if (lane == 0) loss_out[nres] = total;
+    }
 }
 
 cudaError_t launch_loss_finalize(const float* partials, int nitems, int nres, int64_t rows,
                                  double* loss_out, cudaStream_t stream) {
-    return launch_kernel(loss_finalize_kernel, dim3(1), dim3(256), stream, partials, nitems, nres,
+    return launch_kernel(loss_finalize_kernel, dim3(1), dim3(1024), stream, partials, nitems, nres,
                          1.0 / (double)rows, loss_out);
 }
 
