@@ -231,6 +231,15 @@ int fpde_fwd_noalloc(int op,
                      const int* bc,
                      void* stream);
 
+/*
+ * Diagnostic.  The Navier-Stokes kernels that stage their tiles through shared memory with the
+ * copy engine wait on memory barriers with an iteration limit instead of spinning for ever; this
+ * returns how many such waits have given up on the current device since the library was loaded
+ * (0 in a healthy run; results of a launch that timed out are garbage).  Synchronises the device.
+ * Returns UINT_MAX if the counter cannot be read.
+ */
+unsigned int fpde_diag_tma_timeouts(void);
+
 #ifdef __cplusplus
 }
 #endif

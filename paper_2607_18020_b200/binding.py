@@ -77,6 +77,8 @@ def lib():
                                        ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                        ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                        ctypes.c_void_p]
+        L.fpde_diag_tma_timeouts.restype = ctypes.c_uint
+        L.fpde_diag_tma_timeouts.argtypes = []
         _lib = L
     return _lib
 
@@ -247,3 +249,8 @@ def fpde_fwd_noalloc(op, fields, sources, residuals, loss_out, shape, spacing, c
                             _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd_noalloc")
+
+
+def diag_tma_timeouts() -> int:
+    """Bounded barrier waits that gave up on the current device (0 in a healthy run)."""
+    return int(lib().fpde_diag_tma_timeouts())

@@ -387,4 +387,6 @@ int fpde_fwd_noalloc(int op, const float* const* fields, const float* const* sou
                     scratch, scratch ? (size_t)FPDE_NOALLOC_SCRATCH_BYTES : 0, stream);
 }
 
+unsigned int fpde_diag_tma_timeouts(void) { return ns_tma_timeouts(); }
+
 }  // extern "C"

@@ -41,6 +41,18 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
 }
 
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem_bytes,
+                                      cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem_bytes; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+
 // Number of loss partial sums (= work items) per residual field the forward kernel of this
 // operator produces for this grid.  Fixed by the grid alone, so the reduction order is too.
 int fwd_items(int op, const int* n);
@@ -53,6 +65,12 @@ cudaError_t launch_lap2d_bwd(const Problem& p);
 cudaError_t launch_helmholtz_fwd(const Problem& p);
 cudaError_t launch_helmholtz_bwd(const Problem& p);
 cudaError_t launch_ns_fwd(const Problem& p);
+// TMA-staged variants (op_ns3dt_tma.cu); `launched` false = this grid is not eligible
+bool ns_tma_wanted(const int* n);
+int ns_tma_items(const int* n);
+cudaError_t launch_ns_fwd_tma(const Problem& p, bool& launched);
+cudaError_t launch_ns_bwd_tma(const Problem& p, bool& launched);
+unsigned int ns_tma_timeouts();
 cudaError_t launch_ns_bwd(const Problem& p);
 
 // Final, fixed-order fp64 sum of the per-item partials: loss_out[e] = sum/N_r, loss_out[E] = total.

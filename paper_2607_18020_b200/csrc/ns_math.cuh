@@ -1,0 +1,177 @@
+// Per-node arithmetic of the unsteady Navier-Stokes operator, shared by the kernels that stage
+// their neighbours through L1 and those that stage them through shared memory.  Everything is
+// packed fp32x2: a float4 (four consecutive t of one z) is two register-aligned pairs.
+//
+// Forward (Section 2.1 extended by d_t, w, d_z), per momentum component q along axis a_q:
+//   mom_q = d_t q + u d_x q + v d_y q + w d_z q + d_{a_q} p - nu (d_xx + d_yy + d_zz) q
+//   cont  = d_x u + d_y v + d_z w
+// Adjoint (Eq. 1 / Appendix A.2 extended the same way), G = upstream arrays (zero at the first
+// and last t), c = (u,v,w):
+//   g_q(P) = sum_e G_e(P) (d_{a_q} e)(P)                                   local terms
+//          + sum_a [ (G_q c_a)(P-a) - (G_q c_a)(P+a) ] / (2 h_a)           transposed advection
+//          - nu sum_a [ G_q(P-a) - 2 G_q(P) + G_q(P+a) ] / h_a^2           transposed diffusion
+//          + [ G_q(P-t) - G_q(P+t) ] / (2 dt)                              transposed d_t
+//          + [ G_c(P-a_q) - G_c(P+a_q) ] / (2 h_{a_q})                     continuity row
+//   g_p(P) = sum_q [ G_q(P-a_q) - G_q(P+a_q) ] / (2 h_{a_q})
+// with G_e = gscale_e * gres_e; the scales are folded into the constants.
+//
+// Second differences are formed as (q[-1]-q[0]) + (q[+1]-q[0]) before scaling: the viscous term
+// is small against the other terms and must not carry the rounding of the large centre value.
+//
+// Nodes at the first / last t carry no row.  Every spatial read of an output node happens at the
+// node's own t, so in the adjoint that rule only changes (i) the t-neighbour of the nodes next
+// to the two end planes and (ii) the end planes themselves, where only the transposed d_t term
+// survives: the boundary-gradient correction of this operator is a fix-up of two lanes.
+#pragma once
+#include "fpde_common.cuh"
+
+namespace fpde {
+
+struct NsConsts {
+    // forward, splatted
+    float2 ih[3];         // 1/(2 h_a)
+    float2 iht;           // 1/(2 dt)
+    float2 nv[3];         // -nu / h_a^2
+    // adjoint (upstream scales folded in), splatted
+    float2 a_ih[3][3];    // [q][a]  gs_q / (2 h_a)
+    float2 a_nv[3][3];    // [q][a]  -nu gs_q / h_a^2
+    float2 a_t[3];        // [q]     gs_q / (2 dt)
+    float2 l_g[3];        // [e]     gs_e
+    float2 c_ih[3];       // [a]     gs_c / (2 h_a)
+};
+
+// W0/W1/W2: planes x-1, x, x+1 at the own column; Ym/Yp/Zm/Zp: y-+1 and z-+1 neighbours of plane x;
+// arrays u,v,w,p.  l1/r1: t-1 of lane x and t+1 of lane w for u,v,w.  o[e][half].
+__device__ __forceinline__ void ns_fwd_math(const NsConsts& k, const V4 (&W0)[4], const V4 (&W1)[4], const V4 (&W2)[4],
+                                            const V4 (&Ym)[4], const V4 (&Yp)[4], const V4 (&Zm)[4], const V4 (&Zp)[4],
+                                            const float (&l1)[3], const float (&r1)[3], bool t_first, bool t_last,
+                                            float2 (&o)[4][2]) {
+    float2 dtl[3], dth[3];                      // q(t+1) - q(t-1), lanes (x,y) and (z,w)
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        const V4 c = W1[q];
+        dtl[q] = make_float2(c.lo.y - l1[q], c.hi.x - c.lo.x);
+        dth[q] = make_float2(c.hi.y - c.lo.y, r1[q] - c.hi.x);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {               // the two packed halves of the float4
+        auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
+        const float2 us = mul2(H(W1[0]), k.ih[0]);   // advecting velocities, pre-scaled by 1/(2h)
+        const float2 vs = mul2(H(W1[1]), k.ih[1]);
+        const float2 ws = mul2(H(W1[2]), k.ih[2]);
+        float2 dself[3];                        // d_x u, d_y v, d_z w (raw differences)
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const float2 c = H(W1[q]);
+            const float2 xm = sub2(H(W0[q]), c), xp = sub2(H(W2[q]), c);
+            const float2 ym = sub2(H(Ym[q]), c), yp = sub2(H(Yp[q]), c);
+            const float2 zm = sub2(H(Zm[q]), c), zp = sub2(H(Zp[q]), c);
+            const float2 dx = sub2(xp, xm), dy = sub2(yp, ym), dz = sub2(zp, zm);
+            float2 r = mul2(add2(xm, xp), k.nv[0]);
+            r = fma2(add2(ym, yp), k.nv[1], r);
+            r = fma2(add2(zm, zp), k.nv[2], r);
+            r = fma2(us, dx, r);
+            r = fma2(vs, dy, r);
+            r = fma2(ws, dz, r);
+            r = fma2(h == 0 ? dtl[q] : dth[q], k.iht, r);
+            dself[q] = q == 0 ? dx : (q == 1 ? dy : dz);
+            o[q][h] = r;
+        }
+        o[0][h] = fma2(sub2(H(W2[3]), H(W0[3])), k.ih[0], o[0][h]);     // d_x p
+        o[1][h] = fma2(sub2(H(Yp[3]), H(Ym[3])), k.ih[1], o[1][h]);     // d_y p
+        o[2][h] = fma2(sub2(H(Zp[3]), H(Zm[3])), k.ih[2], o[2][h]);     // d_z p
+        o[3][h] = fma2(dself[2], k.ih[2], fma2(dself[1], k.ih[1], mul2(dself[0], k.ih[0])));
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {               // t = 0 and t = n3-1 carry no row
+        if (t_first) o[e][0].x = 0.f;
+        if (t_last) o[e][1].y = 0.f;
+    }
+}
+
+// Arrays 0..2: u,v,w ; 3..6: upstream of mom_x, mom_y, mom_z, continuity.  l1/r1: t-1 of lane x
+// and t+1 of lane w of the three momentum upstream arrays.
+__device__ __forceinline__ void ns_bwd_math(const NsConsts& k, const V4 (&W0)[7], const V4 (&W1)[7], const V4 (&W2)[7],
+                                            const V4 (&Ym)[7], const V4 (&Yp)[7], const V4 (&Zm)[7], const V4 (&Zp)[7],
+                                            const float (&l1)[3], const float (&r1)[3], bool t_first, bool t_last,
+                                            float2 (&o)[4][2]) {
+    float2 dtl[3], dth[3];                      // G_q(t-1) - G_q(t+1) with the end planes counted as 0
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        const V4 c = W1[3 + q];
+        const float tm_y = t_first ? 0.f : c.lo.x;       // t-1 of lane y is the end plane t = 0
+        const float tp_z = t_last ? 0.f : c.hi.y;        // t+1 of lane z is the end plane t = n3-1
+        dtl[q] = make_float2(l1[q] - c.lo.y, tm_y - c.hi.x);
+        dth[q] = make_float2(c.lo.y - tp_z, c.hi.x - r1[q]);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
+        // neighbours of array i along axis a: minus / plus
+        auto NM = [&](int i, int a_) -> float2 { return a_ == 0 ? H(W0[i]) : (a_ == 1 ? H(Ym[i]) : H(Zm[i])); };
+        auto NP = [&](int i, int a_) -> float2 { return a_ == 0 ? H(W2[i]) : (a_ == 1 ? H(Yp[i]) : H(Zp[i])); };
+        float2 gs[3];                            // scaled centre sensitivities
+#pragma unroll
+        for (int e = 0; e < 3; ++e) gs[e] = mul2(H(W1[3 + e]), k.l_g[e]);
+        float2 cm[3], ncp[3];                    // advecting velocity at P-a, minus the one at P+a
+#pragma unroll
+        for (int a_ = 0; a_ < 3; ++a_) {
+            cm[a_] = NM(a_, a_);
+            const float2 cp = NP(a_, a_);
+            ncp[a_] = make_float2(-cp.x, -cp.y);
+        }
+        float2 gp = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const float2 c = H(W1[3 + q]);
+            float2 r = mul2(h == 0 ? dtl[q] : dth[q], k.a_t[q]);
+#pragma unroll
+            for (int a_ = 0; a_ < 3; ++a_) {
+                const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
+                const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
+                r = fma2(adv, k.a_ih[q][a_], r);
+                const float2 dm = sub2(gm, c), dp = sub2(gpl, c);
+                r = fma2(add2(dm, dp), k.a_nv[q][a_], r);
+                if (a_ == q) gp = fma2(sub2(dm, dp), k.a_ih[q][q], gp);
+            }
+            // local terms and continuity row along this component's own axis
+            float2 loc = mul2(gs[0], sub2(NP(0, q), NM(0, q)));
+            loc = fma2(gs[1], sub2(NP(1, q), NM(1, q)), loc);
+            loc = fma2(gs[2], sub2(NP(2, q), NM(2, q)), loc);
+            r = fma2(loc, k.ih[q], r);
+            r = fma2(sub2(NM(6, q), NP(6, q)), k.c_ih[q], r);
+            o[q][h] = r;
+        }
+        o[3][h] = gp;
+    }
+    // end planes of t: only the transposed d_t term exists there, and no pressure gradient
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        const V4 c = W1[3 + q];
+        if (t_first) o[q][0].x = -c.lo.y * k.a_t[q].x;
+        if (t_last) o[q][1].y = c.hi.x * k.a_t[q].x;
+    }
+    if (t_first) o[3][0].x = 0.f;
+    if (t_last) o[3][1].y = 0.f;
+}
+
+// Host side: fill the constants from spacings, viscosity and upstream scales.
+inline void ns_fill_consts(NsConsts& k, const double* h, double nu, const double* gscale) {
+    auto sp = [](double v) { return make_float2((float)v, (float)v); };
+    for (int a = 0; a < 3; ++a) {
+        k.ih[a] = sp(0.5 / h[a]);
+        k.nv[a] = sp(-nu / (h[a] * h[a]));
+        k.c_ih[a] = sp(gscale[3] * 0.5 / h[a]);
+    }
+    k.iht = sp(0.5 / h[3]);
+    for (int q = 0; q < 3; ++q) {
+        k.a_t[q] = sp(gscale[q] * 0.5 / h[3]);
+        k.l_g[q] = sp(gscale[q]);
+        for (int a = 0; a < 3; ++a) {
+            k.a_ih[q][a] = sp(gscale[q] * 0.5 / h[a]);
+            k.a_nv[q][a] = sp(-nu * gscale[q] / (h[a] * h[a]));
+        }
+    }
+}
+
+}  // namespace fpde

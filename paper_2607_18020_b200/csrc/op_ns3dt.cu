@@ -24,6 +24,7 @@
 // it is applied as a fix-up of two lanes instead of masking every load.
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
+#include "ns_math.cuh"
 
 #include <algorithm>
 #include <cstdlib>
@@ -37,16 +38,7 @@ struct NsParams {
     int n0, n1, n3;       // x, y extents; t extent
     int C, C4, nt4;       // row length in floats / float4, float4 per z
     int planes_per_item, ncb, nmb, nitems;
-    // forward constants, splatted
-    float2 ih[3];         // 1/(2 h_a)
-    float2 iht;           // 1/(2 dt)
-    float2 nv[3];         // -nu / h_a^2
-    // adjoint constants (upstream scales folded in), splatted
-    float2 a_ih[3][3];    // [q][a]  gs_q / (2 h_a)
-    float2 a_nv[3][3];    // [q][a]  -nu gs_q / h_a^2
-    float2 a_t[3];        // [q]     gs_q / (2 dt)
-    float2 l_g[3];        // [e]     gs_e
-    float2 c_ih[3];       // [a]     gs_c / (2 h_a)
+    NsConsts k;
     float* partials;
     int prefetch;         // planes ahead of the window to prefetch into L2 (0 = off)
 };
@@ -153,50 +145,11 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
             Zm[k] = ldv4(fp[k] + pl + ix.rowoff + ix.zmcol);
             Zp[k] = ldv4(fp[k] + pl + ix.rowoff + ix.zpcol);
         }
-        float2 dtl[3], dth[3];                      // q(t+1) - q(t-1), lanes (x,y) and (z,w)
+        float l1[3], r1[3];
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            float l1, r1;
-            t_neighbours<TSAFE>(W1[k], fp[k] + pl + ix.rowoff, ix, l1, r1);
-            const V4 c = W1[k];
-            dtl[k] = make_float2(c.lo.y - l1, c.hi.x - c.lo.x);
-            dth[k] = make_float2(c.hi.y - c.lo.y, r1 - c.hi.x);
-        }
+        for (int k = 0; k < 3; ++k) t_neighbours<TSAFE>(W1[k], fp[k] + pl + ix.rowoff, ix, l1[k], r1[k]);
         float2 o[4][2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {               // the two packed halves of the float4
-            auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
-            const float2 us = mul2(H(W1[0]), p.ih[0]);   // advecting velocities, pre-scaled by 1/(2h)
-            const float2 vs = mul2(H(W1[1]), p.ih[1]);
-            const float2 ws = mul2(H(W1[2]), p.ih[2]);
-            float2 dself[3];                        // d_x u, d_y v, d_z w (raw differences)
-#pragma unroll
-            for (int k = 0; k < 3; ++k) {
-                const float2 c = H(W1[k]);
-                const float2 xm = sub2(H(W0[k]), c), xp = sub2(H(W2[k]), c);
-                const float2 ym = sub2(H(Ym[k]), c), yp = sub2(H(Yp[k]), c);
-                const float2 zm = sub2(H(Zm[k]), c), zp = sub2(H(Zp[k]), c);
-                const float2 dx = sub2(xp, xm), dy = sub2(yp, ym), dz = sub2(zp, zm);
-                float2 r = mul2(add2(xm, xp), p.nv[0]);
-                r = fma2(add2(ym, yp), p.nv[1], r);
-                r = fma2(add2(zm, zp), p.nv[2], r);
-                r = fma2(us, dx, r);
-                r = fma2(vs, dy, r);
-                r = fma2(ws, dz, r);
-                r = fma2(h == 0 ? dtl[k] : dth[k], p.iht, r);
-                dself[k] = k == 0 ? dx : (k == 1 ? dy : dz);
-                o[k][h] = r;
-            }
-            o[0][h] = fma2(sub2(H(W2[3]), H(W0[3])), p.ih[0], o[0][h]);     // d_x p
-            o[1][h] = fma2(sub2(H(Yp[3]), H(Ym[3])), p.ih[1], o[1][h]);     // d_y p
-            o[2][h] = fma2(sub2(H(Zp[3]), H(Zm[3])), p.ih[2], o[2][h]);     // d_z p
-            o[3][h] = fma2(dself[2], p.ih[2], fma2(dself[1], p.ih[1], mul2(dself[0], p.ih[0])));
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {               // t = 0 and t = n3-1 carry no row
-            if (ix.t_first) o[e][0].x = 0.f;
-            if (ix.t_last) o[e][1].y = 0.f;
-        }
+        ns_fwd_math(p.k, W0, W1, W2, Ym, Yp, Zm, Zp, l1, r1, ix.t_first, ix.t_last, o);
         if (ix.valid) {
             const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
@@ -267,67 +220,11 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
             Zm[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zmcol);
             Zp[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zpcol);
         }
-        float2 dtl[3], dth[3];                      // G_q(t-1) - G_q(t+1) with the end planes counted as 0
+        float l1[3], r1[3];
 #pragma unroll
-        for (int q = 0; q < 3; ++q) {
-            float l1, r1;
-            t_neighbours<TSAFE>(W1[3 + q], ap[3 + q] + pl + ix.rowoff, ix, l1, r1);
-            const V4 c = W1[3 + q];
-            const float tm_y = ix.t_first ? 0.f : c.lo.x;       // t-1 of lane y is the end plane t = 0
-            const float tp_z = ix.t_last ? 0.f : c.hi.y;        // t+1 of lane z is the end plane t = n3-1
-            dtl[q] = make_float2(l1 - c.lo.y, tm_y - c.hi.x);
-            dth[q] = make_float2(c.lo.y - tp_z, c.hi.x - r1);
-        }
+        for (int q = 0; q < 3; ++q) t_neighbours<TSAFE>(W1[3 + q], ap[3 + q] + pl + ix.rowoff, ix, l1[q], r1[q]);
         float2 o[4][2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
-            // neighbours of array k along axis a: minus / plus
-            auto NM = [&](int k, int a_) -> float2 { return a_ == 0 ? H(W0[k]) : (a_ == 1 ? H(Ym[k]) : H(Zm[k])); };
-            auto NP = [&](int k, int a_) -> float2 { return a_ == 0 ? H(W2[k]) : (a_ == 1 ? H(Yp[k]) : H(Zp[k])); };
-            float2 gs[3];                            // scaled centre sensitivities
-#pragma unroll
-            for (int e = 0; e < 3; ++e) gs[e] = mul2(H(W1[3 + e]), p.l_g[e]);
-            float2 cm[3], ncp[3];                    // advecting velocity at P-a, minus the one at P+a
-#pragma unroll
-            for (int a_ = 0; a_ < 3; ++a_) {
-                cm[a_] = NM(a_, a_);
-                const float2 cp = NP(a_, a_);
-                ncp[a_] = make_float2(-cp.x, -cp.y);
-            }
-            float2 gp = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int q = 0; q < 3; ++q) {
-                const float2 c = H(W1[3 + q]);
-                float2 r = mul2(h == 0 ? dtl[q] : dth[q], p.a_t[q]);
-#pragma unroll
-                for (int a_ = 0; a_ < 3; ++a_) {
-                    const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
-                    const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
-                    r = fma2(adv, p.a_ih[q][a_], r);
-                    const float2 dm = sub2(gm, c), dp = sub2(gpl, c);
-                    r = fma2(add2(dm, dp), p.a_nv[q][a_], r);
-                    if (a_ == q) gp = fma2(sub2(dm, dp), p.a_ih[q][q], gp);
-                }
-                // local terms and continuity row along this component's own axis
-                float2 loc = mul2(gs[0], sub2(NP(0, q), NM(0, q)));
-                loc = fma2(gs[1], sub2(NP(1, q), NM(1, q)), loc);
-                loc = fma2(gs[2], sub2(NP(2, q), NM(2, q)), loc);
-                r = fma2(loc, p.ih[q], r);
-                r = fma2(sub2(NM(6, q), NP(6, q)), p.c_ih[q], r);
-                o[q][h] = r;
-            }
-            o[3][h] = gp;
-        }
-        // end planes of t: only the transposed d_t term exists there, and no pressure gradient
-#pragma unroll
-        for (int q = 0; q < 3; ++q) {
-            const V4 c = W1[3 + q];
-            if (ix.t_first) o[q][0].x = -c.lo.y * p.a_t[q].x;
-            if (ix.t_last) o[q][1].y = c.hi.x * p.a_t[q].x;
-        }
-        if (ix.t_first) o[3][0].x = 0.f;
-        if (ix.t_last) o[3][1].y = 0.f;
+        ns_bwd_math(p.k, W0, W1, W2, Ym, Yp, Zm, Zp, l1, r1, ix.t_first, ix.t_last, o);
         if (ix.valid) {
             const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
@@ -349,8 +246,6 @@ static int env_int(const char* name, int dflt) {
     return v > 0 ? v : dflt;
 }
 
-static float2 sp(double v) { return make_float2((float)v, (float)v); }
-
 static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n3 = q.n[3];
     p.C = q.n[2] * q.n[3]; p.C4 = p.C / 4; p.nt4 = q.n[3] / 4;
@@ -371,6 +266,7 @@ static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
 static bool ns_tsafe(const NsParams& p) { return 32 % p.nt4 == 0; }
 
 int ns_items(const int* n) {
+    if (ns_tma_wanted(n)) return ns_tma_items(n);
     Problem q{};
     for (int a = 0; a < 4; ++a) { q.n[a] = n[a]; q.h[a] = 1.0; }
     NsParams p{}; dim3 block;
@@ -379,15 +275,16 @@ int ns_items(const int* n) {
 }
 
 cudaError_t launch_ns_fwd(const Problem& q) {
+    {
+        bool launched = false;
+        const cudaError_t ce = launch_ns_fwd_tma(q, launched);
+        if (launched || ce != cudaSuccess) return ce;
+    }
     NsParams p{}; dim3 block;
     ns_geometry(q, p, block);
     for (int k = 0; k < 4; ++k) { p.f[k] = q.in[k]; p.out[k] = q.out[k]; }
-    const double nu = q.coef[0];
-    for (int a = 0; a < 3; ++a) {
-        p.ih[a] = sp(0.5 / q.h[a]);
-        p.nv[a] = sp(-nu / (q.h[a] * q.h[a]));
-    }
-    p.iht = sp(0.5 / q.h[3]);
+    const double ones[4] = {1.0, 1.0, 1.0, 1.0};
+    ns_fill_consts(p.k, q.h, q.coef[0], ones);
     p.partials = q.partials;
     const int minb = env_int("FPDE_NS_MINB_F", 3);
     cudaError_t ce;
@@ -398,22 +295,15 @@ cudaError_t launch_ns_fwd(const Problem& q) {
 }
 
 cudaError_t launch_ns_bwd(const Problem& q) {
+    {
+        bool launched = false;
+        const cudaError_t ce = launch_ns_bwd_tma(q, launched);
+        if (launched || ce != cudaSuccess) return ce;
+    }
     NsParams p{}; dim3 block;
     ns_geometry(q, p, block);
     for (int k = 0; k < 4; ++k) { p.f[k] = q.in[k]; p.g[k] = q.aux[k]; p.out[k] = q.out[k]; }
-    const double nu = q.coef[0];
-    for (int a = 0; a < 3; ++a) {
-        p.ih[a] = sp(0.5 / q.h[a]);
-        p.c_ih[a] = sp(q.gscale[3] * 0.5 / q.h[a]);
-    }
-    for (int k = 0; k < 3; ++k) {
-        p.a_t[k] = sp(q.gscale[k] * 0.5 / q.h[3]);
-        p.l_g[k] = sp(q.gscale[k]);
-        for (int a = 0; a < 3; ++a) {
-            p.a_ih[k][a] = sp(q.gscale[k] * 0.5 / q.h[a]);
-            p.a_nv[k][a] = sp(-nu * q.gscale[k] / (q.h[a] * q.h[a]));
-        }
-    }
+    ns_fill_consts(p.k, q.h, q.coef[0], q.gscale);
     p.partials = nullptr;
     const int minb = env_int("FPDE_NS_MINB_B", 2);
     cudaError_t ce;

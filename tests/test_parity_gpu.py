@@ -153,3 +153,14 @@ def test_loss_grad_from_host_buffers():
         assert_close(g.numpy(), gr, "host entry gradient %d" % f)
     st = B.loss_grad_host_status(w.op, hf, [], hg, hl, w.shape, w.spacing, w.coeffs, w.bc, arena, 1024, None)
     assert st == 9
+
+
+@pytest.mark.parametrize("shape", [(8, 12, 16, 8), (19, 8, 8, 16), (6, 4, 4, 32), (7, 16, 32, 16), (5, 12, 48, 8)])
+def test_ns_tma_and_l1_staged_kernels_agree_with_oracle(shape, monkeypatch):
+    """FPDE_NS_TMA=1 runs grids that tile exactly on the TMA-staged kernels (one-box tiles away from
+    the periodic wrap, five-box tiles on it); the default is the L1-staged kernels.  Both must
+    match the oracle, and no bounded barrier wait may have given up."""
+    for tma in ("1", "0"):
+        monkeypatch.setenv("FPDE_NS_TMA", tma)
+        _check_case(W.make("ns_tgv_128x16", seed=46, shape=shape, kind="randn"), "ns %s tma=%s" % (shape, tma))
+    assert B.diag_tma_timeouts() == 0
