@@ -39,14 +39,12 @@ __device__ __forceinline__ void prefetch_l2_line(const float* ptr) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
 }
 
-template <bool FWD>
-__global__ void __launch_bounds__(256, 4) star3d_kernel(const Star3dParams p) {
-    pdl_wait_then_trigger();
+// EDGE: the block touches the two-cell band in x or y, where (adjoint) rows and planes of the
+// upstream array read as zero; blocks away from the band run without those selects.  The first
+// and last float4 of a row (the band in z) are handled in every block.
+template <bool FWD, bool EDGE, int MINB>
+__device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int mb, int ab) {
     const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
-    int item = blockIdx.x;
-    const int cb = item % p.ncb; item /= p.ncb;
-    const int mb = item % p.nmb;
-    const int ab = item / p.nmb;
     const int c4 = cb * blockDim.x + threadIdx.x;
     const int m = mb * blockDim.y + threadIdx.y;
     const int lane = threadIdx.x & 31;
@@ -57,51 +55,55 @@ __global__ void __launch_bounds__(256, 4) star3d_kernel(const Star3dParams p) {
     const int a0 = ab * p.planes_per_item;
     const int a1 = min(a0 + p.planes_per_item, n0);
     const int PS = n1 * n2;
-    constexpr bool MASK_IN = !FWD;
+    constexpr bool MASK_IN = !FWD;                  // the adjoint zero-extends its input outside the rows
+    constexpr bool ROWMASK = MASK_IN && EDGE;
     const float* __restrict__ hin = p.hin;
 
-    // Rows / planes outside the grid are clamped (forward: they only feed masked outputs).  In
-    // the adjoint a row or plane outside the rows of the operator reads as zero: the load is
-    // still issued at the clamped address and the value is then discarded by a select, which
-    // keeps the loads of a step independent of each other (no branches between them).
-    auto yclamp = [&](int d) -> int { return max(0, min(n1 - 1, mc + d)); };
-    auto ydead = [&](int d) -> bool { const int r = mc + d; return MASK_IN && (r < 2 || r > n1 - 3); };
-    const int ym1 = yclamp(-1), yp1 = yclamp(1), ym2 = yclamp(-2), yp2 = yclamp(2), y0 = mc;
-    const bool dm1 = ydead(-1), dp1 = ydead(1), dm2 = ydead(-2), dp2 = ydead(2), d0 = ydead(0);
-    auto load_h = [&](int a, int r, bool rdead) -> V4 {
-        const int pa = max(0, min(n0 - 1, a));
-        V4 v = ldv4(hin + pa * PS + r * n2 + col);
+    // element offsets of the own row and of the four y neighbours (clamped into the grid: out of
+    // range rows only feed outputs that are masked, or are discarded by the selects below)
+    auto yoff = [&](int d) -> int { return max(0, min(n1 - 1, mc + d)) * n2 + col; };
+    auto ydead = [&](int d) -> bool { const int r = mc + d; return ROWMASK && (r < 2 || r > n1 - 3); };
+    const int o_c = yoff(0), o_m1 = yoff(-1), o_p1 = yoff(1), o_m2 = yoff(-2), o_p2 = yoff(2);
+    const bool d0 = ydead(0), dm1 = ydead(-1), dp1 = ydead(1), dm2 = ydead(-2), dp2 = ydead(2);
+    // load from plane offset `pl` (already clamped) + row offset; `dead` = reads as zero
+    auto load_h = [&](int pl, int off, bool dead) -> V4 {
+        V4 v = ldv4(hin + pl + off);
         if (MASK_IN) {
-            const bool dead = rdead || a < 2 || a > n0 - 3;
-            if (dead || first_col) v.lo = make_float2(0.f, 0.f);
-            if (dead || last_col) v.hi = make_float2(0.f, 0.f);
+            if ((ROWMASK && dead) || first_col) v.lo = make_float2(0.f, 0.f);
+            if ((ROWMASK && dead) || last_col) v.hi = make_float2(0.f, 0.f);
         }
         return v;
     };
+    auto pclamp = [&](int a) -> int { return EDGE ? max(0, min(n0 - 1, a)) * PS : a * PS; };
+    auto pdead = [&](int a) -> bool { return ROWMASK && (a < 2 || a > n0 - 3); };
     const bool lfetch = lane == 0 && c4 > 0 && c4 < nc4;
     const bool rfetch = lane == 31 && c4 < nc4 - 1;
 
-    V4 Q0 = load_h(a0 - 2, y0, d0), Q1 = load_h(a0 - 1, y0, d0), Q2 = load_h(a0, y0, d0), Q3 = load_h(a0 + 1, y0, d0), Q4;
+    V4 Q0 = load_h(pclamp(a0 - 2), o_c, d0 || pdead(a0 - 2)), Q1 = load_h(pclamp(a0 - 1), o_c, d0 || pdead(a0 - 1));
+    V4 Q2 = load_h(pclamp(a0), o_c, d0 || pdead(a0)), Q3 = load_h(pclamp(a0 + 1), o_c, d0 || pdead(a0 + 1)), Q4;
     float2 acc = make_float2(0.f, 0.f);
 
     // one x step: q0..q3 = planes a-2..a+1, q4 receives plane a+2
     auto step = [&](int a, const V4& q0, const V4& q1, const V4& q2, const V4& q3, V4& q4) {
+        const int pl = a * PS;
         if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 2 + p.prefetch <= a1 + 1 && a + 2 + p.prefetch < n0) {
-            prefetch_l2_line(hin + (a + 2 + p.prefetch) * PS + mc * n2 + col);
-            if (FWD) prefetch_l2_line(p.cin + min(a + p.prefetch, n0 - 1) * PS + mc * n2 + col);
+            prefetch_l2_line(hin + pl + (2 + p.prefetch) * PS + o_c);
+            if (FWD) prefetch_l2_line(p.cin + pl + p.prefetch * PS + o_c);
         }
-        q4 = load_h(a + 2, y0, d0);
-        const V4 a1v = load_h(a, ym1, dm1), b1v = load_h(a, yp1, dp1), a2v = load_h(a, ym2, dm2), b2v = load_h(a, yp2, dp2);
+        const bool pd = pdead(a);
+        q4 = load_h(pclamp(a + 2), o_c, d0 || pdead(a + 2));
+        const V4 a1v = load_h(pl, o_m1, dm1 || pd), b1v = load_h(pl, o_p1, dp1 || pd);
+        const V4 a2v = load_h(pl, o_m2, dm2 || pd), b2v = load_h(pl, o_p2, dp2 || pd);
         V4 src = v4zero();
-        if (FWD) src = ldv4(p.cin + a * PS + mc * n2 + col);
+        if (FWD) src = ldv4(p.cin + pl + o_c);
         // z neighbours from the adjacent lanes; the outer lanes of a warp fetch theirs
         float l1 = __shfl_up_sync(FULL_MASK, q2.hi.y, 1), l2 = __shfl_up_sync(FULL_MASK, q2.hi.x, 1);
         float r1 = __shfl_down_sync(FULL_MASK, q2.lo.x, 1), r2 = __shfl_down_sync(FULL_MASK, q2.lo.y, 1);
         {
-            const float* rp = hin + a * PS + y0 * n2 + col;      // a is a valid plane here
+            const float* rp = hin + pl + o_c;
             if (lfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp - 2)); l2 = t.x; l1 = t.y; }
             if (rfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp + 4)); r1 = t.x; r2 = t.y; }
-            const bool dead = MASK_IN && (d0 || a < 2 || a > n0 - 3);
+            const bool dead = ROWMASK && (d0 || pd);
             if (dead || first_col) { l1 = 0.f; l2 = 0.f; }
             if (dead || last_col) { r1 = 0.f; r2 = 0.f; }
         }
@@ -119,12 +121,12 @@ __global__ void __launch_bounds__(256, 4) star3d_kernel(const Star3dParams p) {
         if (FWD) {
             o = v4sub(o, src);
             // nodes of the two outer layers carry no row
-            if (a < 2 || a > n0 - 3 || m < 2 || m > n1 - 3) { o = v4zero(); }
+            if (EDGE && (a < 2 || a > n0 - 3 || m < 2 || m > n1 - 3)) { o = v4zero(); }
             if (first_col) o.lo = make_float2(0.f, 0.f);
             if (last_col) o.hi = make_float2(0.f, 0.f);
         }
         if (valid) {
-            stv4(p.out + a * PS + mc * n2 + col, o.lo, o.hi);
+            stv4(p.out + pl + o_c, o.lo, o.hi);
             if (FWD) acc = fma2(o.lo, o.lo, fma2(o.hi, o.hi, acc));
         }
     };
@@ -140,6 +142,20 @@ __global__ void __launch_bounds__(256, 4) star3d_kernel(const Star3dParams p) {
         float s[1] = {acc.x + acc.y};
         block_reduce_store<1>(s, p.partials, p.nitems, blockIdx.x);
     }
+}
+
+template <bool FWD, int MINB>
+__global__ void __launch_bounds__(256, MINB) star3d_kernel(const Star3dParams p) {
+    pdl_wait_then_trigger();
+    int item = blockIdx.x;
+    const int cb = item % p.ncb; item /= p.ncb;
+    const int mb = item % p.nmb;
+    const int ab = item / p.nmb;
+    const int m0 = mb * blockDim.y, a0 = ab * p.planes_per_item;
+    // away from the band: every row m0-2 .. m0+TY+1 and plane a0-2 .. a1+1 is a row of the operator
+    const bool interior = m0 >= 4 && m0 + (int)blockDim.y + 4 <= p.n1 && a0 >= 4 && a0 + p.planes_per_item + 4 <= p.n0;
+    if (interior) star3d_body<FWD, false, MINB>(p, cb, mb, ab);
+    else star3d_body<FWD, true, MINB>(p, cb, mb, ab);
 }
 
 static int env_int(const char* name, int dflt) {
@@ -188,7 +204,8 @@ cudaError_t launch_helmholtz_fwd(const Problem& q) {
     star3d_geometry(q, p, block, 1.0);
     p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0];
     p.partials = q.partials;
-    return launch_kernel(star3d_kernel<true>, dim3(p.nitems), block, q.stream, p);
+    if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<true, 4>, dim3(p.nitems), block, q.stream, p);
+    return launch_kernel(star3d_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
 }
 
 cudaError_t launch_helmholtz_bwd(const Problem& q) {
@@ -196,7 +213,8 @@ cudaError_t launch_helmholtz_bwd(const Problem& q) {
     star3d_geometry(q, p, block, q.gscale[0]);      // the operator is linear: the scale goes into the weights
     p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0];
     p.partials = nullptr;
-    return launch_kernel(star3d_kernel<false>, dim3(p.nitems), block, q.stream, p);
+    if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<false, 4>, dim3(p.nitems), block, q.stream, p);
+    return launch_kernel(star3d_kernel<false, 3>, dim3(p.nitems), block, q.stream, p);
 }
 
 }  // namespace fpde
