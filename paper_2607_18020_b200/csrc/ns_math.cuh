@@ -40,47 +40,109 @@ struct NsConsts {
     float2 c_ih[3];       // [a]     gs_c / (2 h_a)
 };
 
-// W0/W1/W2: planes x-1, x, x+1 at the own column; Ym/Yp/Zm/Zp: y-+1 and z-+1 neighbours of plane x;
-// arrays u,v,w,p.  l1/r1: t-1 of lane x and t+1 of lane w for u,v,w.  o[e][half].
+// ---- one packed pair (two consecutive t of one z) of every array -----------------------------
+// w0/w1/w2: planes x-1, x, x+1 at the own column; ym/yp/zm/zp: y-+1 and z-+1 neighbours of plane x.
+// Forward: arrays u,v,w,p; dt[q] = q(t+1) - q(t-1) for the pair.  o[e]: mom_x, mom_y, mom_z, continuity.
+__device__ __forceinline__ void ns_fwd_pair(const NsConsts& k, const float2 (&w0)[4], const float2 (&w1)[4],
+                                            const float2 (&w2)[4], const float2 (&ym)[4], const float2 (&yp)[4],
+                                            const float2 (&zm)[4], const float2 (&zp)[4], const float2 (&dt)[3],
+                                            float2 (&o)[4]) {
+    const float2 us = mul2(w1[0], k.ih[0]);     // advecting velocities, pre-scaled by 1/(2h)
+    const float2 vs = mul2(w1[1], k.ih[1]);
+    const float2 ws = mul2(w1[2], k.ih[2]);
+    float2 dself[3];                            // d_x u, d_y v, d_z w (raw differences)
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        const float2 c = w1[q];
+        const float2 xm = sub2(w0[q], c), xp = sub2(w2[q], c);
+        const float2 ymd = sub2(ym[q], c), ypd = sub2(yp[q], c);
+        const float2 zmd = sub2(zm[q], c), zpd = sub2(zp[q], c);
+        const float2 dx = sub2(xp, xm), dy = sub2(ypd, ymd), dz = sub2(zpd, zmd);
+        float2 r = mul2(add2(xm, xp), k.nv[0]);
+        r = fma2(add2(ymd, ypd), k.nv[1], r);
+        r = fma2(add2(zmd, zpd), k.nv[2], r);
+        r = fma2(us, dx, r);
+        r = fma2(vs, dy, r);
+        r = fma2(ws, dz, r);
+        r = fma2(dt[q], k.iht, r);
+        dself[q] = q == 0 ? dx : (q == 1 ? dy : dz);
+        o[q] = r;
+    }
+    o[0] = fma2(sub2(w2[3], w0[3]), k.ih[0], o[0]);     // d_x p
+    o[1] = fma2(sub2(yp[3], ym[3]), k.ih[1], o[1]);     // d_y p
+    o[2] = fma2(sub2(zp[3], zm[3]), k.ih[2], o[2]);     // d_z p
+    o[3] = fma2(dself[2], k.ih[2], fma2(dself[1], k.ih[1], mul2(dself[0], k.ih[0])));
+}
+
+// Adjoint: arrays 0..2 = u,v,w ; 3..6 = upstream of mom_x, mom_y, mom_z, continuity;
+// dt[q] = G_q(t-1) - G_q(t+1) for the pair (end planes already counted as zero).  o[f]: g_u, g_v, g_w, g_p.
+__device__ __forceinline__ void ns_bwd_pair(const NsConsts& k, const float2 (&w0)[7], const float2 (&w1)[7],
+                                            const float2 (&w2)[7], const float2 (&ym)[7], const float2 (&yp)[7],
+                                            const float2 (&zm)[7], const float2 (&zp)[7], const float2 (&dt)[3],
+                                            float2 (&o)[4]) {
+    // neighbours of array i along axis a: minus / plus
+    auto NM = [&](int i, int a_) -> float2 { return a_ == 0 ? w0[i] : (a_ == 1 ? ym[i] : zm[i]); };
+    auto NP = [&](int i, int a_) -> float2 { return a_ == 0 ? w2[i] : (a_ == 1 ? yp[i] : zp[i]); };
+    float2 gs[3];                               // scaled centre sensitivities
+#pragma unroll
+    for (int e = 0; e < 3; ++e) gs[e] = mul2(w1[3 + e], k.l_g[e]);
+    float2 cm[3], ncp[3];                       // advecting velocity at P-a, minus the one at P+a
+#pragma unroll
+    for (int a_ = 0; a_ < 3; ++a_) {
+        cm[a_] = NM(a_, a_);
+        const float2 cp = NP(a_, a_);
+        ncp[a_] = make_float2(-cp.x, -cp.y);
+    }
+    float2 gp = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        const float2 c = w1[3 + q];
+        float2 r = mul2(dt[q], k.a_t[q]);
+#pragma unroll
+        for (int a_ = 0; a_ < 3; ++a_) {
+            const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
+            const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
+            r = fma2(adv, k.a_ih[q][a_], r);
+            const float2 dm = sub2(gm, c), dp = sub2(gpl, c);
+            r = fma2(add2(dm, dp), k.a_nv[q][a_], r);
+            if (a_ == q) gp = fma2(sub2(dm, dp), k.a_ih[q][q], gp);
+        }
+        // local terms and continuity row along this component's own axis
+        float2 loc = mul2(gs[0], sub2(NP(0, q), NM(0, q)));
+        loc = fma2(gs[1], sub2(NP(1, q), NM(1, q)), loc);
+        loc = fma2(gs[2], sub2(NP(2, q), NM(2, q)), loc);
+        r = fma2(loc, k.ih[q], r);
+        r = fma2(sub2(NM(6, q), NP(6, q)), k.c_ih[q], r);
+        o[q] = r;
+    }
+    o[3] = gp;
+}
+
+// ---- a float4 (four consecutive t) per thread: two pairs -------------------------------------
+// l1/r1: t-1 of lane x and t+1 of lane w for u,v,w (forward) / the momentum upstream arrays.
+template <int NA>
+__device__ __forceinline__ void v4_half(const V4 (&A)[NA], int h, float2 (&out)[NA]) {
+#pragma unroll
+    for (int i = 0; i < NA; ++i) out[i] = h == 0 ? A[i].lo : A[i].hi;
+}
+
 __device__ __forceinline__ void ns_fwd_math(const NsConsts& k, const V4 (&W0)[4], const V4 (&W1)[4], const V4 (&W2)[4],
                                             const V4 (&Ym)[4], const V4 (&Yp)[4], const V4 (&Zm)[4], const V4 (&Zp)[4],
                                             const float (&l1)[3], const float (&r1)[3], bool t_first, bool t_last,
                                             float2 (&o)[4][2]) {
-    float2 dtl[3], dth[3];                      // q(t+1) - q(t-1), lanes (x,y) and (z,w)
 #pragma unroll
-    for (int q = 0; q < 3; ++q) {
-        const V4 c = W1[q];
-        dtl[q] = make_float2(c.lo.y - l1[q], c.hi.x - c.lo.x);
-        dth[q] = make_float2(c.hi.y - c.lo.y, r1[q] - c.hi.x);
-    }
+    for (int h = 0; h < 2; ++h) {
+        float2 w0[4], w1[4], w2[4], ym[4], yp[4], zm[4], zp[4], dt[3], oo[4];
+        v4_half<4>(W0, h, w0); v4_half<4>(W1, h, w1); v4_half<4>(W2, h, w2);
+        v4_half<4>(Ym, h, ym); v4_half<4>(Yp, h, yp); v4_half<4>(Zm, h, zm); v4_half<4>(Zp, h, zp);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {               // the two packed halves of the float4
-        auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
-        const float2 us = mul2(H(W1[0]), k.ih[0]);   // advecting velocities, pre-scaled by 1/(2h)
-        const float2 vs = mul2(H(W1[1]), k.ih[1]);
-        const float2 ws = mul2(H(W1[2]), k.ih[2]);
-        float2 dself[3];                        // d_x u, d_y v, d_z w (raw differences)
-#pragma unroll
-        for (int q = 0; q < 3; ++q) {
-            const float2 c = H(W1[q]);
-            const float2 xm = sub2(H(W0[q]), c), xp = sub2(H(W2[q]), c);
-            const float2 ym = sub2(H(Ym[q]), c), yp = sub2(H(Yp[q]), c);
-            const float2 zm = sub2(H(Zm[q]), c), zp = sub2(H(Zp[q]), c);
-            const float2 dx = sub2(xp, xm), dy = sub2(yp, ym), dz = sub2(zp, zm);
-            float2 r = mul2(add2(xm, xp), k.nv[0]);
-            r = fma2(add2(ym, yp), k.nv[1], r);
-            r = fma2(add2(zm, zp), k.nv[2], r);
-            r = fma2(us, dx, r);
-            r = fma2(vs, dy, r);
-            r = fma2(ws, dz, r);
-            r = fma2(h == 0 ? dtl[q] : dth[q], k.iht, r);
-            dself[q] = q == 0 ? dx : (q == 1 ? dy : dz);
-            o[q][h] = r;
+        for (int q = 0; q < 3; ++q) {           // q(t+1) - q(t-1)
+            const V4 c = W1[q];
+            dt[q] = h == 0 ? make_float2(c.lo.y - l1[q], c.hi.x - c.lo.x) : make_float2(c.hi.y - c.lo.y, r1[q] - c.hi.x);
         }
-        o[0][h] = fma2(sub2(H(W2[3]), H(W0[3])), k.ih[0], o[0][h]);     // d_x p
-        o[1][h] = fma2(sub2(H(Yp[3]), H(Ym[3])), k.ih[1], o[1][h]);     // d_y p
-        o[2][h] = fma2(sub2(H(Zp[3]), H(Zm[3])), k.ih[2], o[2][h]);     // d_z p
-        o[3][h] = fma2(dself[2], k.ih[2], fma2(dself[1], k.ih[1], mul2(dself[0], k.ih[0])));
+        ns_fwd_pair(k, w0, w1, w2, ym, yp, zm, zp, dt, oo);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e][h] = oo[e];
     }
 #pragma unroll
     for (int e = 0; e < 4; ++e) {               // t = 0 and t = n3-1 carry no row
@@ -89,60 +151,25 @@ __device__ __forceinline__ void ns_fwd_math(const NsConsts& k, const V4 (&W0)[4]
     }
 }
 
-// Arrays 0..2: u,v,w ; 3..6: upstream of mom_x, mom_y, mom_z, continuity.  l1/r1: t-1 of lane x
-// and t+1 of lane w of the three momentum upstream arrays.
 __device__ __forceinline__ void ns_bwd_math(const NsConsts& k, const V4 (&W0)[7], const V4 (&W1)[7], const V4 (&W2)[7],
                                             const V4 (&Ym)[7], const V4 (&Yp)[7], const V4 (&Zm)[7], const V4 (&Zp)[7],
                                             const float (&l1)[3], const float (&r1)[3], bool t_first, bool t_last,
                                             float2 (&o)[4][2]) {
-    float2 dtl[3], dth[3];                      // G_q(t-1) - G_q(t+1) with the end planes counted as 0
-#pragma unroll
-    for (int q = 0; q < 3; ++q) {
-        const V4 c = W1[3 + q];
-        const float tm_y = t_first ? 0.f : c.lo.x;       // t-1 of lane y is the end plane t = 0
-        const float tp_z = t_last ? 0.f : c.hi.y;        // t+1 of lane z is the end plane t = n3-1
-        dtl[q] = make_float2(l1[q] - c.lo.y, tm_y - c.hi.x);
-        dth[q] = make_float2(c.lo.y - tp_z, c.hi.x - r1[q]);
-    }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        auto H = [&](const V4& v) -> float2 { return h == 0 ? v.lo : v.hi; };
-        // neighbours of array i along axis a: minus / plus
-        auto NM = [&](int i, int a_) -> float2 { return a_ == 0 ? H(W0[i]) : (a_ == 1 ? H(Ym[i]) : H(Zm[i])); };
-        auto NP = [&](int i, int a_) -> float2 { return a_ == 0 ? H(W2[i]) : (a_ == 1 ? H(Yp[i]) : H(Zp[i])); };
-        float2 gs[3];                            // scaled centre sensitivities
+        float2 w0[7], w1[7], w2[7], ym[7], yp[7], zm[7], zp[7], dt[3], oo[4];
+        v4_half<7>(W0, h, w0); v4_half<7>(W1, h, w1); v4_half<7>(W2, h, w2);
+        v4_half<7>(Ym, h, ym); v4_half<7>(Yp, h, yp); v4_half<7>(Zm, h, zm); v4_half<7>(Zp, h, zp);
 #pragma unroll
-        for (int e = 0; e < 3; ++e) gs[e] = mul2(H(W1[3 + e]), k.l_g[e]);
-        float2 cm[3], ncp[3];                    // advecting velocity at P-a, minus the one at P+a
-#pragma unroll
-        for (int a_ = 0; a_ < 3; ++a_) {
-            cm[a_] = NM(a_, a_);
-            const float2 cp = NP(a_, a_);
-            ncp[a_] = make_float2(-cp.x, -cp.y);
+        for (int q = 0; q < 3; ++q) {           // G_q(t-1) - G_q(t+1), end planes counted as 0
+            const V4 c = W1[3 + q];
+            const float tm_y = t_first ? 0.f : c.lo.x;       // t-1 of lane y is the end plane t = 0
+            const float tp_z = t_last ? 0.f : c.hi.y;        // t+1 of lane z is the end plane t = n3-1
+            dt[q] = h == 0 ? make_float2(l1[q] - c.lo.y, tm_y - c.hi.x) : make_float2(c.lo.y - tp_z, c.hi.x - r1[q]);
         }
-        float2 gp = make_float2(0.f, 0.f);
+        ns_bwd_pair(k, w0, w1, w2, ym, yp, zm, zp, dt, oo);
 #pragma unroll
-        for (int q = 0; q < 3; ++q) {
-            const float2 c = H(W1[3 + q]);
-            float2 r = mul2(h == 0 ? dtl[q] : dth[q], k.a_t[q]);
-#pragma unroll
-            for (int a_ = 0; a_ < 3; ++a_) {
-                const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
-                const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
-                r = fma2(adv, k.a_ih[q][a_], r);
-                const float2 dm = sub2(gm, c), dp = sub2(gpl, c);
-                r = fma2(add2(dm, dp), k.a_nv[q][a_], r);
-                if (a_ == q) gp = fma2(sub2(dm, dp), k.a_ih[q][q], gp);
-            }
-            // local terms and continuity row along this component's own axis
-            float2 loc = mul2(gs[0], sub2(NP(0, q), NM(0, q)));
-            loc = fma2(gs[1], sub2(NP(1, q), NM(1, q)), loc);
-            loc = fma2(gs[2], sub2(NP(2, q), NM(2, q)), loc);
-            r = fma2(loc, k.ih[q], r);
-            r = fma2(sub2(NM(6, q), NP(6, q)), k.c_ih[q], r);
-            o[q][h] = r;
-        }
-        o[3][h] = gp;
+        for (int e = 0; e < 4; ++e) o[e][h] = oo[e];
     }
     // end planes of t: only the transposed d_t term exists there, and no pressure gradient
 #pragma unroll
