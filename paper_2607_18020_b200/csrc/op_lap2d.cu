@@ -231,7 +231,7 @@ static void lap2d_geometry(const Problem& q, Lap2dParams& p, int& block) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.nc4 = q.n[1] / 4;
     block = env_int("FPDE_LAP2D_BLOCK", 128);
     block = std::max(32, std::min(128, (block / 32) * 32));
-    p.rows_per_item = env_int("FPDE_LAP2D_ROWS", 16);
+    p.rows_per_item = env_int("FPDE_LAP2D_ROWS", 8);
     p.ncb = (p.nc4 + block - 1) / block;
     p.nitems = p.ncb * ((p.n0 + p.rows_per_item - 1) / p.rows_per_item);
     const float ih0 = (float)(1.0 / (q.h[0] * q.h[0])), ih1 = (float)(1.0 / (q.h[1] * q.h[1]));
