@@ -62,15 +62,25 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     // element offsets of the own row and of the four y neighbours (clamped into the grid: out of
     // range rows only feed outputs that are masked, or are discarded by the selects below)
     auto yoff = [&](int d) -> int { return max(0, min(n1 - 1, mc + d)) * n2 + col; };
+    auto yptr = [&](int d) -> const float* { return hin + yoff(d); };
     auto ydead = [&](int d) -> bool { const int r = mc + d; return ROWMASK && (r < 2 || r > n1 - 3); };
-    const int o_c = yoff(0), o_m1 = yoff(-1), o_p1 = yoff(1), o_m2 = yoff(-2), o_p2 = yoff(2);
+    // one pointer per row: the plane offset of a step is then a single multiply-add per load
+    const int o_c = yoff(0);
+    const float* __restrict__ p_c = yptr(0);
+    const float* __restrict__ p_m1 = yptr(-1);
+    const float* __restrict__ p_p1 = yptr(1);
+    const float* __restrict__ p_m2 = yptr(-2);
+    const float* __restrict__ p_p2 = yptr(2);
     const bool d0 = ydead(0), dm1 = ydead(-1), dp1 = ydead(1), dm2 = ydead(-2), dp2 = ydead(2);
-    // load from plane offset `pl` (already clamped) + row offset; `dead` = reads as zero
-    auto load_h = [&](int pl, int off, bool dead) -> V4 {
-        V4 v = ldv4(hin + pl + off);
+    // Load from a row pointer at plane offset `pl` (already clamped); `dead` = reads as zero.
+    // OWN: the thread's own column (the x window).  Only that one is masked in the first / last
+    // float4 of a row (the band in z); the y neighbours are not, their contribution to the two
+    // band columns is removed after the sums instead (see the step).
+    auto load_h = [&](const float* rp, int pl, bool dead, bool own) -> V4 {
+        V4 v = ldv4(rp + pl);
         if (MASK_IN) {
-            if ((ROWMASK && dead) || first_col) v.lo = make_float2(0.f, 0.f);
-            if ((ROWMASK && dead) || last_col) v.hi = make_float2(0.f, 0.f);
+            if ((ROWMASK && dead) || (own && first_col)) v.lo = make_float2(0.f, 0.f);
+            if ((ROWMASK && dead) || (own && last_col)) v.hi = make_float2(0.f, 0.f);
         }
         return v;
     };
@@ -79,28 +89,28 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     const bool lfetch = lane == 0 && c4 > 0 && c4 < nc4;
     const bool rfetch = lane == 31 && c4 < nc4 - 1;
 
-    V4 Q0 = load_h(pclamp(a0 - 2), o_c, d0 || pdead(a0 - 2)), Q1 = load_h(pclamp(a0 - 1), o_c, d0 || pdead(a0 - 1));
-    V4 Q2 = load_h(pclamp(a0), o_c, d0 || pdead(a0)), Q3 = load_h(pclamp(a0 + 1), o_c, d0 || pdead(a0 + 1)), Q4;
+    V4 Q0 = load_h(p_c, pclamp(a0 - 2), d0 || pdead(a0 - 2), true), Q1 = load_h(p_c, pclamp(a0 - 1), d0 || pdead(a0 - 1), true);
+    V4 Q2 = load_h(p_c, pclamp(a0), d0 || pdead(a0), true), Q3 = load_h(p_c, pclamp(a0 + 1), d0 || pdead(a0 + 1), true), Q4;
     float2 acc = make_float2(0.f, 0.f);
 
     // one x step: q0..q3 = planes a-2..a+1, q4 receives plane a+2
     auto step = [&](int a, const V4& q0, const V4& q1, const V4& q2, const V4& q3, V4& q4) {
         const int pl = a * PS;
         if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 2 + p.prefetch <= a1 + 1 && a + 2 + p.prefetch < n0) {
-            prefetch_l2_line(hin + pl + (2 + p.prefetch) * PS + o_c);
+            prefetch_l2_line(p_c + pl + (2 + p.prefetch) * PS);
             if (FWD) prefetch_l2_line(p.cin + pl + p.prefetch * PS + o_c);
         }
         const bool pd = pdead(a);
-        q4 = load_h(pclamp(a + 2), o_c, d0 || pdead(a + 2));
-        const V4 a1v = load_h(pl, o_m1, dm1 || pd), b1v = load_h(pl, o_p1, dp1 || pd);
-        const V4 a2v = load_h(pl, o_m2, dm2 || pd), b2v = load_h(pl, o_p2, dp2 || pd);
+        q4 = load_h(p_c, pclamp(a + 2), d0 || pdead(a + 2), true);
+        const V4 a1v = load_h(p_m1, pl, dm1 || pd, false), b1v = load_h(p_p1, pl, dp1 || pd, false);
+        const V4 a2v = load_h(p_m2, pl, dm2 || pd, false), b2v = load_h(p_p2, pl, dp2 || pd, false);
         V4 src = v4zero();
         if (FWD) src = ldv4(p.cin + pl + o_c);
         // z neighbours from the adjacent lanes; the outer lanes of a warp fetch theirs
         float l1 = __shfl_up_sync(FULL_MASK, q2.hi.y, 1), l2 = __shfl_up_sync(FULL_MASK, q2.hi.x, 1);
         float r1 = __shfl_down_sync(FULL_MASK, q2.lo.x, 1), r2 = __shfl_down_sync(FULL_MASK, q2.lo.y, 1);
         {
-            const float* rp = hin + pl + o_c;
+            const float* rp = p_c + pl;
             if (lfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp - 2)); l2 = t.x; l1 = t.y; }
             if (rfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp + 4)); r1 = t.x; r2 = t.y; }
             const bool dead = ROWMASK && (d0 || pd);
@@ -116,8 +126,16 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
         s2z.hi = make_float2(q2.lo.x + r1, q2.lo.y + r2);
         V4 o = v4mul(q2, p.kc);
         o = v4fma(s1x, p.w16[0], o); o = v4fma(s2x, p.nw[0], o);
-        o = v4fma(s1y, p.w16[1], o); o = v4fma(s2y, p.nw[1], o);
         o = v4fma(s1z, p.w16[2], o); o = v4fma(s2z, p.nw[2], o);
+        const V4 oxz = o;                            // centre + x + z terms
+        o = v4fma(s1y, p.w16[1], o); o = v4fma(s2y, p.nw[1], o);
+        if (MASK_IN) {
+            // band in z (adjoint): columns 0,1 / n-2,n-1 of the upstream array are zero.  The own
+            // column was masked on load, so oxz is already right there; only the (unmasked) y
+            // neighbours have to be taken out again.
+            if (first_col) o.lo = oxz.lo;
+            if (last_col) o.hi = oxz.hi;
+        }
         if (FWD) {
             o = v4sub(o, src);
             // nodes of the two outer layers carry no row
@@ -172,7 +190,7 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     int tx = p.nc4 > 32 ? 64 : 32;
     tx = env_int("FPDE_STAR3D_TX", tx);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
-    int ty = env_int("FPDE_STAR3D_TY", 4);
+    int ty = env_int("FPDE_STAR3D_TY", 2);
     ty = std::max(1, std::min(256 / tx, ty));
     block = dim3(tx, ty, 1);
     p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 16);
