@@ -1,0 +1,84 @@
+"""`torch.autograd.Function` wrappers over the C ABI: the drop-in form of the operators
+(Section 2 of the paper exposes each operator through `torch.autograd.Function`).
+
+    residuals = fused_residual(op, fields, sources, spacing, coeffs, bc)      # tuple of tensors
+    loss      = fused_residual_loss(op, fields, sources, spacing, coeffs, bc) # 0-dim fp64 tensor
+
+`fused_residual` runs `fpde_fwd` (no loss) in the forward pass and `fpde_bwd` on the upstream
+sensitivities autograd hands back.  `fused_residual_loss` also fuses the mean-square loss: the
+forward pass is `fpde_fwd` with the loss, the backward pass is `fpde_bwd` on the residual
+arrays with scale 2/N_r, times the incoming scalar gradient.  Everything runs in the library's
+kernels on the current CUDA stream; torch allocates the outputs and nothing else.
+"""
+from __future__ import annotations
+
+from typing import Sequence
+
+import torch
+
+from . import binding as B
+
+
+def _check(fields, sources):
+    for t in list(fields) + list(sources):
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise ValueError("fields and sources must be contiguous fp32 CUDA tensors")
+
+
+class _FusedResidual(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, op, sources, spacing, coeffs, bc, *fields):
+        _check(fields, sources)
+        shape = tuple(fields[0].shape)
+        ne = B.op_info(op).nresiduals
+        res = [torch.empty(shape, dtype=torch.float32, device=fields[0].device) for _ in range(ne)]
+        B.fpde_fwd(op, fields, sources, res, None, shape, spacing, coeffs, bc, None)
+        ctx.op, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc = op, shape, spacing, coeffs, bc
+        ctx.save_for_backward(*fields)
+        return tuple(res)
+
+    @staticmethod
+    def backward(ctx, *gres):
+        fields = ctx.saved_tensors
+        g = [x.contiguous() if x is not None else torch.zeros(ctx.shape, dtype=torch.float32, device=fields[0].device)
+             for x in gres]
+        out = [torch.empty(ctx.shape, dtype=torch.float32, device=fields[0].device) for _ in fields]
+        B.fpde_bwd(ctx.op, fields, g, None, out, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc)
+        return (None, None, None, None, None) + tuple(out)
+
+
+class _FusedResidualLoss(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, op, sources, spacing, coeffs, bc, *fields):
+        _check(fields, sources)
+        shape = tuple(fields[0].shape)
+        dev = fields[0].device
+        ne = B.op_info(op).nresiduals
+        res = [torch.empty(shape, dtype=torch.float32, device=dev) for _ in range(ne)]
+        loss = torch.empty(ne + 1, dtype=torch.float64, device=dev)
+        ws = torch.empty(B.workspace_bytes(op, shape), dtype=torch.uint8, device=dev)
+        B.fpde_fwd(op, fields, sources, res, loss, shape, spacing, coeffs, bc, ws)
+        ctx.op, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc, ctx.ne = op, shape, spacing, coeffs, bc, ne
+        ctx.save_for_backward(*fields, *res)
+        return loss[ne]
+
+    @staticmethod
+    def backward(ctx, gloss):
+        saved = ctx.saved_tensors
+        nf = len(saved) - ctx.ne
+        fields, res = saved[:nf], saved[nf:]
+        out = [torch.empty(ctx.shape, dtype=torch.float32, device=fields[0].device) for _ in fields]
+        scale = 2.0 / B.row_count(ctx.op, ctx.shape)
+        B.fpde_bwd(ctx.op, fields, res, [scale] * ctx.ne, out, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc)
+        gl = gloss.to(torch.float32)
+        return (None, None, None, None, None) + tuple(o * gl for o in out)
+
+
+def fused_residual(op, fields: Sequence[torch.Tensor], sources: Sequence[torch.Tensor], spacing, coeffs, bc):
+    """All residual fields of operator `op` as differentiable tensors (zero at nodes without a row)."""
+    return _FusedResidual.apply(op, tuple(sources), tuple(spacing), tuple(coeffs), tuple(bc), *fields)
+
+
+def fused_residual_loss(op, fields: Sequence[torch.Tensor], sources: Sequence[torch.Tensor], spacing, coeffs, bc):
+    """Sum over residual fields of the mean-square residual (fp64, 0-dim), differentiable w.r.t. the fields."""
+    return _FusedResidualLoss.apply(op, tuple(sources), tuple(spacing), tuple(coeffs), tuple(bc), *fields)
