@@ -33,7 +33,7 @@
 typedef long long i64;
 
 enum { OP_BURGERS_1D_T = 0, OP_POISSON_2D = 1, OP_GRAYSCOTT_2D = 2, OP_HELMHOLTZ_3D_O4 = 3,
-       OP_NS_3D_T = 4, OP_COUNT = 5 };
+       OP_NS_3D_T = 4, OP_NS_2D_STEADY = 5, OP_COUNT = 6 };
 enum { BC_PERIODIC = 0, BC_INTERIOR = 1, BC_ONE_SIDED = 2 };
 
 /* A 1-D difference formula at one node: value = sum_k w[k] * q[idx[k]] along one axis. */
@@ -114,17 +114,18 @@ static void scatter(const stencil* s, double* line, i64 stride, double a) {
     for (k = 0; k < s->n; ++k) line[s->idx[k] * stride] += a * s->w[k];
 }
 
-static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4 };
-static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4 };
-static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0 };
-static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4 };
-static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1 };
+static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2 };
+static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3 };
+static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0 };
+static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3 };
+static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1 };
 static const int OP_BC[OP_COUNT][4] = {
     { BC_ONE_SIDED, BC_ONE_SIDED, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
     { BC_PERIODIC, BC_PERIODIC, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, BC_INTERIOR, 0 },
     { BC_PERIODIC, BC_PERIODIC, BC_PERIODIC, BC_INTERIOR },
+    { BC_INTERIOR, BC_INTERIOR, 0, 0 },
 };
 
 int fpde_oracle_info(int op, int* ndim, int* nf, int* ns, int* ne, int* nc) {
@@ -309,6 +310,54 @@ static i64 ns3dt(int mode, const double* const* fld, double* const* res, const d
     return rows;
 }
 
+/* Steady incompressible Navier-Stokes on an (x,y) array, exactly the paper's Section 2.1 system:
+ *   res_u = u u_x + v u_y + p_x - nu (u_xx + u_yy),  res_v = u v_x + v v_y + p_y - nu (v_xx + v_yy),
+ *   res_div = u_x + v_y,
+ * centred differences (Appendix A.2), rows at the nodes where they fit (interior points); the
+ * outer ring is data.  fld = {u,v,p}; res / G / grd index: 0 res_u, 1 res_v, 2 res_div. */
+static i64 ns2d(int mode, const double* const* fld, double* const* res, const double* const* G,
+                double* const* grd, const i64* n, const double* h, const double* c) {
+    i64 nx = n[0], ny = n[1], i, j, rows = 0;
+    double nu = c[0];
+    for (i = 0; i < nx; ++i) for (j = 0; j < ny; ++j) {
+        stencil s1x, s1y, s2x, s2y;
+        i64 p = i * ny + j;
+        double vel[2], dq[2][2], lap[2], dp[2];
+        int q;
+        if (!d1(BC_INTERIOR, i, nx, h[0], &s1x) || !d1(BC_INTERIOR, j, ny, h[1], &s1y)) continue;
+        d2(BC_INTERIOR, i, nx, h[0], &s2x); d2(BC_INTERIOR, j, ny, h[1], &s2y);
+        ++rows;
+        for (q = 0; q < 2; ++q) {
+            vel[q] = fld[q][p];
+            dq[q][0] = apply(&s1x, fld[q] + j, ny);          /* d_x q  */
+            dq[q][1] = apply(&s1y, fld[q] + i * ny, 1);      /* d_y q  */
+            lap[q] = apply(&s2x, fld[q] + j, ny) + apply(&s2y, fld[q] + i * ny, 1);
+        }
+        dp[0] = apply(&s1x, fld[2] + j, ny);
+        dp[1] = apply(&s1y, fld[2] + i * ny, 1);
+        if (mode == 0) {
+            for (q = 0; q < 2; ++q)
+                res[q][p] = vel[0] * dq[q][0] + vel[1] * dq[q][1] + dp[q] - nu * lap[q];
+            res[2][p] = dq[0][0] + dq[1][1];
+        } else {
+            for (q = 0; q < 2; ++q) {
+                double Gq = G[q][p];
+                grd[0][p] += Gq * dq[q][0];                                  /* factor u in u d_x q */
+                grd[1][p] += Gq * dq[q][1];                                  /* factor v in v d_y q */
+                scatter(&s1x, grd[q] + j, ny, Gq * vel[0]);                  /* u * d_x q           */
+                scatter(&s1y, grd[q] + i * ny, 1, Gq * vel[1]);              /* v * d_y q           */
+                scatter(&s2x, grd[q] + j, ny, -Gq * nu);                     /* -nu d_xx q          */
+                scatter(&s2y, grd[q] + i * ny, 1, -Gq * nu);                 /* -nu d_yy q          */
+            }
+            scatter(&s1x, grd[2] + j, ny, G[0][p]);                          /* p_x in res_u        */
+            scatter(&s1y, grd[2] + i * ny, 1, G[1][p]);                      /* p_y in res_v        */
+            scatter(&s1x, grd[0] + j, ny, G[2][p]);                          /* u_x in res_div      */
+            scatter(&s1y, grd[1] + i * ny, 1, G[2][p]);                      /* v_y in res_div      */
+        }
+    }
+    return rows;
+}
+
 static i64 total(int ndim, const i64* n) { i64 N = 1; int a; for (a = 0; a < ndim; ++a) N *= n[a]; return N; }
 
 static int check(int op, int ndim, const i64* n) {
@@ -338,6 +387,7 @@ i64 fpde_oracle_fwd(int op, const double* const* fields, const double* const* so
     case OP_GRAYSCOTT_2D: rows = grayscott(0, fields[0], fields[1], residuals[0], residuals[1], NULL, NULL, NULL, NULL, shape, spacing, coeffs); break;
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(0, fields[0], sources[0], residuals[0], NULL, NULL, shape, spacing, coeffs); break;
     case OP_NS_3D_T: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
+    case OP_NS_2D_STEADY: rows = ns2d(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
     }
     if (loss) {
         loss[E] = 0.0;
@@ -366,6 +416,7 @@ i64 fpde_oracle_bwd(int op, const double* const* fields, const double* const* G,
     case OP_GRAYSCOTT_2D: rows = grayscott(1, fields[0], fields[1], NULL, NULL, G[0], G[1], gfields[0], gfields[1], shape, spacing, coeffs); break;
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(1, fields[0], NULL, NULL, G[0], gfields[0], shape, spacing, coeffs); break;
     case OP_NS_3D_T: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
+    case OP_NS_2D_STEADY: rows = ns2d(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
     }
     return rows;
 }

@@ -32,7 +32,8 @@ POISSON_2D = "poisson_2d"
 GRAYSCOTT_2D = "grayscott_2d"
 HELMHOLTZ_3D_O4 = "helmholtz_3d_o4"
 NS_3D_T = "ns_3d_t"
-OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T)
+NS_2D_STEADY = "ns_2d_steady"
+OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY)
 
 # Boundary kinds per array axis.
 PERIODIC = "periodic"      # rows at every node, wrap-around neighbours
@@ -114,6 +115,11 @@ CONFIGS: Dict[str, dict] = {
                           domain=((0.0, 2 * math.pi),) * 3 + ((0.0, 1.0),),
                           bc=(PERIODIC, PERIODIC, PERIODIC, INTERIOR)),
 }
+# beyond the five baseline configurations: the paper's own worked operator (steady 2-D
+# Navier-Stokes, its lid-driven-cavity case) on a grid large enough to measure against HBM
+CONFIGS["ns2d_steady_4096"] = dict(op=NS_2D_STEADY, shape=(4096, 4096),
+                                   domain=((0.0, 1.0), (0.0, 1.0)), bc=(INTERIOR, INTERIOR))
+EXTRA_CONFIGS = ("ns2d_steady_4096",)
 CONFIG_ORDER = ("burgers_256x128", "poisson_1024", "grayscott_4096", "helmholtz_256", "ns_tgv_128x16")
 
 OP_META = {
@@ -123,6 +129,7 @@ OP_META = {
     HELMHOLTZ_3D_O4: dict(fields=("u",), sources=("f",), residuals=("r",), ncoeffs=1),
     NS_3D_T: dict(fields=("u", "v", "w", "p"), sources=(),
                   residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
+    NS_2D_STEADY: dict(fields=("u", "v", "p"), sources=(), residuals=("res_u", "res_v", "res_div"), ncoeffs=1),
 }
 DEFAULT_COEFFS = {
     BURGERS_1D_T: (0.01 / math.pi,),
@@ -130,6 +137,7 @@ DEFAULT_COEFFS = {
     GRAYSCOTT_2D: (2e-5, 1e-5, 0.04, 0.06),
     HELMHOLTZ_3D_O4: (4 * math.pi,),
     NS_3D_T: (0.01,),
+    NS_2D_STEADY: (0.01,),
 }
 
 
@@ -180,10 +188,16 @@ def analytic_fields(op: str, axes: Sequence[np.ndarray], coeffs: Sequence[float]
         w = np.zeros(shape)
         p = (np.cos(2 * x) + np.cos(2 * y)) * (np.cos(2 * z) + 2.0) / 16.0 * e4
         return [np.broadcast_to(a, shape).copy() for a in (u, v, w, p)], []
+    if op == NS_2D_STEADY:
+        x, y = _bcast(axes, 0), _bcast(axes, 1)
+        u = np.sin(math.pi * x) * np.cos(math.pi * y)
+        v = -np.cos(math.pi * x) * np.sin(math.pi * y)
+        p = 0.25 * (np.cos(2 * math.pi * x) + np.cos(2 * math.pi * y))
+        return [np.broadcast_to(a, shape).copy() for a in (u, v, p)], []
     raise ValueError(op)
 
 
-_NOISE_SIGMA = {BURGERS_1D_T: 0.01, POISSON_2D: 0.05, HELMHOLTZ_3D_O4: 0.05, NS_3D_T: 0.01}
+_NOISE_SIGMA = {BURGERS_1D_T: 0.01, POISSON_2D: 0.05, HELMHOLTZ_3D_O4: 0.05, NS_3D_T: 0.01, NS_2D_STEADY: 0.01}
 
 
 def make(name: str, seed: int = 42, shape: Optional[Sequence[int]] = None, kind: str = "config",
@@ -199,7 +213,7 @@ def make(name: str, seed: int = 42, shape: Optional[Sequence[int]] = None, kind:
               profile is then evaluated on the nodes ``lo + i*h``).
     """
     if name in OPS:
-        name = next(k for k in CONFIG_ORDER if CONFIGS[k]["op"] == name)
+        name = next(k for k in CONFIG_ORDER + EXTRA_CONFIGS if CONFIGS[k]["op"] == name)
     cfg = CONFIGS[name]
     op = cfg["op"]
     shape = tuple(int(s) for s in (shape if shape is not None else cfg["shape"]))

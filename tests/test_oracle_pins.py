@@ -297,6 +297,7 @@ CASES = [
     (W.GRAYSCOTT_2D, (6, 7), (0.2, 0.3), (0.7, 0.3, 0.04, 0.06)),
     (W.HELMHOLTZ_3D_O4, (8, 7, 9), (0.2, 0.3, 0.25), (1.3,)),
     (W.NS_3D_T, (5, 6, 5, 6), (0.3, 0.2, 0.25, 0.15), (0.13,)),
+    (W.NS_2D_STEADY, (8, 9), (0.2, 0.3), (0.17,)),
 ]
 
 
@@ -342,6 +343,7 @@ TINY = [
     (W.GRAYSCOTT_2D, (5, 6), (0.2, 0.3), (0.7, 0.3, 0.04, 0.06)),
     (W.HELMHOLTZ_3D_O4, (7, 6, 7), (0.2, 0.3, 0.25), (1.3,)),
     (W.NS_3D_T, (4, 5, 4, 5), (0.3, 0.2, 0.25, 0.15), (0.13,)),
+    (W.NS_2D_STEADY, (6, 7), (0.2, 0.3), (0.17,)),
 ]
 
 
@@ -403,6 +405,54 @@ def test_ns_adjoint_reduces_to_printed_2d_equation():
     # and the pressure gradient is the transposed centred pressure derivatives
     gp = (xm(Gu2) - xp(Gu2)) / (2 * dx) + (ym(Gv2) - yp(Gv2)) / (2 * dy)
     assert np.allclose(g[3][:, :, 1, 3], gp, rtol=0, atol=1e-12)
+
+
+def test_ns2d_steady_printed_u_adjoint_directly():
+    """The operator the paper spells out: at nodes whose four neighbours all carry rows, the
+    oracle's dL/du must be the printed Eq. (1) term by term (no reduction needed here)."""
+    nx, ny, dx, dy, nu = 9, 8, 0.3, 0.2, 0.17
+    r = np.random.default_rng(21)
+    u, v, p = (r.standard_normal((nx, ny)) for _ in range(3))
+    Gu, Gv, Gd = (r.standard_normal((nx, ny)) for _ in range(3))
+    g = oracle.bwd(W.NS_2D_STEADY, [u, v, p], [Gu, Gv, Gd], (nx, ny), (dx, dy), (nu,))
+    for i in range(2, nx - 2):
+        for j in range(2, ny - 2):
+            u_x = (u[i + 1, j] - u[i - 1, j]) / (2 * dx)
+            v_x = (v[i + 1, j] - v[i - 1, j]) / (2 * dx)
+            printed = (Gu[i, j] * (u_x + 2 * nu / dx ** 2 + 2 * nu / dy ** 2)
+                       + Gu[i - 1, j] * (u[i - 1, j] / (2 * dx) - nu / dx ** 2)
+                       + Gu[i + 1, j] * (-u[i + 1, j] / (2 * dx) - nu / dx ** 2)
+                       + Gu[i, j - 1] * (v[i, j - 1] / (2 * dy) - nu / dy ** 2)
+                       + Gu[i, j + 1] * (-v[i, j + 1] / (2 * dy) - nu / dy ** 2)
+                       + Gv[i, j] * v_x
+                       + (Gd[i - 1, j] - Gd[i + 1, j]) / (2 * dx))
+            assert abs(g[0][i, j] - printed) < 1e-11
+    # corner nodes of the ring are read by no row
+    assert g[0][0, 0] == 0 and g[1][-1, -1] == 0 and g[2][0, -1] == 0
+
+
+def test_ns2d_steady_quadratic_exact():
+    shape, h = (7, 8), (0.25, 0.2)
+    x, y = _mesh(shape, h, [0.1, -0.3])
+    def quad(c):
+        return c[0] + c[1] * x + c[2] * y + c[3] * x * y + c[4] * x * x + c[5] * y * y
+    def der(c):
+        return dict(x=c[1] + c[3] * y + 2 * c[4] * x, y=c[2] + c[3] * x + 2 * c[5] * y, lap=2 * c[4] + 2 * c[5])
+    cs = [np.random.default_rng(31 + k).standard_normal(6) for k in range(3)]
+    u, v, p = (quad(c) for c in cs)
+    du, dv, dp = (der(c) for c in cs)
+    nu = 0.23
+    R, loss, rows = oracle.fwd(W.NS_2D_STEADY, [u, v, p], [], shape, h, (nu,))
+    ex = [u * du["x"] + v * du["y"] + dp["x"] - nu * du["lap"],
+          u * dv["x"] + v * dv["y"] + dp["y"] - nu * dv["lap"],
+          du["x"] + dv["y"]]
+    inner = (slice(1, -1),) * 2
+    assert rows == 5 * 6
+    for rr, e in zip(R, ex):
+        assert np.allclose(rr[inner], e[inner], rtol=0, atol=1e-11)
+        mask = np.ones(shape, bool); mask[inner] = False
+        assert np.all(rr[mask] == 0.0)
+    assert abs(loss[3] - sum(np.sum(e[inner] ** 2) for e in ex) / rows) < 1e-10
 
 
 # --------------------------------------------------------------------------------------------
