@@ -44,6 +44,7 @@ ALGO_BYTES = {                      # op: (fwd, bwd)
     W.GRAYSCOTT_2D: (16, 24),
     W.HELMHOLTZ_3D_O4: (12, 8),
     W.NS_3D_T: (32, 44),
+    W.NS_2D_STEADY: (24, 32),
 }
 KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
     W.BURGERS_1D_T: ("burgers_fwd_kernel", "burgers_bwd_kernel"),
@@ -51,6 +52,7 @@ KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
     W.GRAYSCOTT_2D: ("lap2d_kernel<GrayScottFwd>", "lap2d_kernel<GrayScottBwd>"),
     W.HELMHOLTZ_3D_O4: ("star3d_kernel<fwd>", "star3d_kernel<bwd>"),
     W.NS_3D_T: ("ns_fwd_kernel", "ns_bwd_kernel"),
+    W.NS_2D_STEADY: ("ns2d_kernel<fwd>", "ns2d_kernel<bwd>"),
 }
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None where no capture has been taken yet.
@@ -333,7 +335,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(W.CONFIG_ORDER))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(W.CONFIG_ORDER + W.EXTRA_CONFIGS))
     ap.add_argument("--impl", default="fpde", choices=["fpde", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip per-config figures and the CPU baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
@@ -423,7 +425,7 @@ def main():
     if world == 1 and not args.no_extras:
         del prob
         torch.cuda.empty_cache()
-        line["per_config"] = {name: config_line(torch, B, name, 30, 5, peak) for name in W.CONFIG_ORDER}
+        line["per_config"] = {name: config_line(torch, B, name, 30, 5, peak) for name in W.CONFIG_ORDER + W.EXTRA_CONFIGS}
         line["cpu_baseline"] = cpu_baseline(args.workload)
     if rank == 0:
         print(json.dumps(line))

@@ -69,6 +69,12 @@ typedef enum {
  *        mom_q = d_t q + u d_x q + v d_y q + w d_z q + d_{a_q} p - nu Lap q, continuity =
  *        d_x u + d_y v + d_z w (Section 2.1's residuals extended by t, w and z), centred
  *        differences.  bc = (PERIODIC x3, INTERIOR): rows at t-index 1..n_t-2.
+ *  FPDE_OP_NS_2D_STEADY    (x,y) array.  fields [u,v,p]; residuals [res_u, res_v, res_div];
+ *        coeffs [nu].  The paper's worked operator (Section 2.1):
+ *        res_u = u u_x + v u_y + p_x - nu Lap u, res_v = u v_x + v v_y + p_y - nu Lap v,
+ *        res_div = u_x + v_y, centred differences; its adjoint is Eq. 1 (and the analogous
+ *        expressions for v and p).  bc = (INTERIOR, INTERIOR): rows at the interior nodes, the
+ *        outer ring is data and receives gradient.
  *
  * Shape rules: the contiguous extent must be a multiple of 4 (float4 path) except for
  * BURGERS_1D_T; PERIODIC / INTERIOR axes need n >= 2*radius+1, ONE_SIDED axes n >= 4; the
@@ -80,7 +86,8 @@ typedef enum {
     FPDE_OP_GRAYSCOTT_2D = 2,
     FPDE_OP_HELMHOLTZ_3D_O4 = 3,
     FPDE_OP_NS_3D_T = 4,
-    FPDE_OP_COUNT = 5
+    FPDE_OP_NS_2D_STEADY = 5,
+    FPDE_OP_COUNT = 6
 } fpde_op;
 
 /* Boundary kind of one array axis (Appendix A.4 names the three causes of boundary terms:

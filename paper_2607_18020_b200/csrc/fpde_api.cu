@@ -16,6 +16,7 @@ int lap2d_items(const int* n);
 int star3d_items(const int* n);
 int ns_items(const int* n);
 int burgers_items(const int* n);
+int ns2d_items(const int* n);
 
 struct OpEntry {
     int ndim, nf, ns, ne, nc, radius;
@@ -29,6 +30,7 @@ static const OpEntry REGISTRY[FPDE_OP_COUNT] = {
     /* GRAYSCOTT_2D    */ {2, 2, 0, 2, 4, 1, {FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, 0, 0}, true},
     /* HELMHOLTZ_3D_O4 */ {3, 1, 1, 1, 1, 2, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0}, true},
     /* NS_3D_T         */ {4, 4, 0, 4, 1, 1, {FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_INTERIOR}, true},
+    /* NS_2D_STEADY    */ {2, 3, 0, 3, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0, 0}, true},
 };
 
 static int check_shape(int op, int ndim, const int64_t* shape, int* n_out, int64_t* total, int64_t* rows) {
@@ -60,6 +62,7 @@ static size_t workspace_need(int op, const int* n) {
     case FPDE_OP_GRAYSCOTT_2D: items = lap2d_items(n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: items = star3d_items(n); break;
     case FPDE_OP_NS_3D_T: items = ns_items(n); break;
+    case FPDE_OP_NS_2D_STEADY: items = ns2d_items(n); break;
     }
     return (size_t)items * REGISTRY[op].ne * sizeof(float);
 }
@@ -237,6 +240,7 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_fwd(q); items = lap2d_items(q.n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q); items = star3d_items(q.n); break;
     case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n); break;
+    case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_fwd(q); items = ns2d_items(q.n); break;
     }
     if (ce != cudaSuccess) return FPDE_ERR_CUDA;
     if (loss_out) {
@@ -277,6 +281,7 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
     case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_bwd(q); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_bwd(q); break;
     case FPDE_OP_NS_3D_T: ce = launch_ns_bwd(q); break;
+    case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_bwd(q); break;
     }
     return ce == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
 }
