@@ -295,6 +295,35 @@ def e2e_steps(torch, B, w, steps, warmup, barrier):
     return e0.elapsed_time(e1), nbytes * (len(hf) + len(hs)), nbytes * len(hg) + 8 * (ne + 1), loss
 
 
+def graph_points_per_s(torch, prob, N, pairs, replays):
+    """`pairs` forward+adjoint pairs captured into one CUDA graph and replayed; None if capture is
+    not possible here."""
+    try:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            prob.fwd(); prob.bwd()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            for _ in range(pairs):
+                prob.fwd(); prob.bwd()
+        for _ in range(2):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(replays):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return N * pairs * replays / (e0.elapsed_time(e1) * 1e-3)
+    except Exception:
+        torch.cuda.synchronize()
+        return None
+
+
 def config_line(torch, B, name, steps, warmup, peak):
     """Secondary figures for one configuration: per-call medians with an L2 flush (a 256 MiB
     write) before every step, so small grids are measured cold like large ones."""
@@ -310,6 +339,13 @@ def config_line(torch, B, name, steps, warmup, peak):
            "gbs_fwd": fb * N / (fm * 1e-3) / 1e9, "gbs_bwd": bb * N / (bm * 1e-3) / 1e9,
            "gbs_pair": (fb + bb) * N / ((fm + bm) * 1e-3) / 1e9}
     out["frac_pair"] = out["gbs_pair"] / peak
+    out["timing"] = "cold: 256 MiB L2 flush before every step, per-call medians"
+    # warm, back to back (working sets below L2 stay resident: say so), and the same pairs replayed
+    # from one CUDA graph, which removes the host launch gaps of the latency-bound small grids
+    total_ms, _, _ = timed_steps(torch, prob, steps, 3, lambda: None)
+    out["warm_points_per_s"] = N * steps / (total_ms * 1e-3)
+    out["l2_resident"] = bool((fb + bb) * N < (100 << 20))
+    out["graph_points_per_s"] = graph_points_per_s(torch, prob, N, pairs=10, replays=max(3, steps // 10))
     del prob, flush
     torch.cuda.empty_cache()
     return out
