@@ -62,8 +62,10 @@ NCU_TRAFFIC_BYTES = {
     ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 772754432,
     ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 224121600,
     ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 366544128,
-    ("helmholtz_256", "star3d_kernel<fwd>"): 191179264,
-    ("helmholtz_256", "star3d_kernel<bwd>"): 97971968,
+    ("helmholtz_256", "star3d_kernel<fwd>"): 194467328,
+    ("helmholtz_256", "star3d_kernel<bwd>"): 101209600,
+    ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 361327360,
+    ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 507760640,
 }
 FALLBACK_HBM_GBS = 6650.0
 LAUNCHES_PER_STEP = 3               # forward kernel, loss finalise, adjoint kernel
