@@ -53,10 +53,6 @@ inline cudaError_t launch_kernel_smem(void (*kernel)(KArgs...), dim3 grid, dim3 
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
 }
 
-// Number of loss partial sums (= work items) per residual field the forward kernel of this
-// operator produces for this grid.  Fixed by the grid alone, so the reduction order is too.
-int fwd_items(int op, const int* n);
-
 // Launchers: return cudaGetLastError() after queuing the kernels.
 cudaError_t launch_burgers_fwd(const Problem& p);
 cudaError_t launch_burgers_bwd(const Problem& p);
