@@ -33,7 +33,8 @@
 typedef long long i64;
 
 enum { OP_BURGERS_1D_T = 0, OP_POISSON_2D = 1, OP_GRAYSCOTT_2D = 2, OP_HELMHOLTZ_3D_O4 = 3,
-       OP_NS_3D_T = 4, OP_NS_2D_STEADY = 5, OP_COUNT = 6 };
+       OP_NS_3D_T = 4, OP_NS_2D_STEADY = 5, OP_NS_3D_STEADY = 6,
+       OP_COUNT = 7 };
 enum { BC_PERIODIC = 0, BC_INTERIOR = 1, BC_ONE_SIDED = 2 };
 
 /* A 1-D difference formula at one node: value = sum_k w[k] * q[idx[k]] along one axis. */
@@ -114,11 +115,11 @@ static void scatter(const stencil* s, double* line, i64 stride, double a) {
     for (k = 0; k < s->n; ++k) line[s->idx[k] * stride] += a * s->w[k];
 }
 
-static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2 };
-static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3 };
-static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0 };
-static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3 };
-static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1 };
+static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2, 3 };
+static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4 };
+static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0, 0 };
+static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4 };
+static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1, 1 };
 static const int OP_BC[OP_COUNT][4] = {
     { BC_ONE_SIDED, BC_ONE_SIDED, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
@@ -126,6 +127,7 @@ static const int OP_BC[OP_COUNT][4] = {
     { BC_INTERIOR, BC_INTERIOR, BC_INTERIOR, 0 },
     { BC_PERIODIC, BC_PERIODIC, BC_PERIODIC, BC_INTERIOR },
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
+    { BC_INTERIOR, BC_INTERIOR, BC_INTERIOR, 0 },
 };
 
 int fpde_oracle_info(int op, int* ndim, int* nf, int* ns, int* ne, int* nc) {
@@ -358,6 +360,59 @@ static i64 ns2d(int mode, const double* const* fld, double* const* res, const do
     return rows;
 }
 
+/* Steady incompressible Navier-Stokes on an (x,y,z) array: Section 2.1's system with w and d_z
+ * added (the paper's 3-D steady operator), centred differences, rows at the interior nodes:
+ *   mom_q = u d_x q + v d_y q + w d_z q + d_{a_q} p - nu (d_xx + d_yy + d_zz) q,  q in (u,v,w),
+ *   cont  = d_x u + d_y v + d_z w.
+ * fld = {u,v,w,p}; res / G / grd index: 0..2 momentum x,y,z, 3 continuity. */
+static i64 ns3d(int mode, const double* const* fld, double* const* res, const double* const* G,
+                double* const* grd, const i64* n, const double* h, const double* c) {
+    i64 i[3], rows = 0, st[3];
+    double nu = c[0];
+    st[2] = 1; st[1] = n[2]; st[0] = n[1] * n[2];
+    for (i[0] = 0; i[0] < n[0]; ++i[0]) for (i[1] = 0; i[1] < n[1]; ++i[1]) for (i[2] = 0; i[2] < n[2]; ++i[2]) {
+        stencil s1[3], s2[3];
+        i64 p = i[0] * st[0] + i[1] * st[1] + i[2];
+        i64 base[3];
+        double vel[3], dq[3][3], lap[3], dp[3];
+        int a, q, ok = 1;
+        for (a = 0; a < 3; ++a) {
+            if (!d1(BC_INTERIOR, i[a], n[a], h[a], &s1[a])) ok = 0;
+            else d2(BC_INTERIOR, i[a], n[a], h[a], &s2[a]);
+        }
+        if (!ok) continue;
+        for (a = 0; a < 3; ++a) base[a] = p - i[a] * st[a];
+        ++rows;
+        for (q = 0; q < 3; ++q) {
+            vel[q] = fld[q][p];
+            lap[q] = 0.0;
+            for (a = 0; a < 3; ++a) {
+                dq[q][a] = apply(&s1[a], fld[q] + base[a], st[a]);
+                lap[q] += apply(&s2[a], fld[q] + base[a], st[a]);
+            }
+            dp[q] = apply(&s1[q], fld[3] + base[q], st[q]);
+        }
+        if (mode == 0) {
+            for (q = 0; q < 3; ++q)
+                res[q][p] = vel[0] * dq[q][0] + vel[1] * dq[q][1] + vel[2] * dq[q][2] + dp[q] - nu * lap[q];
+            res[3][p] = dq[0][0] + dq[1][1] + dq[2][2];
+        } else {
+            for (q = 0; q < 3; ++q) {
+                double Gq = G[q][p];
+                for (a = 0; a < 3; ++a) {
+                    grd[a][p] += Gq * dq[q][a];                                  /* factor c_a       */
+                    scatter(&s1[a], grd[q] + base[a], st[a], Gq * vel[a]);       /* c_a * d_a q      */
+                    scatter(&s2[a], grd[q] + base[a], st[a], -Gq * nu);          /* -nu d_aa q       */
+                }
+                scatter(&s1[q], grd[3] + base[q], st[q], Gq);                    /* d_{a_q} p        */
+            }
+            for (a = 0; a < 3; ++a)
+                scatter(&s1[a], grd[a] + base[a], st[a], G[3][p]);               /* continuity row   */
+        }
+    }
+    return rows;
+}
+
 static i64 total(int ndim, const i64* n) { i64 N = 1; int a; for (a = 0; a < ndim; ++a) N *= n[a]; return N; }
 
 static int check(int op, int ndim, const i64* n) {
@@ -388,6 +443,7 @@ i64 fpde_oracle_fwd(int op, const double* const* fields, const double* const* so
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(0, fields[0], sources[0], residuals[0], NULL, NULL, shape, spacing, coeffs); break;
     case OP_NS_3D_T: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
     case OP_NS_2D_STEADY: rows = ns2d(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
+    case OP_NS_3D_STEADY: rows = ns3d(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
     }
     if (loss) {
         loss[E] = 0.0;
@@ -417,6 +473,7 @@ i64 fpde_oracle_bwd(int op, const double* const* fields, const double* const* G,
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(1, fields[0], NULL, NULL, G[0], gfields[0], shape, spacing, coeffs); break;
     case OP_NS_3D_T: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
     case OP_NS_2D_STEADY: rows = ns2d(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
+    case OP_NS_3D_STEADY: rows = ns3d(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
     }
     return rows;
 }

@@ -33,7 +33,8 @@ GRAYSCOTT_2D = "grayscott_2d"
 HELMHOLTZ_3D_O4 = "helmholtz_3d_o4"
 NS_3D_T = "ns_3d_t"
 NS_2D_STEADY = "ns_2d_steady"
-OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY)
+NS_3D_STEADY = "ns_3d_steady"
+OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY, NS_3D_STEADY)
 
 # Boundary kinds per array axis.
 PERIODIC = "periodic"      # rows at every node, wrap-around neighbours
@@ -119,7 +120,9 @@ CONFIGS: Dict[str, dict] = {
 # Navier-Stokes, its lid-driven-cavity case) on a grid large enough to measure against HBM
 CONFIGS["ns2d_steady_4096"] = dict(op=NS_2D_STEADY, shape=(4096, 4096),
                                    domain=((0.0, 1.0), (0.0, 1.0)), bc=(INTERIOR, INTERIOR))
-EXTRA_CONFIGS = ("ns2d_steady_4096",)
+CONFIGS["ns3d_steady_256"] = dict(op=NS_3D_STEADY, shape=(256, 256, 256),
+                                  domain=((0.0, 1.0),) * 3, bc=(INTERIOR,) * 3)
+EXTRA_CONFIGS = ("ns2d_steady_4096", "ns3d_steady_256")
 CONFIG_ORDER = ("burgers_256x128", "poisson_1024", "grayscott_4096", "helmholtz_256", "ns_tgv_128x16")
 
 OP_META = {
@@ -130,6 +133,8 @@ OP_META = {
     NS_3D_T: dict(fields=("u", "v", "w", "p"), sources=(),
                   residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
     NS_2D_STEADY: dict(fields=("u", "v", "p"), sources=(), residuals=("res_u", "res_v", "res_div"), ncoeffs=1),
+    NS_3D_STEADY: dict(fields=("u", "v", "w", "p"), sources=(),
+                       residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
 }
 DEFAULT_COEFFS = {
     BURGERS_1D_T: (0.01 / math.pi,),
@@ -138,6 +143,7 @@ DEFAULT_COEFFS = {
     HELMHOLTZ_3D_O4: (4 * math.pi,),
     NS_3D_T: (0.01,),
     NS_2D_STEADY: (0.01,),
+    NS_3D_STEADY: (0.01,),
 }
 
 
@@ -194,10 +200,18 @@ def analytic_fields(op: str, axes: Sequence[np.ndarray], coeffs: Sequence[float]
         v = -np.cos(math.pi * x) * np.sin(math.pi * y)
         p = 0.25 * (np.cos(2 * math.pi * x) + np.cos(2 * math.pi * y))
         return [np.broadcast_to(a, shape).copy() for a in (u, v, p)], []
+    if op == NS_3D_STEADY:
+        x, y, z = (_bcast(axes, a) for a in range(3))
+        pi = math.pi
+        u = np.sin(pi * x) * np.cos(pi * y) * np.cos(pi * z)
+        v = -0.5 * np.cos(pi * x) * np.sin(pi * y) * np.cos(pi * z)
+        w = -0.5 * np.cos(pi * x) * np.cos(pi * y) * np.sin(pi * z)
+        p = 0.25 * (np.cos(2 * pi * x) + np.cos(2 * pi * y) + np.cos(2 * pi * z))
+        return [np.broadcast_to(a, shape).copy() for a in (u, v, w, p)], []
     raise ValueError(op)
 
 
-_NOISE_SIGMA = {BURGERS_1D_T: 0.01, POISSON_2D: 0.05, HELMHOLTZ_3D_O4: 0.05, NS_3D_T: 0.01, NS_2D_STEADY: 0.01}
+_NOISE_SIGMA = {BURGERS_1D_T: 0.01, POISSON_2D: 0.05, HELMHOLTZ_3D_O4: 0.05, NS_3D_T: 0.01, NS_2D_STEADY: 0.01, NS_3D_STEADY: 0.01}
 
 
 def make(name: str, seed: int = 42, shape: Optional[Sequence[int]] = None, kind: str = "config",

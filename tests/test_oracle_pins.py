@@ -298,6 +298,7 @@ CASES = [
     (W.HELMHOLTZ_3D_O4, (8, 7, 9), (0.2, 0.3, 0.25), (1.3,)),
     (W.NS_3D_T, (5, 6, 5, 6), (0.3, 0.2, 0.25, 0.15), (0.13,)),
     (W.NS_2D_STEADY, (8, 9), (0.2, 0.3), (0.17,)),
+    (W.NS_3D_STEADY, (6, 7, 5), (0.2, 0.3, 0.25), (0.17,)),
 ]
 
 
@@ -344,6 +345,7 @@ TINY = [
     (W.HELMHOLTZ_3D_O4, (7, 6, 7), (0.2, 0.3, 0.25), (1.3,)),
     (W.NS_3D_T, (4, 5, 4, 5), (0.3, 0.2, 0.25, 0.15), (0.13,)),
     (W.NS_2D_STEADY, (6, 7), (0.2, 0.3), (0.17,)),
+    (W.NS_3D_STEADY, (5, 4, 5), (0.2, 0.3, 0.25), (0.17,)),
 ]
 
 
@@ -429,6 +431,48 @@ def test_ns2d_steady_printed_u_adjoint_directly():
             assert abs(g[0][i, j] - printed) < 1e-11
     # corner nodes of the ring are read by no row
     assert g[0][0, 0] == 0 and g[1][-1, -1] == 0 and g[2][0, -1] == 0
+
+
+def test_ns3d_steady_reduces_to_printed_2d_equation_and_is_quadratic_exact():
+    # (a) fields constant in z, w = 0: at nodes whose neighbours carry rows, dL/du is Eq. (1)
+    nx, ny, nz, dx, dy, dz, nu = 8, 7, 6, 0.3, 0.2, 0.4, 0.17
+    r = np.random.default_rng(5)
+    ext = lambda a2: np.broadcast_to(a2[:, :, None], (nx, ny, nz)).copy()
+    u2, v2, p2, Gu2, Gv2, Gw2, Gd2 = (r.standard_normal((nx, ny)) for _ in range(7))
+    g = oracle.bwd(W.NS_3D_STEADY, [ext(u2), ext(v2), np.zeros((nx, ny, nz)), ext(p2)],
+                   [ext(Gu2), ext(Gv2), ext(Gw2), ext(Gd2)], (nx, ny, nz), (dx, dy, dz), (nu,))
+    for i in range(2, nx - 2):
+        for j in range(2, ny - 2):
+            u_x = (u2[i + 1, j] - u2[i - 1, j]) / (2 * dx)
+            v_x = (v2[i + 1, j] - v2[i - 1, j]) / (2 * dx)
+            printed = (Gu2[i, j] * (u_x + 2 * nu / dx ** 2 + 2 * nu / dy ** 2)
+                       + Gu2[i - 1, j] * (u2[i - 1, j] / (2 * dx) - nu / dx ** 2)
+                       + Gu2[i + 1, j] * (-u2[i + 1, j] / (2 * dx) - nu / dx ** 2)
+                       + Gu2[i, j - 1] * (v2[i, j - 1] / (2 * dy) - nu / dy ** 2)
+                       + Gu2[i, j + 1] * (-v2[i, j + 1] / (2 * dy) - nu / dy ** 2)
+                       + Gv2[i, j] * v_x + (Gd2[i - 1, j] - Gd2[i + 1, j]) / (2 * dx))
+            for k in range(2, nz - 2):      # z neighbours carry rows too: their terms cancel
+                assert abs(g[0][i, j, k] - printed) < 1e-11
+    # (b) quadratic fields: every centred difference is exact
+    shape, h = (6, 5, 7), (0.25, 0.2, 0.3)
+    x, y, z = _mesh(shape, h, [0.1, -0.3, 0.2])
+    def quad(c):
+        return c[0] + c[1] * x + c[2] * y + c[3] * z + c[4] * x * y + c[5] * y * z + c[6] * x * x + c[7] * y * y + c[8] * z * z
+    def der(c):
+        return dict(x=c[1] + c[4] * y + 2 * c[6] * x, y=c[2] + c[4] * x + c[5] * z + 2 * c[7] * y,
+                    z=c[3] + c[5] * y + 2 * c[8] * z, lap=2 * (c[6] + c[7] + c[8]))
+    cs = [np.random.default_rng(41 + k).standard_normal(9) for k in range(4)]
+    u, v, w, p = (quad(c) for c in cs)
+    du, dv, dw, dp = (der(c) for c in cs)
+    R, loss, rows = oracle.fwd(W.NS_3D_STEADY, [u, v, w, p], [], shape, h, (0.23,))
+    ex = [u * d["x"] + v * d["y"] + w * d["z"] + dp[a] - 0.23 * d["lap"] for d, a in ((du, "x"), (dv, "y"), (dw, "z"))]
+    ex.append(du["x"] + dv["y"] + dw["z"])
+    inner = (slice(1, -1),) * 3
+    assert rows == 4 * 3 * 5
+    for rr, e in zip(R, ex):
+        assert np.allclose(rr[inner], e[inner], rtol=0, atol=1e-11)
+        mask = np.ones(shape, bool); mask[inner] = False
+        assert np.all(rr[mask] == 0.0)
 
 
 def test_ns2d_steady_quadratic_exact():
