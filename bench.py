@@ -45,6 +45,7 @@ ALGO_BYTES = {                      # op: (fwd, bwd)
     W.HELMHOLTZ_3D_O4: (12, 8),
     W.NS_3D_T: (32, 44),
     W.NS_2D_STEADY: (24, 32),
+    W.NS_3D_STEADY: (32, 44),
 }
 KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
     W.BURGERS_1D_T: ("burgers_fwd_kernel", "burgers_bwd_kernel"),
@@ -53,6 +54,7 @@ KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
     W.HELMHOLTZ_3D_O4: ("star3d_kernel<fwd>", "star3d_kernel<bwd>"),
     W.NS_3D_T: ("ns_fwd_kernel", "ns_bwd_kernel"),
     W.NS_2D_STEADY: ("ns2d_kernel<fwd>", "ns2d_kernel<bwd>"),
+    W.NS_3D_STEADY: ("ns3d_kernel<fwd>", "ns3d_kernel<bwd>"),
 }
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None where no capture has been taken yet.

@@ -75,6 +75,11 @@ typedef enum {
  *        res_div = u_x + v_y, centred differences; its adjoint is Eq. 1 (and the analogous
  *        expressions for v and p).  bc = (INTERIOR, INTERIOR): rows at the interior nodes, the
  *        outer ring is data and receives gradient.
+ *  FPDE_OP_NS_3D_STEADY    (x,y,z) array.  fields [u,v,w,p];
+ *        residuals [mom_x, mom_y, mom_z, continuity]; coeffs [nu].  Section 2.1's system with
+ *        the third component: mom_q = u d_x q + v d_y q + w d_z q + d_{a_q} p - nu Lap q,
+ *        continuity = d_x u + d_y v + d_z w, centred differences.  bc = (INTERIOR x3): rows at
+ *        the interior nodes, the outer shell is data and receives gradient.
  *
  * Shape rules: the contiguous extent must be a multiple of 4 (float4 path) except for
  * BURGERS_1D_T; PERIODIC / INTERIOR axes need n >= 2*radius+1, ONE_SIDED axes n >= 4; the
@@ -87,7 +92,8 @@ typedef enum {
     FPDE_OP_HELMHOLTZ_3D_O4 = 3,
     FPDE_OP_NS_3D_T = 4,
     FPDE_OP_NS_2D_STEADY = 5,
-    FPDE_OP_COUNT = 6
+    FPDE_OP_NS_3D_STEADY = 6,
+    FPDE_OP_COUNT = 7
 } fpde_op;
 
 /* Boundary kind of one array axis (Appendix A.4 names the three causes of boundary terms:

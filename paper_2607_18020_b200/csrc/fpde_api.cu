@@ -17,6 +17,7 @@ int star3d_items(const int* n);
 int ns_items(const int* n);
 int burgers_items(const int* n);
 int ns2d_items(const int* n);
+int ns3d_items(const int* n);
 
 struct OpEntry {
     int ndim, nf, ns, ne, nc, radius;
@@ -31,6 +32,7 @@ static const OpEntry REGISTRY[FPDE_OP_COUNT] = {
     /* HELMHOLTZ_3D_O4 */ {3, 1, 1, 1, 1, 2, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0}, true},
     /* NS_3D_T         */ {4, 4, 0, 4, 1, 1, {FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_INTERIOR}, true},
     /* NS_2D_STEADY    */ {2, 3, 0, 3, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0, 0}, true},
+    /* NS_3D_STEADY    */ {3, 4, 0, 4, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0}, true},
 };
 
 static int check_shape(int op, int ndim, const int64_t* shape, int* n_out, int64_t* total, int64_t* rows) {
@@ -63,6 +65,7 @@ static size_t workspace_need(int op, const int* n) {
     case FPDE_OP_HELMHOLTZ_3D_O4: items = star3d_items(n); break;
     case FPDE_OP_NS_3D_T: items = ns_items(n); break;
     case FPDE_OP_NS_2D_STEADY: items = ns2d_items(n); break;
+    case FPDE_OP_NS_3D_STEADY: items = ns3d_items(n); break;
     }
     return (size_t)items * REGISTRY[op].ne * sizeof(float);
 }
@@ -241,6 +244,7 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q); items = star3d_items(q.n); break;
     case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n); break;
     case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_fwd(q); items = ns2d_items(q.n); break;
+    case FPDE_OP_NS_3D_STEADY: ce = launch_ns3d_fwd(q); items = ns3d_items(q.n); break;
     }
     if (ce != cudaSuccess) return FPDE_ERR_CUDA;
     if (loss_out) {
@@ -282,6 +286,7 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_bwd(q); break;
     case FPDE_OP_NS_3D_T: ce = launch_ns_bwd(q); break;
     case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_bwd(q); break;
+    case FPDE_OP_NS_3D_STEADY: ce = launch_ns3d_bwd(q); break;
     }
     return ce == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
 }

@@ -69,6 +69,14 @@ __device__ __forceinline__ V4 v4fma(V4 a, float2 s, V4 c) { V4 r; r.lo = fma2(a.
 // a * b + c
 __device__ __forceinline__ V4 v4fmav(V4 a, V4 b, V4 c) { V4 r; r.lo = fma2(a.lo, b.lo, c.lo); r.hi = fma2(a.hi, b.hi, c.hi); return r; }
 
+// a float4 shifted by one element to the left / right along the row
+__device__ __forceinline__ V4 shift_left(const V4& c, float l1) {    // value at column j-1
+    V4 r; r.lo = make_float2(l1, c.lo.x); r.hi = make_float2(c.lo.y, c.hi.x); return r;
+}
+__device__ __forceinline__ V4 shift_right(const V4& c, float r1) {   // value at column j+1
+    V4 r; r.lo = make_float2(c.lo.y, c.hi.x); r.hi = make_float2(c.hi.y, r1); return r;
+}
+
 // Values one and two elements to the left / right of a thread's float4 along the contiguous
 // axis.  Inside a warp they come from the neighbouring lane's registers; the first and last
 // lane (and the first / last float4 of a row) fetch them from global memory, wrapped around

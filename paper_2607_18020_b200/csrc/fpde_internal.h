@@ -62,6 +62,8 @@ cudaError_t launch_helmholtz_fwd(const Problem& p);
 cudaError_t launch_helmholtz_bwd(const Problem& p);
 cudaError_t launch_ns2d_fwd(const Problem& p);    // steady 2-D Navier-Stokes
 cudaError_t launch_ns2d_bwd(const Problem& p);
+cudaError_t launch_ns3d_fwd(const Problem& p);    // steady 3-D Navier-Stokes
+cudaError_t launch_ns3d_bwd(const Problem& p);
 cudaError_t launch_ns_fwd(const Problem& p);
 // TMA-staged variants (op_ns3dt_tma.cu); `launched` false = this grid is not eligible
 bool ns_tma_wanted(const int* n);

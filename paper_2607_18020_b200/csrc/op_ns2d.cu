@@ -37,14 +37,6 @@ struct Ns2dParams {
     float* partials;
 };
 
-// a float4 shifted by one element to the left / right along the row
-__device__ __forceinline__ V4 shift_left(const V4& c, float l1) {    // value at column j-1
-    V4 r; r.lo = make_float2(l1, c.lo.x); r.hi = make_float2(c.lo.y, c.hi.x); return r;
-}
-__device__ __forceinline__ V4 shift_right(const V4& c, float r1) {   // value at column j+1
-    V4 r; r.lo = make_float2(c.lo.y, c.hi.x); r.hi = make_float2(c.hi.y, r1); return r;
-}
-
 template <bool BWD>
 __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
     constexpr int NA = BWD ? 5 : 3;

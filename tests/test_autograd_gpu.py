@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 CASES = [("poisson_1024", (36, 40)), ("grayscott_4096", (24, 32)), ("helmholtz_256", (12, 10, 16)),
-         ("ns_tgv_128x16", (6, 8, 8, 8)), ("burgers_256x128", (9, 7)), ("ns2d_steady_4096", (10, 12))]
+         ("ns_tgv_128x16", (6, 8, 8, 8)), ("burgers_256x128", (9, 7)), ("ns2d_steady_4096", (10, 12)),
+         ("ns3d_steady_256", (6, 5, 8))]
 
 
 @pytest.mark.parametrize("name,shape", CASES)

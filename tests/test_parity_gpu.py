@@ -24,6 +24,8 @@ MEDIUM = [
     ("ns_tgv_128x16", (36, 21, 20, 16)),
     ("ns2d_steady_4096", (128, 128)),
     ("ns2d_steady_4096", (203, 300)),
+    ("ns3d_steady_256", (37, 22, 136)),     # ragged plane chunks, y blocks and a partial warp
+    ("ns3d_steady_256", (20, 9, 260)),      # warp edges inside a z line, a ragged column block
 ]
 TINY = [
     ("burgers_256x128", (4, 4)),
@@ -39,12 +41,16 @@ TINY = [
     ("ns_tgv_128x16", (5, 6, 7, 12)),
     ("ns2d_steady_4096", (3, 4)),
     ("ns2d_steady_4096", (36, 40)),
+    ("ns3d_steady_256", (3, 3, 4)),
+    ("ns3d_steady_256", (5, 6, 8)),
+    ("ns3d_steady_256", (7, 5, 132)),
 ]
 FULL = [
     ("grayscott_4096", None),
     ("helmholtz_256", None),
     ("ns_tgv_128x16", None),
     ("ns2d_steady_4096", None),
+    ("ns3d_steady_256", None),
 ]
 
 
@@ -107,7 +113,8 @@ def test_adjoint_alone_random_upstream(name, shape):
 def test_unequal_spacing():
     for name, shape, h in [("poisson_1024", (20, 24), (0.3, 0.07)), ("helmholtz_256", (9, 10, 12), (0.2, 0.15, 0.11)),
                            ("ns_tgv_128x16", (5, 6, 7, 8), (0.3, 0.2, 0.25, 0.1)), ("grayscott_4096", (9, 8), (0.01, 0.02)),
-                           ("burgers_256x128", (11, 7), (0.05, 0.02)), ("ns2d_steady_4096", (9, 12), (0.3, 0.2))]:
+                           ("burgers_256x128", (11, 7), (0.05, 0.02)), ("ns2d_steady_4096", (9, 12), (0.3, 0.2)),
+                           ("ns3d_steady_256", (6, 7, 8), (0.3, 0.2, 0.25))]:
         _check_case(W.make(name, seed=45, shape=shape, kind="randn", spacing=h), name + " unequal spacing")
 
 
