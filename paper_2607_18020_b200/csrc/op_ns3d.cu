@@ -39,113 +39,155 @@ __device__ __forceinline__ void ns3d_prefetch_l2(const float* ptr) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
 }
 
+// per-thread constants of a launch
+struct Ns3dThread {
+    int n0, PS;
+    int rowoff, eoff, ymoff, ypoff;    // element offsets inside a plane: own float4, edge float, y-1, y+1
+    int a1;
+    bool valid, first_col, last_col, efetch, lane_first, lane_last;
+    bool y_dead, ym_dead, yp_dead;     // own row / y-1 / y+1 carry no residual row
+};
+
+// zero extension of an upstream float4 along z (elements z = 0 and z = n2-1)
+__device__ __forceinline__ V4 ns3d_zmask(const Ns3dThread& t, V4 v) {
+    if (t.first_col) v.lo.x = 0.f;
+    if (t.last_col) v.hi.y = 0.f;
+    return v;
+}
+
+// array k at plane r (clamped into the array) at the thread's own float4; with `check`, an
+// upstream float4 whose plane or row is outside the rows reads as zero
+template <bool BWD>
+__device__ __forceinline__ V4 ns3d_load_own(const Ns3dParams& p, const Ns3dThread& t, int k, int r, bool check) {
+    const int rr = max(0, min(t.n0 - 1, r));
+    V4 v = ldv4(p.a[k] + rr * t.PS + t.rowoff);
+    if (BWD && k >= 3) {
+        v = ns3d_zmask(t, v);
+        if (check && (t.y_dead || r < 1 || r > t.n0 - 2)) v = v4zero();
+    }
+    return v;
+}
+
+// One x step: W0 = plane a-1, W1 = plane a, W2 receives plane a+1.  EDGE: some float4 the block
+// reads in this step lies outside the rows (a block-uniform property), so the whole-vector
+// zero extension has to be looked at; the other steps skip those selects.
+template <bool BWD, bool EDGE, int NA>
+__device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread& t, int a, const V4 (&W0)[NA],
+                                          const V4 (&W1)[NA], V4 (&W2)[NA], float2 (&acc)[4]) {
+    constexpr int G0 = 3;                            // adjoint: first upstream array
+    const int pl = a * t.PS;
+    const bool x_dead = a < 1 || a > t.n0 - 2;
+    if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= min(t.a1, t.n0 - 1)) {
+        const int po = (a + 1 + p.prefetch) * t.PS + t.rowoff;
+#pragma unroll
+        for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(p.a[k] + po);
+    }
+    V4 Ym[NA], Yp[NA], Zm[NA], Zp[NA];
+    float E[NA];
+#pragma unroll
+    for (int k = 0; k < NA; ++k) {
+        W2[k] = ns3d_load_own<BWD>(p, t, k, a + 1, EDGE);
+        Ym[k] = ldv4(p.a[k] + pl + t.ymoff);
+        Yp[k] = ldv4(p.a[k] + pl + t.ypoff);
+        E[k] = 0.f;
+        if (t.efetch) E[k] = __ldg(p.a[k] + pl + t.eoff);
+    }
+#pragma unroll
+    for (int k = 0; k < NA; ++k) {
+        if (BWD && k >= G0) {
+            Ym[k] = ns3d_zmask(t, Ym[k]); Yp[k] = ns3d_zmask(t, Yp[k]);
+            if (EDGE) {
+                if (x_dead || t.ym_dead) Ym[k] = v4zero();
+                if (x_dead || t.yp_dead) Yp[k] = v4zero();
+                if (x_dead || t.y_dead) E[k] = 0.f;
+            }
+        }
+        float l1 = __shfl_up_sync(FULL_MASK, W1[k].hi.y, 1);
+        float r1 = __shfl_down_sync(FULL_MASK, W1[k].lo.x, 1);
+        if (t.lane_first) l1 = E[k];
+        if (t.lane_last) r1 = E[k];
+        Zm[k] = shift_left(W1[k], l1);
+        Zp[k] = shift_right(W1[k], r1);
+    }
+    float2 o[4][2];
+    const float2 nodt[3] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        float2 w0[NA], w1[NA], w2[NA], ym[NA], yp[NA], zm[NA], zp[NA], oo[4];
+        v4_half<NA>(W0, h, w0); v4_half<NA>(W1, h, w1); v4_half<NA>(W2, h, w2);
+        v4_half<NA>(Ym, h, ym); v4_half<NA>(Yp, h, yp); v4_half<NA>(Zm, h, zm); v4_half<NA>(Zp, h, zp);
+        if constexpr (BWD) ns_bwd_pair(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
+        else ns_fwd_pair(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e][h] = oo[e];
+    }
+    if (!BWD) {                                      // the outer shell carries no row
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (EDGE && (x_dead || t.y_dead)) { o[e][0] = make_float2(0.f, 0.f); o[e][1] = o[e][0]; }
+            if (t.first_col) o[e][0].x = 0.f;
+            if (t.last_col) o[e][1].y = 0.f;
+        }
+    }
+    if (t.valid) {
+        const int off = pl + t.rowoff;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            stv4(p.out[e] + off, o[e][0], o[e][1]);
+            if (!BWD) acc[e] = fma2(o[e][0], o[e][0], fma2(o[e][1], o[e][1], acc[e]));
+        }
+    }
+}
+
 template <bool BWD, int MINB>
 __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     constexpr int NA = BWD ? 7 : 4;
-    constexpr int G0 = 3;                            // adjoint: first upstream array
     pdl_wait_then_trigger();
-    const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
+    const int n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
     int item = blockIdx.x;
     const int cb = item % p.ncb; item /= p.ncb;
     const int mb = item % p.nmb;
     const int ab = item / p.nmb;
     const int c4 = cb * blockDim.x + threadIdx.x;
     const int m = mb * blockDim.y + threadIdx.y;
-    const bool valid = c4 < nc4 && m < n1;
     const int c4c = c4 < nc4 ? c4 : 0, mc = m < n1 ? m : 0;   // out-of-range threads shadow (0,0)
     const int col = 4 * c4c;
-    const bool first_col = c4c == 0, last_col = c4c == nc4 - 1;
     const int lane = threadIdx.x & 31;
-    const bool lfetch = lane == 0 && !first_col;
-    const bool rfetch = lane == 31 && !last_col;
-    const int PS = n1 * n2;
-    const int rowoff = mc * n2 + col;
-    const int ymoff = max(mc - 1, 0) * n2 + col;
-    const int ypoff = min(mc + 1, n1 - 1) * n2 + col;
-    // rows of y that carry no residual: upstream arrays count as zero there
-    const bool y_dead = mc < 1 || mc > n1 - 2;
-    const bool ym_dead = mc - 1 < 1, yp_dead = mc + 1 > n1 - 2;
+    Ns3dThread t;
+    t.n0 = p.n0; t.PS = n1 * n2;
+    t.valid = c4 < nc4 && m < n1;
+    t.first_col = c4c == 0; t.last_col = c4c == nc4 - 1;
+    t.lane_first = lane == 0; t.lane_last = lane == 31;
+    // the one float beyond the float4 that the first / last lane of a warp cannot get by shuffle;
+    // at the ends of a z line it stays 0 (zero extension; the velocities' value there is unused)
+    t.efetch = (lane == 0 && !t.first_col) || (lane == 31 && !t.last_col);
+    t.rowoff = mc * n2 + col;
+    t.eoff = t.rowoff + (lane == 0 ? -1 : 4);
+    t.ymoff = max(mc - 1, 0) * n2 + col;
+    t.ypoff = min(mc + 1, n1 - 1) * n2 + col;
+    t.y_dead = mc < 1 || mc > n1 - 2;
+    t.ym_dead = mc - 1 < 1; t.yp_dead = mc + 1 > n1 - 2;
+    // does any thread of this block touch a y row without residuals (its own or a y neighbour)?
+    const int m_lo = mb * blockDim.y, m_hi = m_lo + blockDim.y - 1;
+    const bool y_edge_block = m_lo <= 1 || m_hi >= n1 - 2;
     const int a0 = ab * p.planes_per_item;
-    const int a1 = min(a0 + p.planes_per_item, n0);
-
-    // zero extension of an upstream float4: whole vector when its plane / row is outside the rows,
-    // else the elements at z = 0 and z = n2-1
-    auto mask = [&](V4 v, bool dead) -> V4 {
-        if (dead) v = v4zero();
-        if (first_col) v.lo.x = 0.f;
-        if (last_col) v.hi.y = 0.f;
-        return v;
-    };
-    auto load_own = [&](int k, int r) -> V4 {
-        const int rr = max(0, min(n0 - 1, r));
-        V4 v = ldv4(p.a[k] + rr * PS + rowoff);
-        if (BWD && k >= G0) v = mask(v, y_dead || r < 1 || r > n0 - 2);
-        return v;
-    };
+    const int a1 = min(a0 + p.planes_per_item, p.n0);
+    t.a1 = a1;
 
     V4 A[NA], B[NA], Cc[NA];
 #pragma unroll
-    for (int k = 0; k < NA; ++k) { A[k] = load_own(k, a0 - 1); B[k] = load_own(k, a0); }
+    for (int k = 0; k < NA; ++k) {
+        A[k] = ns3d_load_own<BWD>(p, t, k, a0 - 1, true);
+        B[k] = ns3d_load_own<BWD>(p, t, k, a0, true);
+    }
     float2 acc[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
 
-    // one x step: W0 = plane a-1, W1 = plane a, W2 receives plane a+1
     auto step = [&](int a, const V4 (&W0)[NA], const V4 (&W1)[NA], V4 (&W2)[NA]) {
-        const int pl = a * PS;
-        const bool x_dead = a < 1 || a > n0 - 2;
-        if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= min(a1, n0 - 1)) {
-            const int po = (a + 1 + p.prefetch) * PS + rowoff;
-#pragma unroll
-            for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(p.a[k] + po);
-        }
-        V4 Ym[NA], Yp[NA], Zm[NA], Zp[NA];
-#pragma unroll
-        for (int k = 0; k < NA; ++k) {
-            W2[k] = load_own(k, a + 1);
-            Ym[k] = ldv4(p.a[k] + pl + ymoff);
-            Yp[k] = ldv4(p.a[k] + pl + ypoff);
-            if (BWD && k >= G0) { Ym[k] = mask(Ym[k], x_dead || ym_dead); Yp[k] = mask(Yp[k], x_dead || yp_dead); }
-            float l1 = __shfl_up_sync(FULL_MASK, W1[k].hi.y, 1);
-            float r1 = __shfl_down_sync(FULL_MASK, W1[k].lo.x, 1);
-            const bool dead = BWD && k >= G0 && (x_dead || y_dead);
-            if (lfetch) l1 = dead ? 0.f : __ldg(p.a[k] + pl + rowoff - 1);
-            if (rfetch) r1 = dead ? 0.f : __ldg(p.a[k] + pl + rowoff + 4);
-            if (BWD && k >= G0) { if (first_col) l1 = 0.f; if (last_col) r1 = 0.f; }
-            Zm[k] = shift_left(W1[k], l1);
-            Zp[k] = shift_right(W1[k], r1);
-        }
-        float2 o[4][2];
-        const float2 nodt[3] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float2 w0[NA], w1[NA], w2[NA], ym[NA], yp[NA], zm[NA], zp[NA], oo[4];
-            v4_half<NA>(W0, h, w0); v4_half<NA>(W1, h, w1); v4_half<NA>(W2, h, w2);
-            v4_half<NA>(Ym, h, ym); v4_half<NA>(Yp, h, yp); v4_half<NA>(Zm, h, zm); v4_half<NA>(Zp, h, zp);
-            if constexpr (BWD) ns_bwd_pair(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
-            else ns_fwd_pair(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) o[e][h] = oo[e];
-        }
-        if (!BWD) {                                  // the outer shell carries no row
-            const bool rowless = x_dead || y_dead;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                if (rowless) { o[e][0] = make_float2(0.f, 0.f); o[e][1] = o[e][0]; }
-                if (first_col) o[e][0].x = 0.f;
-                if (last_col) o[e][1].y = 0.f;
-            }
-        }
-        if (valid) {
-            const int off = pl + rowoff;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                stv4(p.out[e] + off, o[e][0], o[e][1]);
-                if (!BWD) acc[e] = fma2(o[e][0], o[e][0], fma2(o[e][1], o[e][1], acc[e]));
-            }
-        }
+        if (y_edge_block || a <= 1 || a >= p.n0 - 2) ns3d_step<BWD, true, NA>(p, t, a, W0, W1, W2, acc);
+        else ns3d_step<BWD, false, NA>(p, t, a, W0, W1, W2, acc);
     };
-
     for (int a = a0; a < a1; a += 3) {
         step(a, A, B, Cc);
         if (a + 1 < a1) step(a + 1, B, Cc, A);
@@ -168,9 +210,9 @@ static int env_int(const char* name, int dflt) {
 
 static void ns3d_geometry(const int* n, Ns3dParams& p, dim3& block) {
     p.n0 = n[0]; p.n1 = n[1]; p.n2 = n[2]; p.nc4 = n[2] / 4;
-    int tx = env_int("FPDE_NS3D_TX", 32);
+    int tx = env_int("FPDE_NS3D_TX", p.nc4 % 64 == 0 ? 64 : 32);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
-    int ty = env_int("FPDE_NS3D_TY", 4);
+    int ty = env_int("FPDE_NS3D_TY", 128 / tx);
     ty = std::max(1, std::min(128 / tx, ty));
     block = dim3(tx, ty, 1);
     p.planes_per_item = env_int("FPDE_NS3D_PLANES", 16);
@@ -178,7 +220,7 @@ static void ns3d_geometry(const int* n, Ns3dParams& p, dim3& block) {
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     const char* pf = std::getenv("FPDE_NS3D_PREFETCH");
-    p.prefetch = pf && *pf ? std::atoi(pf) : 3;
+    p.prefetch = pf && *pf ? std::atoi(pf) : 1;
     if (p.prefetch < 0 || p.prefetch >= p.n0) p.prefetch = 0;
 }
 
