@@ -86,8 +86,11 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     };
     auto pclamp = [&](int a) -> int { return EDGE ? max(0, min(n0 - 1, a)) * PS : a * PS; };
     auto pdead = [&](int a) -> bool { return ROWMASK && (a < 2 || a > n0 - 3); };
-    const bool lfetch = lane == 0 && c4 > 0 && c4 < nc4;
-    const bool rfetch = lane == 31 && c4 < nc4 - 1;
+    // The two floats beyond the float4 that the first / last lane of a warp cannot get by shuffle:
+    // one predicated 8-byte load, issued with the other loads of the step (a load inside a
+    // divergent branch would be waited for on its own).  At the ends of a z line it stays 0.
+    const bool efetch = (lane == 0 && c4 > 0 && c4 < nc4) || (lane == 31 && c4 < nc4 - 1);
+    const int eoff = lane == 0 ? -2 : 4;
 
     V4 Q0 = load_h(p_c, pclamp(a0 - 2), d0 || pdead(a0 - 2), true), Q1 = load_h(p_c, pclamp(a0 - 1), d0 || pdead(a0 - 1), true);
     V4 Q2 = load_h(p_c, pclamp(a0), d0 || pdead(a0), true), Q3 = load_h(p_c, pclamp(a0 + 1), d0 || pdead(a0 + 1), true), Q4;
@@ -106,17 +109,15 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
         const V4 a2v = load_h(p_m2, pl, dm2 || pd, false), b2v = load_h(p_p2, pl, dp2 || pd, false);
         V4 src = v4zero();
         if (FWD) src = ldv4(p.cin + pl + o_c);
-        // z neighbours from the adjacent lanes; the outer lanes of a warp fetch theirs
+        float2 E = make_float2(0.f, 0.f);
+        if (efetch) E = __ldg(reinterpret_cast<const float2*>(p_c + pl + eoff));
+        if (ROWMASK && (d0 || pd)) E = make_float2(0.f, 0.f);
+        // z neighbours from the adjacent lanes; the outer lanes of a warp take the fetched pair
         float l1 = __shfl_up_sync(FULL_MASK, q2.hi.y, 1), l2 = __shfl_up_sync(FULL_MASK, q2.hi.x, 1);
         float r1 = __shfl_down_sync(FULL_MASK, q2.lo.x, 1), r2 = __shfl_down_sync(FULL_MASK, q2.lo.y, 1);
-        {
-            const float* rp = p_c + pl;
-            if (lfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp - 2)); l2 = t.x; l1 = t.y; }
-            if (rfetch) { const float2 t = __ldg(reinterpret_cast<const float2*>(rp + 4)); r1 = t.x; r2 = t.y; }
-            const bool dead = ROWMASK && (d0 || pd);
-            if (dead || first_col) { l1 = 0.f; l2 = 0.f; }
-            if (dead || last_col) { r1 = 0.f; r2 = 0.f; }
-        }
+        if (lane == 0) { l2 = E.x; l1 = E.y; }
+        if (lane == 31) { r1 = E.x; r2 = E.y; }
+        if (MASK_IN && last_col) { r1 = 0.f; r2 = 0.f; }   // a ragged row ends inside a warp
         const V4 s1x = v4add(q1, q3), s2x = v4add(q0, q4);
         const V4 s1y = v4add(a1v, b1v), s2y = v4add(a2v, b2v);
         V4 s1z, s2z;

@@ -51,8 +51,11 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
     const bool first_col = c4 == 0, last_col = c4 == nc4 - 1;
     const int a0 = rc * p.rows_per_item;
     const int a1 = min(a0 + p.rows_per_item, n0);
-    const bool lfetch = cvalid && lane == 0 && !first_col;
-    const bool rfetch = cvalid && lane == 31 && !last_col;
+    // The one float beyond the float4 that the first / last lane of a warp cannot get by shuffle:
+    // one predicated load per array, issued with the other loads of the row (a load inside a
+    // divergent branch would be waited for on its own).  At the ends of a row it stays 0.
+    const bool efetch = cvalid && ((lane == 0 && !first_col) || (lane == 31 && !last_col));
+    const int eoff = col + (lane == 0 ? -1 : 4);
 
     // array k at row r (clamped into the grid).  Upstream arrays (adjoint, k >= 2) are scaled and
     // read as zero outside the rows of the operator.
@@ -77,18 +80,24 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
 
     for (int row = a0; row < a1; ++row) {
         V4 L[NA], R[NA];
+        float E[NA];
 #pragma unroll
         for (int k = 0; k < NA; ++k) {
             nxt[k] = load(k, row + 1);
+            E[k] = 0.f;
+            if (efetch) E[k] = __ldg(p.in[k] + row * n1 + eoff);
+        }
+#pragma unroll
+        for (int k = 0; k < NA; ++k) {
+            if (BWD && k >= 2) {
+                E[k] *= p.gs[k - 2].x;
+                if (row < 1 || row > n0 - 2) E[k] = 0.f;
+            }
             float l1 = __shfl_up_sync(FULL_MASK, cur[k].hi.y, 1);
             float r1 = __shfl_down_sync(FULL_MASK, cur[k].lo.x, 1);
-            const float* rp = p.in[k] + row * n1 + col;
-            const bool dead = BWD && k >= 2 && (row < 1 || row > n0 - 2);
-            const float s = (BWD && k >= 2) ? p.gs[k - 2].x : 1.f;
-            if (lfetch) l1 = dead ? 0.f : s * __ldg(rp - 1);
-            if (rfetch) r1 = dead ? 0.f : s * __ldg(rp + 4);
-            if (first_col) l1 = 0.f;
-            if (last_col) r1 = 0.f;
+            if (lane == 0) l1 = E[k];
+            if (lane == 31) r1 = E[k];
+            if (last_col) r1 = 0.f;                   // a ragged row ends inside a warp
             L[k] = shift_left(cur[k], l1);
             R[k] = shift_right(cur[k], r1);
         }

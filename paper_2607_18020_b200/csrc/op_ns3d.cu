@@ -106,6 +106,8 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
         float r1 = __shfl_down_sync(FULL_MASK, W1[k].lo.x, 1);
         if (t.lane_first) l1 = E[k];
         if (t.lane_last) r1 = E[k];
+        // (a z line that ends inside a warp: the lane after it shadows column 0, whose upstream
+        // lo.x is zero-extended, so r1 of the last column is 0 there as well)
         Zm[k] = shift_left(W1[k], l1);
         Zp[k] = shift_right(W1[k], r1);
     }
