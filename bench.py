@@ -232,6 +232,7 @@ class DeviceProblem:
         self.loss = torch.zeros(ne + 1, dtype=torch.float64, device="cuda")
         self.ws = torch.empty(B.workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
         self.gscale = [2.0 / B.row_count(w.op, w.shape)] * ne
+        self.ws2 = None
 
     def fwd(self):
         w = self.w
@@ -240,6 +241,14 @@ class DeviceProblem:
     def bwd(self):
         w = self.w
         self.B.fpde_bwd(w.op, self.fields, self.res, self.gscale, self.grads, w.shape, w.spacing, w.coeffs, w.bc)
+
+    def fwd_bwd(self):
+        """The loss-specialised pass: loss + dL/dfield, residual arrays not stored."""
+        w = self.w
+        if self.ws2 is None:
+            self.ws2 = self.torch.empty(self.B.fwd_bwd_workspace_bytes(w.op, w.shape), dtype=self.torch.uint8, device="cuda")
+        self.B.fpde_fwd_bwd(w.op, self.fields, self.sources, None, self.grads, self.loss, w.shape, w.spacing,
+                            w.coeffs, w.bc, self.ws2)
 
 
 def timed_steps(torch, prob, steps, warmup, barrier, flush=None, inner_events=False):
@@ -328,6 +337,34 @@ def graph_points_per_s(torch, prob, N, pairs, replays):
         return None
 
 
+def single_pass_figures(torch, prob, steps, warmup, flush, peak):
+    """fpde_fwd_bwd (one kernel: residuals stay in registers, loss and gradients come out): cold
+    per-call median and a warm back-to-back figure.  Algorithmic bytes: every field and source
+    read once, every gradient written once."""
+    w = prob.w
+    N = w.npoints
+    bpp = 4 * (2 * len(w.fields) + len(w.sources))
+    for _ in range(warmup):
+        prob.fwd_bwd()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+    torch.cuda.synchronize()
+    for k in range(steps):
+        flush.fill_(k)
+        ev[k][0].record(); prob.fwd_bwd(); ev[k][1].record()
+    torch.cuda.synchronize()
+    ms = statistics.median(e[0].elapsed_time(e[1]) for e in ev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        prob.fwd_bwd()
+    e1.record(); torch.cuda.synchronize()
+    warm_ms = e0.elapsed_time(e1) / steps
+    gbs = bpp * N / (ms * 1e-3) / 1e9
+    return {"ms": ms, "points_per_s": N / (ms * 1e-3), "warm_points_per_s": N / (warm_ms * 1e-3),
+            "algorithmic_bytes_per_point": bpp, "gbs": gbs, "frac": gbs / peak,
+            "what": "fpde_fwd_bwd, residual arrays not stored; launches: 1 kernel + loss finalise"}
+
+
 def config_line(torch, B, name, steps, warmup, peak):
     """Secondary figures for one configuration: per-call medians with an L2 flush (a 256 MiB
     write) before every step, so small grids are measured cold like large ones."""
@@ -350,6 +387,8 @@ def config_line(torch, B, name, steps, warmup, peak):
     out["warm_points_per_s"] = N * steps / (total_ms * 1e-3)
     out["l2_resident"] = bool((fb + bb) * N < (100 << 20))
     out["graph_points_per_s"] = graph_points_per_s(torch, prob, N, pairs=10, replays=max(3, steps // 10))
+    if B.has_single_pass(w.op):
+        out["single_pass"] = single_pass_figures(torch, prob, steps, warmup, flush, peak)
     del prob, flush
     torch.cuda.empty_cache()
     return out

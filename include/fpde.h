@@ -181,6 +181,43 @@ int fpde_bwd(int op,
              void* stream);
 
 /*
+ * Loss-specialised single pass: residuals (Section 2.1), the mean-square loss and its gradient
+ * through the discrete adjoint (Sections 2.2, 2.3) from one call,
+ *   L = sum_e L_e,  L_e = (1/N_r) sum over rows r_e^2,   gfields[f] = dL/dfield_f
+ * i.e. what fpde_fwd followed by fpde_bwd with gres = residuals, gscale[e] = 2/N_r computes.
+ * Where fpde_has_single_pass(op) is 1 this is ONE kernel in which the residuals stay in
+ * registers between the forward stencil and the adjoint (the upstream array of the adjoint is
+ * (2/N_r) r, so nothing else of the forward pass is needed): it reads the fields and sources
+ * and writes the gradients, and the residual arrays only if asked for.  For the other
+ * operators it queues the forward kernel, the loss sum and the adjoint kernel.
+ *
+ *   fields, sources, ndim ... bc, stream   as in fpde_fwd
+ *   residuals  host array of nresiduals device pointers, or NULL.  Single-pass operators: a
+ *              NULL array or NULL entries mean "do not store that residual"; a non-NULL entry
+ *              is overwritten as by fpde_fwd.  Other operators: every entry is required
+ *              (FPDE_ERR_NULL otherwise), the arrays serve as the intermediate.
+ *   gfields    host array of nfields device pointers, overwritten at every node
+ *   loss_out   device, nresiduals+1 doubles (as in fpde_fwd), or NULL to skip the loss
+ *   workspace  device scratch of at least fpde_fwd_bwd_workspace_bytes() bytes (needed only
+ *              when loss_out is given)
+ * Same status codes as fpde_fwd / fpde_bwd.
+ */
+int fpde_has_single_pass(int op);
+size_t fpde_fwd_bwd_workspace_bytes(int op, int ndim, const int64_t* shape);
+int fpde_fwd_bwd(int op,
+                 const float* const* fields,
+                 const float* const* sources,
+                 float* const* residuals,
+                 float* const* gfields,
+                 double* loss_out,
+                 int ndim, const int64_t* shape,
+                 const double* spacing,
+                 const double* coeffs, int ncoeffs,
+                 const int* bc,
+                 void* workspace, size_t workspace_bytes,
+                 void* stream);
+
+/*
  * Loss gradient from HOST buffers in one call: copies the fields (and sources) to the device,
  * runs fpde_fwd, then fpde_bwd with the upstream sensitivities of the mean-square loss,
  * G_e = (2/N_r) r_e (Section 2.2: the operator receives G = dL/dres from the loss), and copies

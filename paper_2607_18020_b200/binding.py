@@ -65,6 +65,15 @@ def lib():
                                ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fpde_has_single_pass.restype = ctypes.c_int
+        L.fpde_has_single_pass.argtypes = [ctypes.c_int]
+        L.fpde_fwd_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.fpde_fwd_bwd_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_fwd_bwd.restype = ctypes.c_int
+        L.fpde_fwd_bwd.argtypes = [ctypes.c_int, vpp, vpp, vpp, vpp, ctypes.c_void_p, ctypes.c_int,
+                                   ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                   ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                                   ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         L.fpde_host_arena_bytes.restype = ctypes.c_size_t
         L.fpde_host_arena_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
         L.fpde_loss_grad_host.restype = ctypes.c_int
@@ -172,6 +181,32 @@ def bwd_status(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, wo
                           int(workspace_bytes_), stream)
 
 
+def has_single_pass(op) -> bool:
+    return bool(lib().fpde_has_single_pass(_opid(op)))
+
+
+def fwd_bwd_workspace_bytes(op, shape) -> int:
+    return int(lib().fpde_fwd_bwd_workspace_bytes(_opid(op), len(shape), _i64(shape)))
+
+
+def fwd_bwd_status(op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc, workspace,
+                   workspace_bytes_, stream, ndim=None, ncoeffs=None) -> int:
+    return lib().fpde_fwd_bwd(_opid(op),
+                              _ptr_array(_dev_ptrs(fields)) if fields is not None else None,
+                              _ptr_array(_dev_ptrs(sources)) if sources is not None else None,
+                              _ptr_array(_dev_ptrs(residuals)) if residuals is not None else None,
+                              _ptr_array(_dev_ptrs(gfields)) if gfields is not None else None,
+                              _dev_ptrs([loss_out])[0] if loss_out is not None else None,
+                              len(shape) if ndim is None else ndim,
+                              _i64(shape) if shape is not None else None,
+                              _f64(spacing) if spacing is not None else None,
+                              _f64(coeffs) if coeffs is not None else None,
+                              len(coeffs) if ncoeffs is None else ncoeffs,
+                              _bcs(bc) if bc is not None else None,
+                              _dev_ptrs([workspace])[0] if workspace is not None else None,
+                              int(workspace_bytes_), stream)
+
+
 def _stream_handle(stream) -> Optional[int]:
     if stream is None:
         import torch
@@ -192,6 +227,20 @@ def fpde_fwd(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, b
                     _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd")
+
+
+def fpde_fwd_bwd(op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc, workspace,
+                 stream=None):
+    """Queue the loss-specialised pass: loss and dL/dfield (and the residual arrays, where given).
+
+    residuals: None, or a sequence with None entries for residual arrays that need not be stored
+    (only where has_single_pass(op); the other operators need all of them).  workspace: a CUDA
+    tensor of at least fwd_bwd_workspace_bytes(op, shape) bytes."""
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    st = fwd_bwd_status(op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc, workspace,
+                        wsb, _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_fwd_bwd")
 
 
 def fpde_bwd(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace=None, stream=None):

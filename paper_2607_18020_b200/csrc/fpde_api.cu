@@ -291,6 +291,77 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
     return ce == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
 }
 
+int fpde_has_single_pass(int op) {
+    return (op >= 0 && op < FPDE_OP_COUNT && fused2d_supported(op)) ? 1 : 0;
+}
+
+size_t fpde_fwd_bwd_workspace_bytes(int op, int ndim, const int64_t* shape) {
+    int n[MAX_D] = {0, 0, 0, 0};
+    if (check_shape(op, ndim, shape, n, nullptr, nullptr) != FPDE_OK) return 0;
+    if (!fused2d_supported(op)) return fpde_workspace_bytes(op, ndim, shape);
+    const size_t need = (size_t)fused2d_items(n) * REGISTRY[op].ne * sizeof(float);
+    return ((need + 255) / 256) * 256 + 4096;
+}
+
+int fpde_fwd_bwd(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+                 float* const* gfields, double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+                 const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+                 void* stream) {
+    Problem q;
+    std::memset(&q, 0, sizeof(q));
+    int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!gfields) return FPDE_ERR_NULL;
+    if (!fused2d_supported(op)) {
+        // two kernels with the residual arrays as the intermediate
+        if (!residuals) return FPDE_ERR_NULL;
+        for (int f = 0; f < e.nf; ++f) {
+            if (!gfields[f]) return FPDE_ERR_NULL;
+            if (!aligned16(gfields[f])) return FPDE_ERR_ALIGN;
+        }
+        st = fpde_fwd(op, fields, sources, residuals, loss_out, ndim, shape, spacing, coeffs, ncoeffs, bc, workspace,
+                      workspace_bytes, stream);
+        if (st != FPDE_OK) return st;
+        double gscale[MAX_F];
+        for (int r = 0; r < e.ne; ++r) gscale[r] = 2.0 / (double)q.rows;
+        return fpde_bwd(op, fields, residuals, gscale, gfields, ndim, shape, spacing, coeffs, ncoeffs, bc, nullptr, 0,
+                        stream);
+    }
+    if (e.ns > 0 && !sources) return FPDE_ERR_NULL;
+    for (int s = 0; s < e.ns; ++s) {
+        if (!sources[s]) return FPDE_ERR_NULL;
+        if (!aligned16(sources[s])) return FPDE_ERR_ALIGN;
+        q.aux[s] = sources[s];
+    }
+    float* res[MAX_F] = {nullptr, nullptr, nullptr, nullptr};
+    for (int r = 0; r < e.ne; ++r) {
+        res[r] = residuals ? residuals[r] : nullptr;
+        if (res[r] && !aligned16(res[r])) return FPDE_ERR_ALIGN;
+    }
+    for (int f = 0; f < e.nf; ++f) {
+        if (!gfields[f]) return FPDE_ERR_NULL;
+        if (!aligned16(gfields[f])) return FPDE_ERR_ALIGN;
+        q.out[f] = gfields[f];
+    }
+    const int items = fused2d_items(q.n);
+    if (loss_out) {
+        if (!aligned16(loss_out)) return FPDE_ERR_ALIGN;
+        if (!workspace || !aligned16(workspace) || workspace_bytes < (size_t)items * e.ne * sizeof(float))
+            return FPDE_ERR_WORKSPACE;
+        q.partials = static_cast<float*>(workspace);
+        q.loss_out = loss_out;
+    }
+    q.stream = static_cast<cudaStream_t>(stream);
+    cudaError_t ce = launch_fused2d(q, res);
+    if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+    if (loss_out) {
+        ce = launch_loss_finalize(q.partials, items, e.ne, q.rows, loss_out, q.stream);
+        if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+    }
+    return FPDE_OK;
+}
+
 static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 
 size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape) {

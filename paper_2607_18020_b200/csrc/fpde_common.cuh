@@ -69,6 +69,13 @@ __device__ __forceinline__ V4 v4fma(V4 a, float2 s, V4 c) { V4 r; r.lo = fma2(a.
 // a * b + c
 __device__ __forceinline__ V4 v4fmav(V4 a, V4 b, V4 c) { V4 r; r.lo = fma2(a.lo, b.lo, c.lo); r.hi = fma2(a.hi, b.hi, c.hi); return r; }
 
+// half h (0: lo, 1: hi) of each float4 of an array
+template <int NA>
+__device__ __forceinline__ void v4_half(const V4 (&A)[NA], int h, float2 (&out)[NA]) {
+#pragma unroll
+    for (int i = 0; i < NA; ++i) out[i] = h == 0 ? A[i].lo : A[i].hi;
+}
+
 // a float4 shifted by one element to the left / right along the row
 __device__ __forceinline__ V4 shift_left(const V4& c, float l1) {    // value at column j-1
     V4 r; r.lo = make_float2(l1, c.lo.x); r.hi = make_float2(c.lo.y, c.hi.x); return r;

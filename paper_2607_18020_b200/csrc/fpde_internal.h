@@ -71,6 +71,10 @@ int ns_tma_items(const int* n);
 cudaError_t launch_ns_fwd_tma(const Problem& p, bool& launched);
 cudaError_t launch_ns_bwd_tma(const Problem& p, bool& launched);
 unsigned int ns_tma_timeouts();
+// single-pass residual + loss + gradient (op_fused2d.cu); `res` entries may be NULL
+bool fused2d_supported(int op);
+int fused2d_items(const int* n);
+cudaError_t launch_fused2d(const Problem& p, float* const* res);
 cudaError_t launch_ns_bwd(const Problem& p);
 
 // Final, fixed-order fp64 sum of the per-item partials: loss_out[e] = sum/N_r, loss_out[E] = total.

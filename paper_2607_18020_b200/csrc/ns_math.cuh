@@ -120,12 +120,6 @@ __device__ __forceinline__ void ns_bwd_pair(const NsConsts& k, const float2 (&w0
 
 // ---- a float4 (four consecutive t) per thread: two pairs -------------------------------------
 // l1/r1: t-1 of lane x and t+1 of lane w for u,v,w (forward) / the momentum upstream arrays.
-template <int NA>
-__device__ __forceinline__ void v4_half(const V4 (&A)[NA], int h, float2 (&out)[NA]) {
-#pragma unroll
-    for (int i = 0; i < NA; ++i) out[i] = h == 0 ? A[i].lo : A[i].hi;
-}
-
 __device__ __forceinline__ void ns_fwd_math(const NsConsts& k, const V4 (&W0)[4], const V4 (&W1)[4], const V4 (&W2)[4],
                                             const V4 (&Ym)[4], const V4 (&Yp)[4], const V4 (&Zm)[4], const V4 (&Zp)[4],
                                             const float (&l1)[3], const float (&r1)[3], bool t_first, bool t_last,
