@@ -299,7 +299,7 @@ size_t fpde_fwd_bwd_workspace_bytes(int op, int ndim, const int64_t* shape) {
     int n[MAX_D] = {0, 0, 0, 0};
     if (check_shape(op, ndim, shape, n, nullptr, nullptr) != FPDE_OK) return 0;
     if (!fused2d_supported(op)) return fpde_workspace_bytes(op, ndim, shape);
-    const size_t need = (size_t)fused2d_items(n) * REGISTRY[op].ne * sizeof(float);
+    const size_t need = (size_t)fused2d_max_items(n) * REGISTRY[op].ne * sizeof(float);
     return ((need + 255) / 256) * 256 + 4096;
 }
 
@@ -344,7 +344,7 @@ int fpde_fwd_bwd(int op, const float* const* fields, const float* const* sources
         if (!aligned16(gfields[f])) return FPDE_ERR_ALIGN;
         q.out[f] = gfields[f];
     }
-    const int items = fused2d_items(q.n);
+    const int items = fused2d_items(op, q.n);
     if (loss_out) {
         if (!aligned16(loss_out)) return FPDE_ERR_ALIGN;
         if (!workspace || !aligned16(workspace) || workspace_bytes < (size_t)items * e.ne * sizeof(float))

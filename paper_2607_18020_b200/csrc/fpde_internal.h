@@ -73,7 +73,8 @@ cudaError_t launch_ns_bwd_tma(const Problem& p, bool& launched);
 unsigned int ns_tma_timeouts();
 // single-pass residual + loss + gradient (op_fused2d.cu); `res` entries may be NULL
 bool fused2d_supported(int op);
-int fused2d_items(const int* n);
+int fused2d_items(int op, const int* n);
+int fused2d_max_items(const int* n);
 cudaError_t launch_fused2d(const Problem& p, float* const* res);
 cudaError_t launch_ns_bwd(const Problem& p);
 

@@ -37,6 +37,7 @@ struct Fused2dParams {
     int n0, n1, nc4;
     int rows_per_item, ncg, ncb, nitems;
     float* partials;
+    int prefetch;           // rows ahead of the newest requested row to pull into L2 (0 = off)
 };
 
 constexpr int FUSED2D_OWN = 30;     // float4 columns a warp owns (lanes 1..30)
@@ -233,6 +234,13 @@ __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams 
                     V4 (&Fnew)[NF], const V4 (&Sp)[NSA], V4 (&Snew)[NSA], const V4 (&Rm)[NE], const V4 (&R0)[NE],
                     V4 (&Rp)[NE]) {
         if (i + 1 < a1) load_row(i + 3, Fnew, Snew);
+        if (p.prefetch > 0 && (lane & 7) == 0 && i + 3 + p.prefetch <= a1 + 1) {
+            const int off = row_of(i + 3 + p.prefetch) * n1 + col;
+#pragma unroll
+            for (int k = 0; k < NF; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.f[k] + off));
+#pragma unroll
+            for (int k = 0; k < NS; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.src[k] + off));
+        }
         residual_row(i + 1, F0, Fp, Fpp, Sp, Rp);
         V4 RL[NE], RR[NE], FL[NF], FR[NF];
 #pragma unroll
@@ -295,29 +303,60 @@ bool fused2d_supported(int op) {
     return op == 1 || op == 2 || op == 5;            // Poisson 2-D, Gray-Scott, steady 2-D Navier-Stokes
 }
 
-static void fused2d_geometry(const int* n, Fused2dParams& p) {
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else n = 148;
+    }
+    return n;
+}
+
+static int fused2d_blocks_per_sm(int op) { return op == 1 ? 4 : (op == 2 ? 3 : 2); }
+
+// Rows per work item: every item recomputes r on two extra rows, and the last wave of items
+// should be nearly full; pick the row count with the smallest (waves x rows marched per item).
+static void fused2d_geometry(int op, const int* n, Fused2dParams& p) {
     p.n0 = n[0]; p.n1 = n[1]; p.nc4 = n[1] / 4;
     p.ncg = (p.nc4 + FUSED2D_OWN - 1) / FUSED2D_OWN;
     p.ncb = (p.ncg + 3) / 4;
     int rows = env_int("FPDE_FUSED2D_ROWS", 0);
-    if (rows == 0) {                                 // enough items to fill the machine a few times over
-        rows = 32;
-        while (rows > 4 && (long)p.ncb * ((p.n0 + rows - 1) / rows) < 1184) rows /= 2;
+    if (rows > 0 && rows < 4) rows = 4;
+    if (rows == 0) {
+        const long slots = (long)sm_count() * fused2d_blocks_per_sm(op);
+        long best = -1;
+        for (int r = 4; r <= 96; ++r) {
+            const long items = (long)p.ncb * ((p.n0 + r - 1) / r);
+            const long cost = ((items + slots - 1) / slots) * (r + 4);
+            if (best < 0 || cost < best) { best = cost; rows = r; }
+        }
     }
     p.rows_per_item = rows;
+    const char* pf = std::getenv("FPDE_FUSED2D_PREFETCH");
+    p.prefetch = pf && *pf ? std::atoi(pf) : 2;
+    if (p.prefetch < 0) p.prefetch = 0;
     p.nitems = p.ncb * ((p.n0 + rows - 1) / rows);
 }
 
-int fused2d_items(const int* n) {
+// upper bound of the item count over every row count the geometry can choose (>= 4 rows per
+// item), for workspace sizing that does not depend on the device the query runs on
+int fused2d_max_items(const int* n) {
+    const int nc4 = n[1] / 4, ncg = (nc4 + FUSED2D_OWN - 1) / FUSED2D_OWN, ncb = (ncg + 3) / 4;
+    return ncb * ((n[0] + 3) / 4);
+}
+
+int fused2d_items(int op, const int* n) {
     Fused2dParams p{};
-    fused2d_geometry(n, p);
+    fused2d_geometry(op, n, p);
     return p.nitems;
 }
 
 // q.in = fields, q.aux = sources, q.out = dL/dfield; `res` = residual arrays (entries may be NULL)
 cudaError_t launch_fused2d(const Problem& q, float* const* res) {
     Fused2dParams p{};
-    fused2d_geometry(q.n, p);
+    fused2d_geometry(q.op, q.n, p);
     p.partials = q.partials;
     p.gs = sp(2.0 / (double)q.rows);
     const double h0 = q.h[0], h1 = q.h[1];
