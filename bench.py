@@ -418,6 +418,9 @@ def main():
     ap.add_argument("--impl", default="fpde", choices=["fpde", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip per-config figures and the CPU baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--single-pass", action="store_true",
+                    help="time fpde_fwd_bwd (one kernel: loss + gradient, residual arrays not stored) as the step; "
+                         "only for operators that have a single-pass kernel")
     ap.add_argument("--shape", default=None, help="override the grid extents, e.g. 64,128,128,16 (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "fpde" else args.warmup
@@ -449,6 +452,10 @@ def main():
     w = W.make(args.workload, seed=42 + rank, shape=shape,
                spacing=_spacing_of(args.workload) if shape else None)
     prob = DeviceProblem(torch, B, w)
+    if args.single_pass:
+        if not B.has_single_pass(w.op):
+            raise SystemExit("--single-pass: operator %s has no single-pass kernel" % w.op)
+        prob.fwd, prob.bwd = prob.fwd_bwd, (lambda: None)
     N = w.npoints
 
     sampler = ClockSampler(torch, local_rank)
@@ -469,17 +476,23 @@ def main():
     e2e_value = job_value(world, N, e2e_k, e2e_ms)
 
     fb, bb = ALGO_BYTES[w.op]
+    knames = KERNEL_NAMES[w.op]
     f_avg, b_avg = sum(fwd_ms) / len(fwd_ms), sum(bwd_ms) / len(bwd_ms)
+    if args.single_pass:        # every field and source read once, every gradient written once
+        fb, bb = 4 * (2 * len(w.fields) + len(w.sources)), 0
+        knames = ("fused2d_kernel<%s>" % w.op, "-")
+        b_avg = 0.0
     dom = 1 if b_avg >= f_avg else 0
     dom_bytes = (fb, bb)[dom] * N
     dom_ms = (f_avg, b_avg)[dom]
-    dom_name = KERNEL_NAMES[w.op][dom]
+    dom_name = knames[dom]
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom_name)),
                 "algorithmic_bytes": dom_bytes, "avg_ms": dom_ms,
-                "other_kernel": {"kernel": KERNEL_NAMES[w.op][1 - dom], "avg_ms": (f_avg, b_avg)[1 - dom],
+                "other_kernel": None if args.single_pass else
+                                {"kernel": knames[1 - dom], "avg_ms": (f_avg, b_avg)[1 - dom],
                                  "note": "forward figure includes the one-block loss finalise launch",
                                  "achieved": (fb, bb)[1 - dom] * N / ((f_avg, b_avg)[1 - dom] * 1e-3) / 1e9},
                 "pair_achieved": (fb + bb) * N * args.steps / (total_ms * 1e-3) / 1e9,
@@ -490,14 +503,15 @@ def main():
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "operator": w.op, "shape": list(w.shape), "points": N,
-                   "fields": len(w.fields), "parallelism": "replicas x%d (no exchange step)" % world,
+                   "fields": len(w.fields), "step": "fpde_fwd_bwd (single pass)" if args.single_pass else "fpde_fwd + fpde_bwd",
+                   "parallelism": "replicas x%d (no exchange step)" % world,
                    "l2": "per-step traffic %.0f MB >> L2, no flush needed" % ((fb + bb) * N / 1e6)
                          if (fb + bb) * N > (256 << 20) else "working set fits L2: warm-cache number"},
         "clocks": sampler.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_k, "ms_per_step": e2e_ms / e2e_k,
                 "what": "fpde_loss_grad_host from pinned host buffers: H2D fields, fwd, bwd, D2H gradients + loss, sync"},
-        "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        "gpu_launches": (2 if args.single_pass else LAUNCHES_PER_STEP) * args.steps,
         "roofline": roofline,
         "loss": float(prob.loss[-1].item()),
     }

@@ -219,7 +219,7 @@ int fpde_fwd_bwd(int op,
 
 /*
  * Loss gradient from HOST buffers in one call: copies the fields (and sources) to the device,
- * runs fpde_fwd, then fpde_bwd with the upstream sensitivities of the mean-square loss,
+ * runs fpde_fwd_bwd, i.e. the adjoint with the upstream sensitivities of the mean-square loss,
  * G_e = (2/N_r) r_e (Section 2.2: the operator receives G = dL/dres from the loss), and copies
  * dL/dfield and the loss vector back.  Everything is queued on `stream`; the host buffers may be
  * read / written until the stream has been synchronised (use page-locked memory for the copies to

@@ -370,7 +370,7 @@ size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape) {
     const OpEntry& e = REGISTRY[op];
     const size_t arr = round256((size_t)N * sizeof(float));
     return arr * (size_t)(2 * e.nf + e.ns + e.ne) + round256((e.ne + 1) * sizeof(double))
-         + fpde_workspace_bytes(op, ndim, shape);
+         + fpde_fwd_bwd_workspace_bytes(op, ndim, shape);
 }
 
 int fpde_loss_grad_host(int op, const float* const* h_fields, const float* const* h_sources,
@@ -404,17 +404,16 @@ int fpde_loss_grad_host(int op, const float* const* h_fields, const float* const
     for (int f = 0; f < e.nf; ++f) { d_g[f] = reinterpret_cast<float*>(base); base += arr; }
     double* d_loss = reinterpret_cast<double*>(base); base += round256((e.ne + 1) * sizeof(double));
     void* d_ws = base;
-    const size_t ws_bytes = fpde_workspace_bytes(op, ndim, shape);
+    const size_t ws_bytes = fpde_fwd_bwd_workspace_bytes(op, ndim, shape);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     for (int f = 0; f < e.nf; ++f)
         if (cudaMemcpyAsync(d_f[f], h_fields[f], bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FPDE_ERR_CUDA;
     for (int s = 0; s < e.ns; ++s)
         if (cudaMemcpyAsync(d_s[s], h_sources[s], bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FPDE_ERR_CUDA;
-    st = fpde_fwd(op, d_f, d_s, d_r, d_loss, ndim, shape, spacing, coeffs, ncoeffs, bc, d_ws, ws_bytes, stream);
-    if (st != FPDE_OK) return st;
-    double gscale[MAX_F];
-    for (int r = 0; r < e.ne; ++r) gscale[r] = 2.0 / (double)rows;
-    st = fpde_bwd(op, d_f, d_r, gscale, d_g, ndim, shape, spacing, coeffs, ncoeffs, bc, nullptr, 0, stream);
+    // one kernel where the operator has a single-pass kernel (the staged residual arrays are
+    // then not written), forward + adjoint through them otherwise
+    st = fpde_fwd_bwd(op, d_f, d_s, fused2d_supported(op) ? nullptr : d_r, d_g, d_loss, ndim, shape, spacing, coeffs,
+                      ncoeffs, bc, d_ws, ws_bytes, stream);
     if (st != FPDE_OK) return st;
     for (int f = 0; f < e.nf; ++f)
         if (cudaMemcpyAsync(h_gfields[f], d_g[f], bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return FPDE_ERR_CUDA;
