@@ -68,6 +68,10 @@ NCU_TRAFFIC_BYTES = {
     ("helmholtz_256", "star3d_kernel<bwd>"): 101209600,
     ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 361327360,
     ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 507760640,
+    ("ns3d_steady_256", "ns3d_kernel<fwd>"): 518983168,
+    ("ns3d_steady_256", "ns3d_kernel<bwd>"): 730601728,
+    ("grayscott_4096", "fused2d_kernel<grayscott_2d>"): 234423552,
+    ("ns2d_steady_4096", "fused2d_kernel<ns_2d_steady>"): 373796864,
 }
 FALLBACK_HBM_GBS = 6650.0
 LAUNCHES_PER_STEP = 3               # forward kernel, loss finalise, adjoint kernel
