@@ -7,7 +7,9 @@
 `fused_residual` runs `fpde_fwd` (no loss) in the forward pass and `fpde_bwd` on the upstream
 sensitivities autograd hands back.  `fused_residual_loss` also fuses the mean-square loss: the
 forward pass is `fpde_fwd` with the loss, the backward pass is `fpde_bwd` on the residual
-arrays with scale 2/N_r, times the incoming scalar gradient.  Everything runs in the library's
+arrays with scale 2/N_r, times the incoming scalar gradient; where the operator has a
+single-pass kernel and a gradient is wanted, the forward pass is `fpde_fwd_bwd` (loss and
+dL/dfield from one kernel) and the backward pass only applies the incoming scalar.  Everything runs in the library's
 kernels on the current CUDA stream; torch allocates the outputs and nothing else.
 """
 from __future__ import annotations
@@ -54,23 +56,33 @@ class _FusedResidualLoss(torch.autograd.Function):
         shape = tuple(fields[0].shape)
         dev = fields[0].device
         ne = B.op_info(op).nresiduals
-        res = [torch.empty(shape, dtype=torch.float32, device=dev) for _ in range(ne)]
         loss = torch.empty(ne + 1, dtype=torch.float64, device=dev)
+        ctx.op, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc, ctx.ne = op, shape, spacing, coeffs, bc, ne
+        ctx.single_pass = B.has_single_pass(op) and any(ctx.needs_input_grad[5:])
+        if ctx.single_pass:
+            # one kernel: the loss and dL/dfield together, no residual arrays kept for backward
+            grads = [torch.empty(shape, dtype=torch.float32, device=dev) for _ in fields]
+            ws = torch.empty(B.fwd_bwd_workspace_bytes(op, shape), dtype=torch.uint8, device=dev)
+            B.fpde_fwd_bwd(op, fields, sources, None, grads, loss, shape, spacing, coeffs, bc, ws)
+            ctx.save_for_backward(*grads)
+            return loss[ne]
+        res = [torch.empty(shape, dtype=torch.float32, device=dev) for _ in range(ne)]
         ws = torch.empty(B.workspace_bytes(op, shape), dtype=torch.uint8, device=dev)
         B.fpde_fwd(op, fields, sources, res, loss, shape, spacing, coeffs, bc, ws)
-        ctx.op, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc, ctx.ne = op, shape, spacing, coeffs, bc, ne
         ctx.save_for_backward(*fields, *res)
         return loss[ne]
 
     @staticmethod
     def backward(ctx, gloss):
         saved = ctx.saved_tensors
+        gl = gloss.to(torch.float32)
+        if ctx.single_pass:
+            return (None, None, None, None, None) + tuple(g * gl for g in saved)
         nf = len(saved) - ctx.ne
         fields, res = saved[:nf], saved[nf:]
         out = [torch.empty(ctx.shape, dtype=torch.float32, device=fields[0].device) for _ in fields]
         scale = 2.0 / B.row_count(ctx.op, ctx.shape)
         B.fpde_bwd(ctx.op, fields, res, [scale] * ctx.ne, out, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc)
-        gl = gloss.to(torch.float32)
         return (None, None, None, None, None) + tuple(o * gl for o in out)
 
 

@@ -259,7 +259,7 @@ static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     const char* pf = std::getenv("FPDE_NS_PREFETCH");
-    p.prefetch = pf && *pf ? std::atoi(pf) : 3;
+    p.prefetch = pf && *pf ? std::atoi(pf) : 1;
     if (p.prefetch < 0 || p.prefetch >= p.n0) p.prefetch = 0;
 }
 
