@@ -218,6 +218,38 @@ int fpde_fwd_bwd(int op,
                  void* stream);
 
 /*
+ * Double-precision verification path (the paper trains and times in fp32 and uses fp64 only to
+ * verify its hand-derived adjoints): fpde_fwd / fpde_bwd with every array in double, computed by
+ * separate one-thread-per-node kernels written for clarity, not speed.  Same operators, shapes,
+ * boundary kinds, status codes and semantics (rows, zero at nodes without a row, loss in a fixed
+ * order, gradients overwritten at every node) as the fp32 entry points; pointers are device
+ * pointers to doubles, 16-byte aligned.  fpde_workspace_bytes_f64 gives the scratch fpde_fwd_f64
+ * needs when loss_out is given; fpde_bwd_f64 needs none.
+ */
+size_t fpde_workspace_bytes_f64(int op, int ndim, const int64_t* shape);
+int fpde_fwd_f64(int op,
+                 const double* const* fields,
+                 const double* const* sources,
+                 double* const* residuals,
+                 double* loss_out,
+                 int ndim, const int64_t* shape,
+                 const double* spacing,
+                 const double* coeffs, int ncoeffs,
+                 const int* bc,
+                 void* workspace, size_t workspace_bytes,
+                 void* stream);
+int fpde_bwd_f64(int op,
+                 const double* const* fields,
+                 const double* const* gres,
+                 const double* gscale,
+                 double* const* gfields,
+                 int ndim, const int64_t* shape,
+                 const double* spacing,
+                 const double* coeffs, int ncoeffs,
+                 const int* bc,
+                 void* stream);
+
+/*
  * Loss gradient from HOST buffers in one call: copies the fields (and sources) to the device,
  * runs fpde_fwd_bwd, i.e. the adjoint with the upstream sensitivities of the mean-square loss,
  * G_e = (2/N_r) r_e (Section 2.2: the operator receives G = dL/dres from the loss), and copies

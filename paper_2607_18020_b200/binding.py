@@ -74,6 +74,15 @@ def lib():
                                    ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                    ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                    ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fpde_workspace_bytes_f64.restype = ctypes.c_size_t
+        L.fpde_workspace_bytes_f64.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_fwd_f64.restype = ctypes.c_int
+        L.fpde_fwd_f64.argtypes = L.fpde_fwd.argtypes
+        L.fpde_bwd_f64.restype = ctypes.c_int
+        L.fpde_bwd_f64.argtypes = [ctypes.c_int, vpp, vpp, ctypes.POINTER(ctypes.c_double), vpp, ctypes.c_int,
+                                   ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                   ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                                   ctypes.c_void_p]
         L.fpde_host_arena_bytes.restype = ctypes.c_size_t
         L.fpde_host_arena_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
         L.fpde_loss_grad_host.restype = ctypes.c_int
@@ -241,6 +250,33 @@ def fpde_fwd_bwd(op, fields, sources, residuals, gfields, loss_out, shape, spaci
                         wsb, _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd_bwd")
+
+
+def workspace_bytes_f64(op, shape) -> int:
+    return int(lib().fpde_workspace_bytes_f64(_opid(op), len(shape), _i64(shape)))
+
+
+def fpde_fwd_f64(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, stream=None):
+    """fpde_fwd on fp64 CUDA tensors (verification path)."""
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    st = lib().fpde_fwd_f64(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(sources)),
+                            _ptr_array(_dev_ptrs(residuals)),
+                            _dev_ptrs([loss_out])[0] if loss_out is not None else None, len(shape), _i64(shape),
+                            _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                            _dev_ptrs([workspace])[0] if workspace is not None else None, int(wsb),
+                            _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_fwd_f64")
+
+
+def fpde_bwd_f64(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, stream=None):
+    """fpde_bwd on fp64 CUDA tensors (verification path)."""
+    st = lib().fpde_bwd_f64(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(gres)),
+                            _f64(gscale) if gscale is not None else None, _ptr_array(_dev_ptrs(gfields)),
+                            len(shape), _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                            _stream_handle(stream))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_bwd_f64")
 
 
 def fpde_bwd(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace=None, stream=None):

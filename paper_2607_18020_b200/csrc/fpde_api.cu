@@ -362,6 +362,99 @@ int fpde_fwd_bwd(int op, const float* const* fields, const float* const* sources
     return FPDE_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// double-precision verification path
+// ------------------------------------------------------------------------------------------
+static int validate_f64(int op, const double* const* fields, int ndim, const int64_t* shape, const double* spacing,
+                        const double* coeffs, int ncoeffs, const int* bc, ProblemF64& q, int64_t* total) {
+    int st = check_shape(op, ndim, shape, q.n, total, &q.rows);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!fields || !spacing || !bc) return FPDE_ERR_NULL;
+    if (ncoeffs != e.nc) return FPDE_ERR_COEFF_COUNT;
+    if (e.nc > 0 && !coeffs) return FPDE_ERR_NULL;
+    for (int a = 0; a < ndim; ++a) {
+        if (!(spacing[a] > 0.0) || !std::isfinite(spacing[a])) return FPDE_ERR_SPACING;
+        if (bc[a] != e.bc[a]) return FPDE_ERR_BC;
+        q.h[a] = spacing[a]; q.bc[a] = bc[a];
+    }
+    for (int c = 0; c < e.nc; ++c) {
+        if (!std::isfinite(coeffs[c])) return FPDE_ERR_SPACING;
+        q.coef[c] = coeffs[c];
+    }
+    for (int f = 0; f < e.nf; ++f) {
+        if (!fields[f]) return FPDE_ERR_NULL;
+        if (!aligned16(fields[f])) return FPDE_ERR_ALIGN;
+        q.in[f] = fields[f];
+    }
+    q.op = op; q.ndim = ndim; q.radius = e.radius;
+    return FPDE_OK;
+}
+
+size_t fpde_workspace_bytes_f64(int op, int ndim, const int64_t* shape) {
+    int64_t N = 0;
+    if (check_shape(op, ndim, shape, nullptr, &N, nullptr) != FPDE_OK) return 0;
+    return (size_t)f64_blocks(N) * REGISTRY[op].ne * sizeof(double) + 256;
+}
+
+int fpde_fwd_f64(int op, const double* const* fields, const double* const* sources, double* const* residuals,
+                 double* loss_out, int ndim, const int64_t* shape, const double* spacing, const double* coeffs,
+                 int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes, void* stream) {
+    ProblemF64 q;
+    std::memset(&q, 0, sizeof(q));
+    int64_t N = 0;
+    int st = validate_f64(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q, &N);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!residuals) return FPDE_ERR_NULL;
+    if (e.ns > 0 && !sources) return FPDE_ERR_NULL;
+    for (int s = 0; s < e.ns; ++s) {
+        if (!sources[s]) return FPDE_ERR_NULL;
+        if (!aligned16(sources[s])) return FPDE_ERR_ALIGN;
+        q.aux[s] = sources[s];
+    }
+    for (int r = 0; r < e.ne; ++r) {
+        if (!residuals[r]) return FPDE_ERR_NULL;
+        if (!aligned16(residuals[r])) return FPDE_ERR_ALIGN;
+        q.out[r] = residuals[r];
+    }
+    if (loss_out) {
+        if (!aligned16(loss_out)) return FPDE_ERR_ALIGN;
+        if (!workspace || !aligned16(workspace) ||
+            workspace_bytes < (size_t)f64_blocks(N) * e.ne * sizeof(double))
+            return FPDE_ERR_WORKSPACE;
+        q.partials = static_cast<double*>(workspace);
+        q.loss_out = loss_out;
+    }
+    q.stream = static_cast<cudaStream_t>(stream);
+    return launch_f64_fwd(q, e.ne) == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
+}
+
+int fpde_bwd_f64(int op, const double* const* fields, const double* const* gres, const double* gscale,
+                 double* const* gfields, int ndim, const int64_t* shape, const double* spacing, const double* coeffs,
+                 int ncoeffs, const int* bc, void* stream) {
+    ProblemF64 q;
+    std::memset(&q, 0, sizeof(q));
+    int st = validate_f64(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q, nullptr);
+    if (st != FPDE_OK) return st;
+    const OpEntry& e = REGISTRY[op];
+    if (!gres || !gfields) return FPDE_ERR_NULL;
+    for (int r = 0; r < e.ne; ++r) {
+        if (!gres[r]) return FPDE_ERR_NULL;
+        if (!aligned16(gres[r])) return FPDE_ERR_ALIGN;
+        q.aux[r] = gres[r];
+        q.gscale[r] = gscale ? gscale[r] : 1.0;
+        if (!std::isfinite(q.gscale[r])) return FPDE_ERR_SPACING;
+    }
+    for (int f = 0; f < e.nf; ++f) {
+        if (!gfields[f]) return FPDE_ERR_NULL;
+        if (!aligned16(gfields[f])) return FPDE_ERR_ALIGN;
+        q.out[f] = gfields[f];
+    }
+    q.stream = static_cast<cudaStream_t>(stream);
+    return launch_f64_bwd(q, e.nf) == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
+}
+
 static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 
 size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape) {

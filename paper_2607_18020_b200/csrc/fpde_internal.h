@@ -27,6 +27,26 @@ struct Problem {
     cudaStream_t stream;
 };
 
+// The same for the double-precision verification path (ops_f64.cu).
+struct ProblemF64 {
+    int op, ndim, radius;
+    int n[MAX_D];
+    int bc[MAX_D];
+    double h[MAX_D];
+    double coef[8];
+    const double* in[MAX_F];
+    const double* aux[MAX_F];
+    double* out[MAX_F];
+    double gscale[MAX_F];
+    double* partials;        // fwd: one double per block and residual (NULL = no loss)
+    double* loss_out;
+    int64_t rows;
+    cudaStream_t stream;
+};
+int f64_blocks(int64_t N);
+cudaError_t launch_f64_fwd(const ProblemF64& p, int nresiduals);
+cudaError_t launch_f64_bwd(const ProblemF64& p, int nfields);
+
 // Launch with programmatic stream serialisation allowed (kernels call pdl_wait_then_trigger()).
 // FPDE_PDL=0 in the environment falls back to plain stream order (for A/B measurements).
 bool pdl_enabled();

@@ -46,3 +46,18 @@ def test_residuals_with_downstream_loss(name, shape):
     ref = oracle.bwd(w.op, w.fields, [x.astype(np.float64) for x in wts], w.shape, w.spacing, w.coeffs)
     for f, gr in zip(fields, ref):
         assert_close(f.grad.cpu().numpy(), gr, name + " autograd J^T w")
+
+
+@pytest.mark.parametrize("name,shape", [("grayscott_4096", (5, 8)), ("ns2d_steady_4096", (5, 8)), ("burgers_256x128", (6, 5)),
+                                        ("ns3d_steady_256", (4, 4, 4))])
+def test_gradcheck_in_double_precision(name, shape):
+    """fp64 tensors go through the double-precision kernels, so torch's own finite-difference
+    check of the adjoint applies (the paper's fp64 verification mode)."""
+    from paper_2607_18020_b200.autograd import fused_residual, fused_residual_loss
+    w = W.make(name, seed=47, shape=shape, kind="randn")
+    fields = [torch.from_numpy(f.astype(np.float64)).cuda().requires_grad_(True) for f in w.fields]
+    sources = [torch.from_numpy(s.astype(np.float64)).cuda() for s in w.sources]
+    assert torch.autograd.gradcheck(lambda *f: fused_residual(w.op, f, sources, w.spacing, w.coeffs, w.bc), fields,
+                                    eps=1e-6, atol=1e-6, rtol=1e-6, nondet_tol=0.0)
+    assert torch.autograd.gradcheck(lambda *f: fused_residual_loss(w.op, f, sources, w.spacing, w.coeffs, w.bc), fields,
+                                    eps=1e-6, atol=1e-5, rtol=1e-5, nondet_tol=0.0)
