@@ -33,8 +33,8 @@
 typedef long long i64;
 
 enum { OP_BURGERS_1D_T = 0, OP_POISSON_2D = 1, OP_GRAYSCOTT_2D = 2, OP_HELMHOLTZ_3D_O4 = 3,
-       OP_NS_3D_T = 4, OP_NS_2D_STEADY = 5, OP_NS_3D_STEADY = 6,
-       OP_COUNT = 7 };
+       OP_NS_3D_T = 4, OP_NS_2D_STEADY = 5, OP_NS_3D_STEADY = 6, OP_NS_3D_T_XSLAB = 7,
+       OP_COUNT = 8 };
 enum { BC_PERIODIC = 0, BC_INTERIOR = 1, BC_ONE_SIDED = 2 };
 
 /* A 1-D difference formula at one node: value = sum_k w[k] * q[idx[k]] along one axis. */
@@ -115,11 +115,11 @@ static void scatter(const stencil* s, double* line, i64 stride, double a) {
     for (k = 0; k < s->n; ++k) line[s->idx[k] * stride] += a * s->w[k];
 }
 
-static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2, 3 };
-static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4 };
-static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0, 0 };
-static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4 };
-static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1, 1 };
+static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2, 3, 4 };
+static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4, 4 };
+static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0, 0, 0 };
+static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4, 4 };
+static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1, 1, 1 };
 static const int OP_BC[OP_COUNT][4] = {
     { BC_ONE_SIDED, BC_ONE_SIDED, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
@@ -128,6 +128,7 @@ static const int OP_BC[OP_COUNT][4] = {
     { BC_PERIODIC, BC_PERIODIC, BC_PERIODIC, BC_INTERIOR },
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, BC_INTERIOR, 0 },
+    { BC_INTERIOR, BC_PERIODIC, BC_PERIODIC, BC_INTERIOR },
 };
 
 int fpde_oracle_info(int op, int* ndim, int* nf, int* ns, int* ne, int* nc) {
@@ -254,13 +255,16 @@ static i64 helmholtz(int mode, const double* u, const double* f, double* r, cons
 }
 
 /* Unsteady incompressible Navier-Stokes on an (x,y,z,t) array, space periodic, rows at the
- * interior t nodes.  Section 2.1's residuals extended by d_t, w and d_z:
+ * interior t nodes.  With bcx = BC_INTERIOR the x axis is not periodic: rows only where the
+ * centred x formulas fit (x-index 1..n_x-2), the first and last x-plane are data.  That is the
+ * form one slab of a grid split along x takes (its outer planes are copies of the neighbours'
+ * planes), and on the planes that carry rows it is the same formula.  Section 2.1's residuals extended by d_t, w and d_z:
  *   mom_q = d_t q + u d_x q + v d_y q + w d_z q + d_{a_q} p - nu (d_xx+d_yy+d_zz) q, q in (u,v,w),
  *           a_u = x, a_v = y, a_w = z;
  *   cont  = d_x u + d_y v + d_z w.
  * fld = {u,v,w,p}; res / G / grd index: 0..2 momentum x,y,z, 3 continuity. */
 static i64 ns3dt(int mode, const double* const* fld, double* const* res, const double* const* G,
-                 double* const* grd, const i64* n, const double* h, const double* c) {
+                 double* const* grd, const i64* n, const double* h, const double* c, int bcx) {
     i64 i[4], rows = 0;
     i64 st[4];
     double nu = c[0];
@@ -273,7 +277,9 @@ static i64 ns3dt(int mode, const double* const* fld, double* const* res, const d
         double vel[3], dq[3][3], lap[3], dt[3], dp[3];
         int a, q;
         if (!d1(BC_INTERIOR, i[3], n[3], h[3], &stt)) continue;
-        for (a = 0; a < 3; ++a) {
+        if (!d1(bcx, i[0], n[0], h[0], &s1[0])) continue;
+        d2(bcx, i[0], n[0], h[0], &s2[0]);
+        for (a = 1; a < 3; ++a) {
             d1(BC_PERIODIC, i[a], n[a], h[a], &s1[a]);
             d2(BC_PERIODIC, i[a], n[a], h[a], &s2[a]);
         }
@@ -441,7 +447,8 @@ i64 fpde_oracle_fwd(int op, const double* const* fields, const double* const* so
     case OP_POISSON_2D: rows = poisson(0, fields[0], sources[0], residuals[0], NULL, NULL, shape, spacing); break;
     case OP_GRAYSCOTT_2D: rows = grayscott(0, fields[0], fields[1], residuals[0], residuals[1], NULL, NULL, NULL, NULL, shape, spacing, coeffs); break;
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(0, fields[0], sources[0], residuals[0], NULL, NULL, shape, spacing, coeffs); break;
-    case OP_NS_3D_T: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
+    case OP_NS_3D_T: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs, BC_PERIODIC); break;
+    case OP_NS_3D_T_XSLAB: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs, BC_INTERIOR); break;
     case OP_NS_2D_STEADY: rows = ns2d(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
     case OP_NS_3D_STEADY: rows = ns3d(0, fields, residuals, NULL, NULL, shape, spacing, coeffs); break;
     }
@@ -471,7 +478,8 @@ i64 fpde_oracle_bwd(int op, const double* const* fields, const double* const* G,
     case OP_POISSON_2D: rows = poisson(1, fields[0], NULL, NULL, G[0], gfields[0], shape, spacing); break;
     case OP_GRAYSCOTT_2D: rows = grayscott(1, fields[0], fields[1], NULL, NULL, G[0], G[1], gfields[0], gfields[1], shape, spacing, coeffs); break;
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(1, fields[0], NULL, NULL, G[0], gfields[0], shape, spacing, coeffs); break;
-    case OP_NS_3D_T: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
+    case OP_NS_3D_T: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs, BC_PERIODIC); break;
+    case OP_NS_3D_T_XSLAB: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs, BC_INTERIOR); break;
     case OP_NS_2D_STEADY: rows = ns2d(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
     case OP_NS_3D_STEADY: rows = ns3d(1, fields, NULL, G, gfields, shape, spacing, coeffs); break;
     }

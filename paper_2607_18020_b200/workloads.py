@@ -34,7 +34,8 @@ HELMHOLTZ_3D_O4 = "helmholtz_3d_o4"
 NS_3D_T = "ns_3d_t"
 NS_2D_STEADY = "ns_2d_steady"
 NS_3D_STEADY = "ns_3d_steady"
-OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY, NS_3D_STEADY)
+NS_3D_T_XSLAB = "ns_3d_t_xslab"     # NS_3D_T with a non-periodic x axis: the form of one slab of a grid split along x
+OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY, NS_3D_STEADY, NS_3D_T_XSLAB)
 
 # Boundary kinds per array axis.
 PERIODIC = "periodic"      # rows at every node, wrap-around neighbours
@@ -122,7 +123,12 @@ CONFIGS["ns2d_steady_4096"] = dict(op=NS_2D_STEADY, shape=(4096, 4096),
                                    domain=((0.0, 1.0), (0.0, 1.0)), bc=(INTERIOR, INTERIOR))
 CONFIGS["ns3d_steady_256"] = dict(op=NS_3D_STEADY, shape=(256, 256, 256),
                                   domain=((0.0, 1.0),) * 3, bc=(INTERIOR,) * 3)
+# one of four x-slabs of the 128^3 x 16 Navier-Stokes grid, with its two halo planes
+CONFIGS["ns_tgv_xslab_34"] = dict(op=NS_3D_T_XSLAB, shape=(34, 128, 128, 16),
+                                  domain=((0.0, 2 * math.pi * 33 / 128),) + ((0.0, 2 * math.pi),) * 2 + ((0.0, 1.0),),
+                                  bc=(INTERIOR, PERIODIC, PERIODIC, INTERIOR))
 EXTRA_CONFIGS = ("ns2d_steady_4096", "ns3d_steady_256")
+SLAB_CONFIGS = ("ns_tgv_xslab_34",)
 CONFIG_ORDER = ("burgers_256x128", "poisson_1024", "grayscott_4096", "helmholtz_256", "ns_tgv_128x16")
 
 OP_META = {
@@ -135,6 +141,8 @@ OP_META = {
     NS_2D_STEADY: dict(fields=("u", "v", "p"), sources=(), residuals=("res_u", "res_v", "res_div"), ncoeffs=1),
     NS_3D_STEADY: dict(fields=("u", "v", "w", "p"), sources=(),
                        residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
+    NS_3D_T_XSLAB: dict(fields=("u", "v", "w", "p"), sources=(),
+                        residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
 }
 DEFAULT_COEFFS = {
     BURGERS_1D_T: (0.01 / math.pi,),
@@ -144,6 +152,7 @@ DEFAULT_COEFFS = {
     NS_3D_T: (0.01,),
     NS_2D_STEADY: (0.01,),
     NS_3D_STEADY: (0.01,),
+    NS_3D_T_XSLAB: (0.01,),
 }
 
 
@@ -185,7 +194,7 @@ def analytic_fields(op: str, axes: Sequence[np.ndarray], coeffs: Sequence[float]
         us = np.sin(2 * math.pi * x) * np.sin(2 * math.pi * y) * np.sin(2 * math.pi * z)
         k = coeffs[0]
         return [us.copy()], [(k * k - 12 * math.pi ** 2) * us]
-    if op == NS_3D_T:
+    if op in (NS_3D_T, NS_3D_T_XSLAB):
         x, y, z, t = (_bcast(axes, a) for a in range(4))
         nu = coeffs[0]
         e2, e4 = np.exp(-2 * nu * t), np.exp(-4 * nu * t)
@@ -211,7 +220,8 @@ def analytic_fields(op: str, axes: Sequence[np.ndarray], coeffs: Sequence[float]
     raise ValueError(op)
 
 
-_NOISE_SIGMA = {BURGERS_1D_T: 0.01, POISSON_2D: 0.05, HELMHOLTZ_3D_O4: 0.05, NS_3D_T: 0.01, NS_2D_STEADY: 0.01, NS_3D_STEADY: 0.01}
+_NOISE_SIGMA = {BURGERS_1D_T: 0.01, POISSON_2D: 0.05, HELMHOLTZ_3D_O4: 0.05, NS_3D_T: 0.01, NS_2D_STEADY: 0.01, NS_3D_STEADY: 0.01,
+                NS_3D_T_XSLAB: 0.01}
 
 
 def make(name: str, seed: int = 42, shape: Optional[Sequence[int]] = None, kind: str = "config",
@@ -227,7 +237,7 @@ def make(name: str, seed: int = 42, shape: Optional[Sequence[int]] = None, kind:
               profile is then evaluated on the nodes ``lo + i*h``).
     """
     if name in OPS:
-        name = next(k for k in CONFIG_ORDER + EXTRA_CONFIGS if CONFIGS[k]["op"] == name)
+        name = next(k for k in CONFIG_ORDER + EXTRA_CONFIGS + SLAB_CONFIGS if CONFIGS[k]["op"] == name)
     cfg = CONFIGS[name]
     op = cfg["op"]
     shape = tuple(int(s) for s in (shape if shape is not None else cfg["shape"]))

@@ -299,6 +299,7 @@ CASES = [
     (W.NS_3D_T, (5, 6, 5, 6), (0.3, 0.2, 0.25, 0.15), (0.13,)),
     (W.NS_2D_STEADY, (8, 9), (0.2, 0.3), (0.17,)),
     (W.NS_3D_STEADY, (6, 7, 5), (0.2, 0.3, 0.25), (0.17,)),
+    (W.NS_3D_T_XSLAB, (6, 5, 4, 6), (0.3, 0.2, 0.25, 0.15), (0.13,)),
 ]
 
 
@@ -346,6 +347,7 @@ TINY = [
     (W.NS_3D_T, (4, 5, 4, 5), (0.3, 0.2, 0.25, 0.15), (0.13,)),
     (W.NS_2D_STEADY, (6, 7), (0.2, 0.3), (0.17,)),
     (W.NS_3D_STEADY, (5, 4, 5), (0.2, 0.3, 0.25), (0.17,)),
+    (W.NS_3D_T_XSLAB, (5, 4, 4, 5), (0.3, 0.2, 0.25, 0.15), (0.13,)),
 ]
 
 
@@ -604,3 +606,27 @@ def test_inputs_are_seeded_and_reproducible():
     assert 0 < u.min() and u.max() < 1 and abs(u.mean() - 0.5) < 0.005
     # counter-based: a slice can be regenerated on its own
     assert np.array_equal(W.normal01(42, 3, 10, start=1000), z[1000:1010])
+
+
+def test_ns3dt_xslab_is_the_periodic_operator_on_its_inner_planes():
+    """The slab form (x not periodic, rows at x-index 1..n-2) against the periodic operator on
+    the same array: identical residuals on the inner planes, none on the two outer ones; and for
+    upstream arrays that vanish on the outer planes, the same adjoint at every node."""
+    shape, h, c = (7, 5, 4, 6), (0.3, 0.2, 0.25, 0.15), (0.13,)
+    r = np.random.default_rng(77)
+    F = [r.standard_normal(shape) for _ in range(4)]
+    Rp, _, rows_p = oracle.fwd(W.NS_3D_T, F, [], shape, h, c)
+    Rs, _, rows_s = oracle.fwd(W.NS_3D_T_XSLAB, F, [], shape, h, c)
+    assert rows_p == 7 * 5 * 4 * 4 and rows_s == 5 * 5 * 4 * 4
+    for a, b in zip(Rp, Rs):
+        assert np.array_equal(a[1:-1], b[1:-1])
+        assert np.all(b[0] == 0.0) and np.all(b[-1] == 0.0)
+        assert np.any(a[0] != 0.0)
+    G = [r.standard_normal(shape) for _ in range(4)]
+    G0 = [g.copy() for g in G]
+    for g in G0:
+        g[0] = 0.0; g[-1] = 0.0
+    gs = oracle.bwd(W.NS_3D_T_XSLAB, F, G, shape, h, c)          # outer planes of G are ignored
+    gp = oracle.bwd(W.NS_3D_T, F, G0, shape, h, c)
+    for a, b in zip(gs, gp):
+        assert np.allclose(a, b, rtol=0, atol=1e-12)
