@@ -80,6 +80,11 @@ typedef enum {
  *        the third component: mom_q = u d_x q + v d_y q + w d_z q + d_{a_q} p - nu Lap q,
  *        continuity = d_x u + d_y v + d_z w, centred differences.  bc = (INTERIOR x3): rows at
  *        the interior nodes, the outer shell is data and receives gradient.
+ *  FPDE_OP_NS_3D_T_XSLAB   FPDE_OP_NS_3D_T with a non-periodic x axis, bc = (INTERIOR, PERIODIC,
+ *        PERIODIC, INTERIOR): rows at x-index 1..n_x-2 (and t-index 1..n_t-2), the first and last
+ *        x-plane are data.  This is the form one slab of a grid split along x takes: its outer
+ *        planes are copies of the neighbouring slabs' planes, and on the planes that carry rows
+ *        the residuals are those of the periodic operator on the whole grid.
  *
  * Shape rules: the contiguous extent must be a multiple of 4 (float4 path) except for
  * BURGERS_1D_T; PERIODIC / INTERIOR axes need n >= 2*radius+1, ONE_SIDED axes n >= 4; the
@@ -93,7 +98,8 @@ typedef enum {
     FPDE_OP_NS_3D_T = 4,
     FPDE_OP_NS_2D_STEADY = 5,
     FPDE_OP_NS_3D_STEADY = 6,
-    FPDE_OP_COUNT = 7
+    FPDE_OP_NS_3D_T_XSLAB = 7,
+    FPDE_OP_COUNT = 8
 } fpde_op;
 
 /* Boundary kind of one array axis (Appendix A.4 names the three causes of boundary terms:

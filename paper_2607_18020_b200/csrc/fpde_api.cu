@@ -14,7 +14,7 @@ namespace fpde {
 
 int lap2d_items(const int* n);
 int star3d_items(const int* n);
-int ns_items(const int* n);
+int ns_items(const int* n, bool xint);
 int burgers_items(const int* n);
 int ns2d_items(const int* n);
 int ns3d_items(const int* n);
@@ -33,6 +33,7 @@ static const OpEntry REGISTRY[FPDE_OP_COUNT] = {
     /* NS_3D_T         */ {4, 4, 0, 4, 1, 1, {FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_INTERIOR}, true},
     /* NS_2D_STEADY    */ {2, 3, 0, 3, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0, 0}, true},
     /* NS_3D_STEADY    */ {3, 4, 0, 4, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0}, true},
+    /* NS_3D_T_XSLAB   */ {4, 4, 0, 4, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_INTERIOR}, true},
 };
 
 static int check_shape(int op, int ndim, const int64_t* shape, int* n_out, int64_t* total, int64_t* rows) {
@@ -63,7 +64,8 @@ static size_t workspace_need(int op, const int* n) {
     case FPDE_OP_POISSON_2D:
     case FPDE_OP_GRAYSCOTT_2D: items = lap2d_items(n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: items = star3d_items(n); break;
-    case FPDE_OP_NS_3D_T: items = ns_items(n); break;
+    case FPDE_OP_NS_3D_T: items = ns_items(n, false); break;
+    case FPDE_OP_NS_3D_T_XSLAB: items = ns_items(n, true); break;
     case FPDE_OP_NS_2D_STEADY: items = ns2d_items(n); break;
     case FPDE_OP_NS_3D_STEADY: items = ns3d_items(n); break;
     }
@@ -102,6 +104,7 @@ static int validate(int op, const float* const* fields, int ndim, const int64_t*
         q.in[f] = fields[f];
     }
     q.op = op; q.ndim = ndim;
+    q.bc0_interior = op == FPDE_OP_NS_3D_T_XSLAB;
     return FPDE_OK;
 }
 
@@ -242,7 +245,8 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     case FPDE_OP_POISSON_2D:
     case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_fwd(q); items = lap2d_items(q.n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q); items = star3d_items(q.n); break;
-    case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n); break;
+    case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n, false); break;
+    case FPDE_OP_NS_3D_T_XSLAB: ce = launch_ns_fwd(q); items = ns_items(q.n, true); break;
     case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_fwd(q); items = ns2d_items(q.n); break;
     case FPDE_OP_NS_3D_STEADY: ce = launch_ns3d_fwd(q); items = ns3d_items(q.n); break;
     }
@@ -284,7 +288,8 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
     case FPDE_OP_POISSON_2D:
     case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_bwd(q); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_bwd(q); break;
-    case FPDE_OP_NS_3D_T: ce = launch_ns_bwd(q); break;
+    case FPDE_OP_NS_3D_T:
+    case FPDE_OP_NS_3D_T_XSLAB: ce = launch_ns_bwd(q); break;
     case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_bwd(q); break;
     case FPDE_OP_NS_3D_STEADY: ce = launch_ns3d_bwd(q); break;
     }

@@ -25,6 +25,7 @@ struct Problem {
     double* loss_out;        // fwd: device, E+1 doubles
     int64_t rows;            // N_r
     cudaStream_t stream;
+    bool bc0_interior;       // unsteady NS only: x axis not periodic (the slab form of the operator)
 };
 
 // The same for the double-precision verification path (ops_f64.cu).

@@ -41,6 +41,7 @@ struct NsParams {
     NsConsts k;
     float* partials;
     int prefetch;         // planes ahead of the window to prefetch into L2 (0 = off)
+    int xint;             // x axis not periodic: rows at x-index 1..n0-2 only (one slab of a split grid)
 };
 
 struct NsIndex {
@@ -53,6 +54,17 @@ struct NsIndex {
 };
 
 __device__ __forceinline__ int wrapi(int i, int n) { return i < 0 ? i + n : (i >= n ? i - n : i); }
+// x-plane a step reads: wrapped, or (non-periodic x) clamped into the array; a clamped plane only
+// ever feeds an output that is zeroed or an upstream value that counts as zero
+__device__ __forceinline__ int xplane(const NsParams& p, int a) {
+    return p.xint ? max(0, min(p.n0 - 1, a)) : wrapi(a, p.n0);
+}
+__device__ __forceinline__ bool xdead(const NsParams& p, int a) { return p.xint && (a < 1 || a > p.n0 - 2); }
+template <int NA>
+__device__ __forceinline__ void zero_from(V4 (&W)[NA], int first) {
+#pragma unroll
+    for (int k = 0; k < NA; ++k) if (k >= first) W[k] = v4zero();
+}
 
 // Ask L2 for the line holding `ptr` (no register, no wait): hides most of the DRAM latency of
 // the plane the register window will pull in a few steps later.
@@ -117,7 +129,7 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
 
     V4 A[4], B[4], Cc[4];                           // three x-planes of u,v,w,p at the own column
     {
-        const int om = wrapi(a0 - 1, n0) * PS + ix.rowoff + ix.col;
+        const int om = xplane(p, a0 - 1) * PS + ix.rowoff + ix.col;
         const int oc = a0 * PS + ix.rowoff + ix.col;
 #pragma unroll
         for (int k = 0; k < 4; ++k) { A[k] = ldv4(fp[k] + om); B[k] = ldv4(fp[k] + oc); }
@@ -129,9 +141,9 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
     // one x step: W0 = plane a-1, W1 = plane a, W2 receives plane a+1
     auto step = [&](int a, const V4 (&W0)[4], const V4 (&W1)[4], V4 (&W2)[4]) {
         const int pl = a * PS;
-        const int ap = wrapi(a + 1, n0) * PS;
+        const int ap = xplane(p, a + 1) * PS;
         if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= a1) {   // one lane per 128-byte line
-            int af = a + 1 + p.prefetch; if (af >= n0) af -= n0;
+            const int af = xplane(p, a + 1 + p.prefetch);
             const int po = af * PS + ix.rowoff + ix.col;
 #pragma unroll
             for (int k = 0; k < 4; ++k) prefetch_l2(fp[k] + po);
@@ -150,6 +162,10 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
         for (int k = 0; k < 3; ++k) t_neighbours<TSAFE>(W1[k], fp[k] + pl + ix.rowoff, ix, l1[k], r1[k]);
         float2 o[4][2];
         ns_fwd_math(p.k, W0, W1, W2, Ym, Yp, Zm, Zp, l1, r1, ix.t_first, ix.t_last, o);
+        if (xdead(p, a)) {                          // the two outer x-planes of a slab carry no row
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { o[e][0] = make_float2(0.f, 0.f); o[e][1] = o[e][0]; }
+        }
         if (ix.valid) {
             const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
@@ -196,17 +212,20 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
 
     V4 A[7], B[7], Cc[7];
     {
-        const int om = wrapi(a0 - 1, n0) * PS + ix.rowoff + ix.col;
+        const int om = xplane(p, a0 - 1) * PS + ix.rowoff + ix.col;
         const int oc = a0 * PS + ix.rowoff + ix.col;
 #pragma unroll
         for (int k = 0; k < 7; ++k) { A[k] = ldv4(ap[k] + om); B[k] = ldv4(ap[k] + oc); }
+        // upstream arrays count as zero on planes without rows
+        if (xdead(p, a0 - 1)) zero_from<7>(A, 3);
+        if (xdead(p, a0)) zero_from<7>(B, 3);
     }
 
     auto step = [&](int a, const V4 (&W0)[7], const V4 (&W1)[7], V4 (&W2)[7]) {
         const int pl = a * PS;
-        const int apl = wrapi(a + 1, n0) * PS;
+        const int apl = xplane(p, a + 1) * PS;
         if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= a1) {
-            int af = a + 1 + p.prefetch; if (af >= n0) af -= n0;
+            const int af = xplane(p, a + 1 + p.prefetch);
             const int po = af * PS + ix.rowoff + ix.col;
 #pragma unroll
             for (int k = 0; k < 7; ++k) prefetch_l2(ap[k] + po);
@@ -220,9 +239,14 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
             Zm[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zmcol);
             Zp[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zpcol);
         }
+        if (xdead(p, a + 1)) zero_from<7>(W2, 3);
+        if (xdead(p, a)) { zero_from<7>(Ym, 3); zero_from<7>(Yp, 3); zero_from<7>(Zm, 3); zero_from<7>(Zp, 3); }
         float l1[3], r1[3];
 #pragma unroll
-        for (int q = 0; q < 3; ++q) t_neighbours<TSAFE>(W1[3 + q], ap[3 + q] + pl + ix.rowoff, ix, l1[q], r1[q]);
+        for (int q = 0; q < 3; ++q) {
+            t_neighbours<TSAFE>(W1[3 + q], ap[3 + q] + pl + ix.rowoff, ix, l1[q], r1[q]);
+            if (xdead(p, a)) { l1[q] = 0.f; r1[q] = 0.f; }
+        }
         float2 o[4][2];
         ns_bwd_math(p.k, W0, W1, W2, Ym, Yp, Zm, Zp, l1, r1, ix.t_first, ix.t_last, o);
         if (ix.valid) {
@@ -261,21 +285,23 @@ static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
     const char* pf = std::getenv("FPDE_NS_PREFETCH");
     p.prefetch = pf && *pf ? std::atoi(pf) : 1;
     if (p.prefetch < 0 || p.prefetch >= p.n0) p.prefetch = 0;
+    p.xint = q.bc0_interior ? 1 : 0;
 }
 
 static bool ns_tsafe(const NsParams& p) { return 32 % p.nt4 == 0; }
 
-int ns_items(const int* n) {
-    if (ns_tma_wanted(n)) return ns_tma_items(n);
+int ns_items(const int* n, bool xint) {
+    if (!xint && ns_tma_wanted(n)) return ns_tma_items(n);
     Problem q{};
     for (int a = 0; a < 4; ++a) { q.n[a] = n[a]; q.h[a] = 1.0; }
+    q.bc0_interior = xint;
     NsParams p{}; dim3 block;
     ns_geometry(q, p, block);
     return p.nitems;
 }
 
 cudaError_t launch_ns_fwd(const Problem& q) {
-    {
+    if (!q.bc0_interior) {
         bool launched = false;
         const cudaError_t ce = launch_ns_fwd_tma(q, launched);
         if (launched || ce != cudaSuccess) return ce;
@@ -295,7 +321,7 @@ cudaError_t launch_ns_fwd(const Problem& q) {
 }
 
 cudaError_t launch_ns_bwd(const Problem& q) {
-    {
+    if (!q.bc0_interior) {
         bool launched = false;
         const cudaError_t ce = launch_ns_bwd_tma(q, launched);
         if (launched || ce != cudaSuccess) return ce;

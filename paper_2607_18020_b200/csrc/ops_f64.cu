@@ -171,12 +171,12 @@ __device__ void residual_at(const F64Params& p, const Node& q, double* r) {
         r[0] = d2o4(p, p.in[0], q, 0) + d2o4(p, p.in[0], q, 1) + d2o4(p, p.in[0], q, 2)
              + p.coef[0] * p.coef[0] * p.in[0][q.idx] - p.aux[0][q.idx];
         break;
-    default: {                                            // Navier-Stokes: 3-D+T (4), steady 2-D (5), steady 3-D (6)
+    default: {                                            // Navier-Stokes: 3-D+T (4, slab form 7), steady 2-D (5), steady 3-D (6)
         const double* pr = p.in[nv];
         double cont = 0.0;
         for (int c = 0; c < nv; ++c) {
             const double* f = p.in[c];
-            double m = p.op == 4 ? d1c(p, f, q, 3) : 0.0;
+            double m = (p.op == 4 || p.op == 7) ? d1c(p, f, q, 3) : 0.0;
             for (int a = 0; a < nv; ++a) m += p.in[a][q.idx] * d1c(p, f, q, a) - p.coef[0] * d2c(p, f, q, a);
             r[c] = m + d1c(p, pr, q, c);
             cont += d1c(p, f, q, c);
@@ -282,7 +282,7 @@ __device__ void adjoint_at(const F64Params& p, const Node& q, double* g) {
                      / (2.0 * p.h[a]);
                 s -= p.coef[0] * G_d2c(p, c, q, a);
             }
-            if (p.op == 4) s += G_d1T(p, c, q, 3);
+            if (p.op == 4 || p.op == 7) s += G_d1T(p, c, q, 3);
             s += G_d1T(p, nv, q, c);
             g[c] = s;
             gp += G_d1T(p, c, q, c);

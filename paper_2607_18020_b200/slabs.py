@@ -1,0 +1,284 @@
+"""One grid split into slabs along its slowest axis (x), one slab per rank.
+
+The operators have exactly one exchange step when a grid is split: a node's residual reads the
+fields `radius` planes to either side, and the gather-form adjoint reads the upstream arrays
+`radius` planes to either side (and, where the Jacobian depends on the fields, the fields at
+those rows' own neighbours).  So per step a rank
+
+  1. receives 2*radius halo planes of every field from each x neighbour,
+  2. runs the forward kernel on the planes [x0 - radius, x1 + radius): rows on its own planes,
+  3. receives radius halo planes of every residual array,
+  4. runs the adjoint kernel on the planes [x0 - 2 radius, x1 + 2 radius): with the interior-axis
+     rule (rows where the stencil fits) the upstream arrays are honoured on [x0 - radius,
+     x1 + radius), which is what the gradients on the own planes [x0, x1) need,
+  5. sums the loss over ranks (nresiduals + 1 doubles).
+
+Every array is stored once per rank with the widest halo; the forward call is handed a
+sub-range of planes (contiguous, because x is the slowest axis), so nothing is copied locally.
+An operator whose x axis is an interior axis is its own slab form (at the two ends of the
+domain the halo is simply absent); the periodic unsteady Navier-Stokes operator has a slab form
+with a non-periodic x axis (`ns_3d_t_xslab`).  The kernels are the single-GPU kernels; this
+module only plans the ranges and moves the halo planes (torch.distributed point-to-point, or
+plain copies when several slabs live in one process).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Sequence, Tuple
+
+from . import workloads as W
+
+# operator on the whole grid -> operator one slab runs
+SLAB_OP = {
+    W.POISSON_2D: W.POISSON_2D,
+    W.HELMHOLTZ_3D_O4: W.HELMHOLTZ_3D_O4,
+    W.NS_2D_STEADY: W.NS_2D_STEADY,
+    W.NS_3D_STEADY: W.NS_3D_STEADY,
+    W.NS_3D_T: W.NS_3D_T_XSLAB,
+}
+RADIUS = {W.POISSON_2D: 1, W.HELMHOLTZ_3D_O4: 2, W.NS_2D_STEADY: 1, W.NS_3D_STEADY: 1, W.NS_3D_T: 1}
+
+
+@dataclass(frozen=True)
+class Transfer:
+    """`count` planes starting at global plane `start`, owned by `peer`, land at local plane `dst`."""
+    peer: int
+    start: int
+    count: int
+    dst: int
+
+
+@dataclass(frozen=True)
+class SlabPlan:
+    op: str                    # operator on the whole grid
+    shape: Tuple[int, ...]     # whole grid
+    world: int
+    rank: int
+
+    @property
+    def local_op(self) -> str:
+        return SLAB_OP[self.op]
+
+    @property
+    def radius(self) -> int:
+        return RADIUS[self.op]
+
+    @property
+    def periodic(self) -> bool:
+        return W.CONFIGS[next(k for k, c in W.CONFIGS.items() if c["op"] == self.op)]["bc"][0] == W.PERIODIC
+
+    def owned_of(self, rank: int) -> Tuple[int, int]:
+        n0 = self.shape[0]
+        return rank * n0 // self.world, (rank + 1) * n0 // self.world
+
+    @property
+    def owned(self) -> Tuple[int, int]:
+        return self.owned_of(self.rank)
+
+    def _range(self, halo: int) -> Tuple[int, int]:
+        x0, x1 = self.owned
+        if self.periodic:
+            return x0 - halo, x1 + halo                      # may run past the ends: planes wrap
+        return max(0, x0 - halo), min(self.shape[0], x1 + halo)
+
+    @property
+    def wide(self) -> Tuple[int, int]:
+        """Planes every local array holds."""
+        return self._range(2 * self.radius)
+
+    @property
+    def tight(self) -> Tuple[int, int]:
+        """Planes the forward kernel is run on."""
+        return self._range(self.radius)
+
+    @property
+    def local_shape(self) -> Tuple[int, ...]:
+        w0, w1 = self.wide
+        return (w1 - w0,) + tuple(self.shape[1:])
+
+    @property
+    def tight_shape(self) -> Tuple[int, ...]:
+        t0, t1 = self.tight
+        return (t1 - t0,) + tuple(self.shape[1:])
+
+    def local_of(self, plane: int) -> int:
+        """Local plane index of a global plane index of this rank's wide range."""
+        return plane - self.wide[0]
+
+    def owner(self, plane: int) -> int:
+        n0 = self.shape[0]
+        g = plane % n0
+        for r in range(self.world):
+            a, b = self.owned_of(r)
+            if a <= g < b:
+                return r
+        raise AssertionError(plane)
+
+    def check(self):
+        if self.op not in SLAB_OP:
+            raise ValueError("operator %s has no slab form" % self.op)
+        for r in range(self.world):
+            a, b = self.owned_of(r)
+            if b - a < 2 * self.radius:
+                raise ValueError("slab of rank %d has %d planes; at least %d are needed" % (r, b - a, 2 * self.radius))
+        if self.periodic and self.shape[0] < 4 * self.radius:
+            raise ValueError("grid too short along x")
+
+    def halo_transfers(self, halo: int) -> List[Transfer]:
+        """What this rank receives to fill `halo` planes beyond each end of its own planes: runs of
+        consecutive planes with one owner, in ascending local order."""
+        x0, x1 = self.owned
+        lo, hi = self._range(halo)
+        out: List[Transfer] = []
+        for a, b in ((lo, x0), (x1, hi)):
+            g = a
+            while g < b:
+                peer = self.owner(g)
+                pa, pb = self.owned_of(peer)
+                start = g % self.shape[0]
+                count = min(b - g, pb - start)
+                out.append(Transfer(peer, start, count, self.local_of(g)))
+                g += count
+        return out
+
+    def sends(self, halo: int) -> List[Tuple[int, Transfer]]:
+        """(destination rank, transfer as seen by the destination) for everything this rank owns
+        that another rank's halo needs, in the destination's order."""
+        out = []
+        for r in range(self.world):
+            plan = SlabPlan(self.op, self.shape, self.world, r)
+            for t in plan.halo_transfers(halo):
+                if t.peer == self.rank:
+                    out.append((r, t))
+        return out
+
+
+def plans(op: str, shape: Sequence[int], world: int) -> List[SlabPlan]:
+    ps = [SlabPlan(op, tuple(int(s) for s in shape), world, r) for r in range(world)]
+    ps[0].check()
+    return ps
+
+
+def exchange_local(plan_list: Sequence[SlabPlan], arrays: Sequence[Sequence], halo: int):
+    """Fill the halo planes when all slabs live in this process: arrays[rank][k] is the k-th
+    local array (wide range) of that rank."""
+    for plan in plan_list:
+        for t in plan.halo_transfers(halo):
+            src_plan = plan_list[t.peer]
+            s = src_plan.local_of(t.start)
+            for dst_arr, src_arr in zip(arrays[plan.rank], arrays[t.peer]):
+                dst_arr[t.dst:t.dst + t.count].copy_(src_arr[s:s + t.count])
+
+
+def exchange_dist(plan: SlabPlan, arrays: Sequence, halo: int, dist):
+    """Fill the halo planes of this rank's arrays from the other ranks (torch.distributed
+    point-to-point; both sides enumerate the transfers in the same order).  Planes a rank
+    needs from itself (one rank on a periodic axis) are copied."""
+    ops = []
+    for t in plan.halo_transfers(halo):
+        for arr in arrays:
+            if t.peer == plan.rank:
+                s = plan.local_of(t.start)
+                arr[t.dst:t.dst + t.count].copy_(arr[s:s + t.count].clone())
+            else:
+                ops.append(dist.P2POp(dist.irecv, arr[t.dst:t.dst + t.count], t.peer))
+    for dst, t in plan.sends(halo):
+        if dst == plan.rank:
+            continue
+        s = plan.local_of(t.start)
+        for arr in arrays:
+            ops.append(dist.P2POp(dist.isend, arr[s:s + t.count], dst))
+    if ops:
+        for req in dist.batch_isend_irecv(ops):
+            req.wait()
+
+
+class SlabRank:
+    """The arrays and kernel calls of one slab."""
+
+    def __init__(self, torch, B, plan: SlabPlan, spacing, coeffs, device="cuda"):
+        plan.check()
+        self.torch, self.B, self.plan = torch, B, plan
+        self.spacing, self.coeffs = tuple(spacing), tuple(coeffs)
+        meta = W.OP_META[plan.op]
+        self.nf, self.ns, self.ne = len(meta["fields"]), len(meta["sources"]), len(meta["residuals"])
+        self.bc = W.CONFIGS[next(k for k, c in W.CONFIGS.items() if c["op"] == plan.local_op)]["bc"]
+        ls = plan.local_shape
+        new = lambda: torch.zeros(ls, dtype=torch.float32, device=device)
+        self.fields = [new() for _ in range(self.nf)]
+        self.sources = [new() for _ in range(self.ns)]
+        self.res = [new() for _ in range(self.ne)]
+        self.grads = [new() for _ in range(self.nf)]
+        self.loss = torch.zeros(self.ne + 1, dtype=torch.float64, device=device)
+        self.ws = torch.empty(max(16, B.workspace_bytes(plan.local_op, plan.tight_shape)), dtype=torch.uint8, device=device) \
+            if device != "cpu" else None
+        self.rows_global = B.row_count(plan.op, plan.shape) if device != "cpu" else 0
+        self.rows_local = B.row_count(plan.local_op, plan.tight_shape) if device != "cpu" else 0
+
+    def _owned_slice(self):
+        x0, x1 = self.plan.owned
+        return slice(self.plan.local_of(x0), self.plan.local_of(x1))
+
+    def _tight_slice(self):
+        t0, t1 = self.plan.tight
+        return slice(self.plan.local_of(t0), self.plan.local_of(t1))
+
+    def owned(self, arrays):
+        s = self._owned_slice()
+        return [a[s] for a in arrays]
+
+    def load_owned(self, fields, sources):
+        """Copy this rank's planes of whole-grid arrays (numpy or torch) into the local arrays."""
+        x0, x1 = self.plan.owned
+        for dst, src in zip(self.owned(self.fields) + self.owned(self.sources), list(fields) + list(sources)):
+            dst.copy_(self.torch.as_tensor(src[x0:x1]))
+
+    def fwd(self, stream=None):
+        s = self._tight_slice()
+        p = self.plan
+        self.B.fpde_fwd(p.local_op, [a[s] for a in self.fields], [a[s] for a in self.sources], [a[s] for a in self.res],
+                        self.loss, p.tight_shape, self.spacing, self.coeffs, self.bc, self.ws, stream)
+
+    def bwd(self, stream=None):
+        p = self.plan
+        self.B.fpde_bwd(p.local_op, self.fields, self.res, [2.0 / self.rows_global] * self.ne, self.grads,
+                        p.local_shape, self.spacing, self.coeffs, self.bc, None, stream)
+
+    def loss_sums(self):
+        """Sum over this rank's rows of r_e^2 (fp64 tensor, one entry per residual)."""
+        return self.loss[:self.ne] * float(self.rows_local)
+
+
+def global_loss(torch, sums, rows_global: int):
+    """Loss vector (L_0..L_{E-1}, sum) from the rank-summed squared-residual sums."""
+    per = sums / float(rows_global)
+    return torch.cat([per, per.sum().reshape(1)])
+
+
+def step_local(ranks: Sequence[SlabRank]):
+    """One loss + gradient step over slabs that all live in this process (one GPU standing in for
+    several: the kernels of different slabs run one after the other, nothing waits on anything)."""
+    plan_list = [r.plan for r in ranks]
+    R = plan_list[0].radius
+    exchange_local(plan_list, [r.fields for r in ranks], 2 * R)
+    for r in ranks:
+        r.fwd()
+    exchange_local(plan_list, [r.res for r in ranks], R)
+    for r in ranks:
+        r.bwd()
+    torch = ranks[0].torch
+    sums = sum(r.loss_sums() for r in ranks)
+    return global_loss(torch, sums, ranks[0].rows_global)
+
+
+def step_dist(rank: SlabRank, dist):
+    """The same step with one slab per process."""
+    R = rank.plan.radius
+    exchange_dist(rank.plan, rank.fields, 2 * R, dist)
+    rank.fwd()
+    exchange_dist(rank.plan, rank.res, R, dist)
+    rank.bwd()
+    sums = rank.loss_sums().clone()
+    if rank.plan.world > 1:
+        dist.all_reduce(sums, op=dist.ReduceOp.SUM)
+    return global_loss(rank.torch, sums, rank.rows_global)

@@ -20,6 +20,7 @@ CASES = [
     ("ns_tgv_128x16", (3, 3, 3, 4)), ("ns_tgv_128x16", (5, 6, 7, 12)),
     ("ns2d_steady_4096", (3, 4)), ("ns2d_steady_4096", (36, 40)),
     ("ns3d_steady_256", (3, 3, 4)), ("ns3d_steady_256", (7, 5, 12)),
+    ("ns_tgv_xslab_34", (3, 3, 3, 4)), ("ns_tgv_xslab_34", (6, 5, 4, 8)),
 ]
 
 

@@ -26,6 +26,8 @@ MEDIUM = [
     ("ns2d_steady_4096", (203, 300)),
     ("ns3d_steady_256", (37, 22, 136)),     # ragged plane chunks, y blocks and a partial warp
     ("ns3d_steady_256", (20, 9, 260)),      # warp edges inside a z line, a ragged column block
+    ("ns_tgv_xslab_34", (34, 21, 20, 16)),  # slab form: first / last x-plane without rows, three plane chunks
+    ("ns_tgv_xslab_34", (17, 8, 8, 12)),    # t groups that straddle warps
 ]
 TINY = [
     ("burgers_256x128", (4, 4)),
@@ -44,6 +46,8 @@ TINY = [
     ("ns3d_steady_256", (3, 3, 4)),
     ("ns3d_steady_256", (5, 6, 8)),
     ("ns3d_steady_256", (7, 5, 132)),
+    ("ns_tgv_xslab_34", (3, 3, 3, 4)),
+    ("ns_tgv_xslab_34", (5, 6, 7, 12)),
 ]
 FULL = [
     ("grayscott_4096", None),

@@ -1,0 +1,70 @@
+"""Slab decomposition on the GPU: several x-slabs of one grid processed in one process (the
+kernels of different slabs run one after the other, halos are copied between the slabs' arrays)
+must reproduce the whole-grid kernels, and the oracle on the whole grid."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2607_18020_b200 import binding as B
+from paper_2607_18020_b200 import slabs as S
+from paper_2607_18020_b200 import workloads as W
+
+from gpu_util import LOSS_TOL, assert_close, run_bwd, run_fwd
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+CASES = [
+    ("ns_tgv_128x16", (16, 8, 8, 8), 1),          # one slab: its halo planes are its own far planes
+    ("ns_tgv_128x16", (16, 8, 8, 8), 2),
+    ("ns_tgv_128x16", (37, 12, 8, 16), 3),        # uneven slabs, several plane chunks per slab
+    ("helmholtz_256", (23, 10, 16), 3),
+    ("poisson_1024", (40, 36), 4),
+    ("ns2d_steady_4096", (30, 40), 2),
+    ("ns3d_steady_256", (14, 6, 8), 3),
+]
+
+
+@pytest.mark.parametrize("name,shape,world", CASES)
+def test_slabs_reproduce_the_whole_grid(name, shape, world):
+    w = W.make(name, seed=42, shape=shape, kind="randn")
+    plan_list = S.plans(w.op, w.shape, world)
+    ranks = [S.SlabRank(torch, B, p, w.spacing, w.coeffs) for p in plan_list]
+    for r in ranks:
+        r.load_owned(w.fields, w.sources)
+    loss = S.step_local(ranks)
+    torch.cuda.synchronize()
+    # assemble the owned planes
+    res = [torch.cat([r.owned(r.res)[e] for r in ranks]).cpu().numpy() for e in range(ranks[0].ne)]
+    grads = [torch.cat([r.owned(r.grads)[f] for r in ranks]).cpu().numpy() for f in range(ranks[0].nf)]
+    # (a) the whole-grid kernels: the same arithmetic per node, so identical bits
+    fields, sources, res_w, loss_w = run_fwd(torch, w)
+    rows = B.row_count(w.op, w.shape)
+    grads_w = run_bwd(torch, w, fields, [r.view for r in res_w], [2.0 / rows] * len(res_w))
+    for e, r in enumerate(res_w):
+        assert np.array_equal(res[e], r.view.cpu().numpy()), "residual %d differs from the whole-grid kernel" % e
+    for f, g in enumerate(grads_w):
+        assert np.array_equal(grads[f], g.view.cpu().numpy()), "gradient %d differs from the whole-grid kernel" % f
+    # (b) the oracle on the whole grid
+    R_ref, loss_ref, g_ref, rows_ref = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    assert rows == rows_ref == sum(r.rows_local for r in ranks)
+    L = loss.cpu().numpy()
+    assert np.all(np.abs(L - loss_ref) <= LOSS_TOL * np.abs(loss_ref) + 1e-300), (L, loss_ref)
+    for e in range(len(res)):
+        assert_close(res[e], R_ref[e], "%s slabs residual %d" % (name, e))
+    for f in range(len(grads)):
+        assert_close(grads[f], g_ref[f], "%s slabs gradient %d" % (name, f))
+
+
+def test_step_dist_with_one_rank():
+    """The per-process step on one rank (no process group needed: a periodic slab's halos are its
+    own far planes)."""
+    w = W.make("ns_tgv_128x16", seed=43, shape=(12, 8, 8, 8), kind="randn")
+    rank = S.SlabRank(torch, B, S.plans(w.op, w.shape, 1)[0], w.spacing, w.coeffs)
+    rank.load_owned(w.fields, w.sources)
+    loss = S.step_dist(rank, dist=None)
+    torch.cuda.synchronize()
+    _, loss_ref, g_ref, _ = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    assert abs(float(loss[-1]) - loss_ref[-1]) <= LOSS_TOL * abs(loss_ref[-1])
+    for f, g in enumerate(rank.owned(rank.grads)):
+        assert_close(g.cpu().numpy(), g_ref[f], "one-rank slab gradient %d" % f)
