@@ -255,6 +255,31 @@ class DeviceProblem:
                             w.coeffs, w.bc, self.ws2)
 
 
+class SlabProblem:
+    """One grid split into x-slabs, one per rank: fwd() = field halo exchange + forward kernel,
+    bwd() = residual halo exchange + adjoint kernel + loss all-reduce."""
+
+    def __init__(self, torch, B, w, world, rank, dist):
+        from paper_2607_18020_b200 import slabs as S
+        self.S, self.dist, self.w = S, dist, w
+        self.rank = S.SlabRank(torch, B, S.plans(w.op, w.shape, world)[rank], w.spacing, w.coeffs)
+        self.rank.load_owned(w.fields, w.sources)
+        self.R = self.rank.plan.radius
+        self.loss = torch.zeros(self.rank.ne + 1, dtype=torch.float64, device="cuda")
+
+    def fwd(self):
+        self.S.exchange_dist(self.rank.plan, self.rank.fields, 2 * self.R, self.dist)
+        self.rank.fwd()
+
+    def bwd(self):
+        self.S.exchange_dist(self.rank.plan, self.rank.res, self.R, self.dist)
+        self.rank.bwd()
+        sums = self.rank.loss_sums().clone()
+        if self.dist is not None:
+            self.dist.all_reduce(sums, op=self.dist.ReduceOp.SUM)
+        self.loss = self.S.global_loss(self.rank.torch, sums, self.rank.rows_global)
+
+
 def timed_steps(torch, prob, steps, warmup, barrier, flush=None, inner_events=False):
     """K back-to-back steps between two events.  With inner_events, every forward and adjoint call
     is bracketed by its own events as well (per-call durations; the extra records sit between
@@ -425,6 +450,9 @@ def main():
     ap.add_argument("--single-pass", action="store_true",
                     help="time fpde_fwd_bwd (one kernel: loss + gradient, residual arrays not stored) as the step; "
                          "only for operators that have a single-pass kernel")
+    ap.add_argument("--slabs", action="store_true",
+                    help="strong scaling: ONE grid split into x-slabs, one per rank, with halo exchange "
+                         "(default: independent replicas, weak scaling)")
     ap.add_argument("--shape", default=None, help="override the grid extents, e.g. 64,128,128,16 (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "fpde" else args.warmup
@@ -453,9 +481,9 @@ def main():
 
     peak, peak_src = measured_peak()
     shape = [int(x) for x in args.shape.split(",")] if args.shape else None
-    w = W.make(args.workload, seed=42 + rank, shape=shape,
+    w = W.make(args.workload, seed=42 if args.slabs else 42 + rank, shape=shape,
                spacing=_spacing_of(args.workload) if shape else None)
-    prob = DeviceProblem(torch, B, w)
+    prob = SlabProblem(torch, B, w, world, rank, dist) if args.slabs else DeviceProblem(torch, B, w)
     if args.single_pass:
         if not B.has_single_pass(w.op):
             raise SystemExit("--single-pass: operator %s has no single-pass kernel" % w.op)
@@ -469,15 +497,17 @@ def main():
     _, fwd_ms, bwd_ms = timed_steps(torch, prob, args.steps, 0, barrier, inner_events=True)
     sampler.stop()
     total_ms = max_over_ranks(total_ms, dist, "cuda")
-    value = job_value(world, N, args.steps, total_ms)
+    value = job_value(1 if args.slabs else world, N, args.steps, total_ms)
 
     e2e_k = max(1, min(args.steps, 20))
-    if args.no_e2e:
+    if args.no_e2e or args.slabs:
         e2e_ms, h2d, d2h = float("nan"), 0, 0
     else:
         e2e_ms, h2d, d2h, _ = e2e_steps(torch, B, w, e2e_k, 3, barrier)
     e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
-    e2e_value = job_value(world, N, e2e_k, e2e_ms)
+    e2e_value = None if e2e_ms != e2e_ms else job_value(world, N, e2e_k, e2e_ms)
+    if e2e_ms != e2e_ms:
+        e2e_ms = None
 
     fb, bb = ALGO_BYTES[w.op]
     knames = KERNEL_NAMES[w.op]
@@ -487,7 +517,8 @@ def main():
         knames = ("fused2d_kernel<%s>" % w.op, "-")
         b_avg = 0.0
     dom = 1 if b_avg >= f_avg else 0
-    dom_bytes = (fb, bb)[dom] * N
+    Nk = N // world if args.slabs else N       # grid points one rank's kernels process (own planes)
+    dom_bytes = (fb, bb)[dom] * Nk
     dom_ms = (f_avg, b_avg)[dom]
     dom_name = knames[dom]
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
@@ -498,22 +529,25 @@ def main():
                 "other_kernel": None if args.single_pass else
                                 {"kernel": knames[1 - dom], "avg_ms": (f_avg, b_avg)[1 - dom],
                                  "note": "forward figure includes the one-block loss finalise launch",
-                                 "achieved": (fb, bb)[1 - dom] * N / ((f_avg, b_avg)[1 - dom] * 1e-3) / 1e9},
-                "pair_achieved": (fb + bb) * N * args.steps / (total_ms * 1e-3) / 1e9,
-                "pair_frac": (fb + bb) * N * args.steps / (total_ms * 1e-3) / 1e9 / peak}
+                                 "achieved": (fb, bb)[1 - dom] * Nk / ((f_avg, b_avg)[1 - dom] * 1e-3) / 1e9},
+                "pair_achieved": (fb + bb) * Nk * args.steps / (total_ms * 1e-3) / 1e9,
+                "pair_frac": (fb + bb) * Nk * args.steps / (total_ms * 1e-3) / 1e9 / peak}
+    if args.slabs:
+        roofline["note"] = "per-call times include the halo exchange of the step (and the loss all-reduce)"
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "strong" if args.slabs else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "operator": w.op, "shape": list(w.shape), "points": N,
                    "fields": len(w.fields), "step": "fpde_fwd_bwd (single pass)" if args.single_pass else "fpde_fwd + fpde_bwd",
-                   "parallelism": "replicas x%d (no exchange step)" % world,
+                   "parallelism": ("x-slabs x%d of one grid, halo exchange per step" if args.slabs
+                                   else "replicas x%d (no exchange step)") % world,
                    "l2": "per-step traffic %.0f MB >> L2, no flush needed" % ((fb + bb) * N / 1e6)
                          if (fb + bb) * N > (256 << 20) else "working set fits L2: warm-cache number"},
         "clocks": sampler.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_k, "ms_per_step": e2e_ms / e2e_k,
+                "steps": e2e_k, "ms_per_step": None if e2e_ms is None else e2e_ms / e2e_k,
                 "what": "fpde_loss_grad_host from pinned host buffers: H2D fields, fwd, bwd, D2H gradients + loss, sync"},
         "gpu_launches": (2 if args.single_pass else LAUNCHES_PER_STEP) * args.steps,
         "roofline": roofline,
