@@ -119,7 +119,6 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
     pdl_wait_then_trigger();
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
-    const int n0 = p.n0;
     const int PS = p.n1 * p.C;                      // plane stride
     const float* __restrict__ f0 = p.f[0];
     const float* __restrict__ f1 = p.f[1];
@@ -205,7 +204,6 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
     pdl_wait_then_trigger();
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
-    const int n0 = p.n0;
     const int PS = p.n1 * p.C;
     // arrays 0..2: u,v,w ; 3..6: upstream of mom_x, mom_y, mom_z, continuity
     const float* const ap[7] = {p.f[0], p.f[1], p.f[2], p.g[0], p.g[1], p.g[2], p.g[3]};
