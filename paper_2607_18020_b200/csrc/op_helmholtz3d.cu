@@ -194,7 +194,7 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     int ty = env_int("FPDE_STAR3D_TY", 2);
     ty = std::max(1, std::min(256 / tx, ty));
     block = dim3(tx, ty, 1);
-    p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 16);
+    p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 12);
     p.ncb = (p.nc4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
@@ -207,7 +207,7 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     }
     p.kc = sp((q.coef[0] * q.coef[0] - 30.0 * wsum) * scale);
     const char* pf = std::getenv("FPDE_STAR3D_PREFETCH");
-    p.prefetch = pf && *pf ? std::atoi(pf) : 2;
+    p.prefetch = pf && *pf ? std::atoi(pf) : 1;
     if (p.prefetch < 0) p.prefetch = 0;
 }
 

@@ -199,8 +199,8 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
 //   g_p(P) = sum_q [ G_q(P-a_q) - G_q(P+a_q) ] / (2 h_{a_q})
 // G_e = gscale_e * gres_e; the scales are folded into the constants.
 // ------------------------------------------------------------------------------------------
-template <bool TSAFE, int MINB>
-__global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
+template <bool TSAFE, int MINB, int THREADS = 128>
+__global__ void __launch_bounds__(THREADS, MINB) ns_bwd_kernel(const NsParams p) {
     pdl_wait_then_trigger();
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
@@ -268,20 +268,21 @@ static int env_int(const char* name, int dflt) {
     return v > 0 ? v : dflt;
 }
 
-static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
+static void ns_geometry(const Problem& q, NsParams& p, dim3& block, int ty_override = 0) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n3 = q.n[3];
     p.C = q.n[2] * q.n[3]; p.C4 = p.C / 4; p.nt4 = q.n[3] / 4;
-    int tx = env_int("FPDE_NS_TX", 32);
+    int tx = env_int("FPDE_NS_TX", p.C4 % 64 == 0 ? 64 : 32);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
-    int ty = env_int("FPDE_NS_TY", 4);
+    int ty = env_int("FPDE_NS_TY", 128 / tx);
     ty = std::max(1, std::min(128 / tx, ty));
+    if (ty_override > 0) ty = ty_override;
     block = dim3(tx, ty, 1);
-    p.planes_per_item = env_int("FPDE_NS_PLANES", 16);
+    p.planes_per_item = env_int("FPDE_NS_PLANES", 24);
     p.ncb = (p.C4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     const char* pf = std::getenv("FPDE_NS_PREFETCH");
-    p.prefetch = pf && *pf ? std::atoi(pf) : 1;
+    p.prefetch = pf && *pf ? std::atoi(pf) : 2;
     if (p.prefetch < 0 || p.prefetch >= p.n0) p.prefetch = 0;
     p.xint = q.bc0_interior ? 1 : 0;
 }
@@ -325,12 +326,14 @@ cudaError_t launch_ns_bwd(const Problem& q) {
         if (launched || ce != cudaSuccess) return ce;
     }
     NsParams p{}; dim3 block;
-    ns_geometry(q, p, block);
+    const int ty_b = env_int("FPDE_NS_BWD_TY", 0);        // 8: one 256-thread block per SM (experiment)
+    ns_geometry(q, p, block, ty_b == 8 ? 8 : 0);
     for (int k = 0; k < 4; ++k) { p.f[k] = q.in[k]; p.g[k] = q.aux[k]; p.out[k] = q.out[k]; }
     ns_fill_consts(p.k, q.h, q.coef[0], q.gscale);
     p.partials = nullptr;
     const int minb = env_int("FPDE_NS_MINB_B", 2);
     cudaError_t ce;
+    if (ty_b == 8 && ns_tsafe(p) && block.x == 32) return launch_kernel(ns_bwd_kernel<true, 1, 256>, dim3(p.nitems), block, q.stream, p);
     if (!ns_tsafe(p)) ce = launch_kernel(ns_bwd_kernel<false, 2>, dim3(p.nitems), block, q.stream, p);
     else if (minb == 3) ce = launch_kernel(ns_bwd_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
     else ce = launch_kernel(ns_bwd_kernel<true, 2>, dim3(p.nitems), block, q.stream, p);
