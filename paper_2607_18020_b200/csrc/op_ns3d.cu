@@ -176,6 +176,14 @@ __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     const int a1 = min(a0 + p.planes_per_item, p.n0);
     t.a1 = a1;
 
+    // the planes the first steps load are not covered by the per-step prefetch: ask for them now
+    if (p.prefetch > 0 && (threadIdx.x & 7) == 0) {
+        for (int d = 1; d <= p.prefetch && a0 + d <= min(a1, p.n0 - 1); ++d) {
+            const int po = (a0 + d) * t.PS + t.rowoff;
+#pragma unroll
+            for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(p.a[k] + po);
+        }
+    }
     V4 A[NA], B[NA], Cc[NA];
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
