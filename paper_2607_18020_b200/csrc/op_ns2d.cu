@@ -35,6 +35,7 @@ struct Ns2dParams {
     int n0, n1, nc4;
     int rows_per_item, ncb, nitems;
     float* partials;
+    int prefetch;           // rows ahead of the window to pull into L2 (0 = off)
 };
 
 template <bool BWD>
@@ -71,6 +72,14 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
         return v;
     };
 
+    auto prefetch_row = [&](int r) {                 // one lane per 128-byte line
+        if ((threadIdx.x & 7) == 0 && cvalid && r < n0) {
+#pragma unroll
+            for (int k = 0; k < NA; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.in[k] + r * n1 + col));
+        }
+    };
+    if (p.prefetch > 0)
+        for (int d = 1; d <= p.prefetch; ++d) if (a0 + d <= a1) prefetch_row(a0 + d);
     V4 prev[NA], cur[NA], nxt[NA];
 #pragma unroll
     for (int k = 0; k < NA; ++k) { prev[k] = load(k, a0 - 1); cur[k] = load(k, a0); }
@@ -79,6 +88,7 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
     for (int e = 0; e < 3; ++e) acc[e] = make_float2(0.f, 0.f);
 
     for (int row = a0; row < a1; ++row) {
+        if (p.prefetch > 0 && row + 1 + p.prefetch <= a1) prefetch_row(row + 1 + p.prefetch);
         V4 L[NA], R[NA];
         float E[NA];
 #pragma unroll
@@ -202,6 +212,9 @@ static void ns2d_geometry(const int* n, Ns2dParams& p, int& block) {
     p.rows_per_item = env_int("FPDE_NS2D_ROWS", 4);
     p.ncb = (p.nc4 + block - 1) / block;
     p.nitems = p.ncb * ((p.n0 + p.rows_per_item - 1) / p.rows_per_item);
+    const char* pf = std::getenv("FPDE_NS2D_PREFETCH");
+    p.prefetch = pf && *pf ? std::atoi(pf) : 1;
+    if (p.prefetch < 0) p.prefetch = 0;
 }
 
 int ns2d_items(const int* n) {
