@@ -38,7 +38,6 @@ struct Lap2dParams {
     int n0, n1, nc4;
     int rows_per_item, ncb, nitems;
     float* partials;
-    int prefetch;        // pull the next batch of rows into L2 while this one is worked on (0 = off)
 };
 
 // out = -Lap u - f
@@ -144,23 +143,6 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
     const float2 m2 = splat2(-2.f);
 
     for (int a = a0; a < a1; a += U) {
-        if (p.prefetch && cvalid && (threadIdx.x & 7) == 0) {      // one lane per 128-byte line
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int r = a + U + u + 1;                        // halo-input rows of the next batch
-                if (r <= a1) {
-                    const int rr = in_row(r);
-                    if (rr >= 0) {
-#pragma unroll
-                        for (int k = 0; k < NH; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.hin[k] + rr * n1 + col));
-                    }
-                    if (r - 1 < a1) {
-#pragma unroll
-                        for (int k = 0; k < NC; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.cin[k] + (r - 1) * n1 + col));
-                    }
-                }
-            }
-        }
         V4 nxt[U][NH];
         V4 cen[U][NCA];
         float le[U][NH], re[U][NH];
@@ -255,8 +237,6 @@ static void lap2d_geometry(const Problem& q, Lap2dParams& p, int& block) {
     const float ih0 = (float)(1.0 / (q.h[0] * q.h[0])), ih1 = (float)(1.0 / (q.h[1] * q.h[1]));
     p.ih0 = make_float2(ih0, ih0);
     p.ih1 = make_float2(ih1, ih1);
-    const char* pf = std::getenv("FPDE_LAP2D_PREFETCH");
-    p.prefetch = pf && *pf ? std::atoi(pf) : 1;
 }
 
 int lap2d_items(const int* n) {
