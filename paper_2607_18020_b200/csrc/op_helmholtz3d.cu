@@ -186,7 +186,7 @@ static int env_int(const char* name, int dflt) {
 
 static float2 sp(double v) { return make_float2((float)v, (float)v); }
 
-static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, double scale) {
+static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, double scale, bool fwd) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n2 = q.n[2]; p.nc4 = q.n[2] / 4;
     int tx = p.nc4 > 32 ? 64 : 32;
     tx = env_int("FPDE_STAR3D_TX", tx);
@@ -194,7 +194,8 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     int ty = env_int("FPDE_STAR3D_TY", 2);
     ty = std::max(1, std::min(256 / tx, ty));
     block = dim3(tx, ty, 1);
-    p.planes_per_item = env_int("FPDE_STAR3D_PLANES", 12);
+    // the forward kernel (two input streams) runs best on long items, the adjoint on short ones
+    p.planes_per_item = fwd ? env_int("FPDE_STAR3D_PLANES_F", 32) : env_int("FPDE_STAR3D_PLANES_B", 10);
     p.ncb = (p.nc4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
@@ -214,13 +215,13 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
 int star3d_items(const int* n) {
     Problem q{}; q.n[0] = n[0]; q.n[1] = n[1]; q.n[2] = n[2]; q.h[0] = q.h[1] = q.h[2] = 1.0;
     Star3dParams p{}; dim3 block;
-    star3d_geometry(q, p, block, 1.0);
+    star3d_geometry(q, p, block, 1.0, true);
     return p.nitems;
 }
 
 cudaError_t launch_helmholtz_fwd(const Problem& q) {
     Star3dParams p{}; dim3 block;
-    star3d_geometry(q, p, block, 1.0);
+    star3d_geometry(q, p, block, 1.0, true);
     p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0];
     p.partials = q.partials;
     if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<true, 4>, dim3(p.nitems), block, q.stream, p);
@@ -229,7 +230,7 @@ cudaError_t launch_helmholtz_fwd(const Problem& q) {
 
 cudaError_t launch_helmholtz_bwd(const Problem& q) {
     Star3dParams p{}; dim3 block;
-    star3d_geometry(q, p, block, q.gscale[0]);      // the operator is linear: the scale goes into the weights
+    star3d_geometry(q, p, block, q.gscale[0], false);      // the operator is linear: the scale goes into the weights
     p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0];
     p.partials = nullptr;
     if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<false, 4>, dim3(p.nitems), block, q.stream, p);
