@@ -109,6 +109,48 @@ def test_argument_validation_without_a_gpu():
     assert callb(bc=(W.PERIODIC, W.ONE_SIDED)) == 8
 
 
+def test_fwd_bwd_and_f64_validation_without_a_gpu():
+    """The loss-specialised pass and the fp64 path check their arguments before any launch."""
+    P = 0x1000
+    ok = dict(op=W.GRAYSCOTT_2D, fields=[P, P], sources=None, residuals=None, gfields=[P, P], loss_out=None,
+              shape=(8, 8), spacing=(0.1, 0.1), coeffs=(1, 1, 1, 1), bc=(W.PERIODIC, W.PERIODIC), workspace=None,
+              workspace_bytes_=0, stream=None)
+    def call(**kw):
+        a = dict(ok); a.update(kw)
+        return B.fwd_bwd_status(**a)
+    assert B.has_single_pass(W.GRAYSCOTT_2D) and B.has_single_pass(W.POISSON_2D) and B.has_single_pass(W.NS_2D_STEADY)
+    assert not B.has_single_pass(W.NS_3D_T) and not B.has_single_pass(W.HELMHOLTZ_3D_O4)
+    assert call(op=23) == 1
+    assert call(gfields=None) == 2
+    assert call(gfields=[P, None]) == 2
+    assert call(residuals=[P + 4, None]) == 5            # an optional residual array, if given, must be aligned
+    assert call(gfields=[P, P + 8]) == 5
+    assert call(shape=(8, 10)) == 4
+    assert call(coeffs=(1, 1, 1)) == 7
+    assert call(loss_out=P) == 9                          # loss wanted, no workspace
+    assert call(loss_out=P, workspace=P, workspace_bytes_=4) == 9
+    # operators without a single-pass kernel need every residual array
+    assert call(op=W.HELMHOLTZ_3D_O4, fields=[P], sources=[P], gfields=[P], shape=(8, 8, 8), spacing=(.1, .1, .1),
+                coeffs=(1.0,), bc=(W.INTERIOR,) * 3) == 2
+    assert call(op=W.HELMHOLTZ_3D_O4, fields=[P], sources=[P], residuals=[None], gfields=[P], shape=(8, 8, 8),
+                spacing=(.1, .1, .1), coeffs=(1.0,), bc=(W.INTERIOR,) * 3) == 2
+    # workspace sizes are host-only queries and do not depend on a device being present
+    assert 0 < B.fwd_bwd_workspace_bytes(W.GRAYSCOTT_2D, (4096, 4096)) < (1 << 20)
+    assert B.fwd_bwd_workspace_bytes(W.NS_3D_T, (128, 128, 128, 16)) == B.workspace_bytes(W.NS_3D_T, (128, 128, 128, 16))
+    assert 0 < B.workspace_bytes_f64(W.HELMHOLTZ_3D_O4, (64, 64, 64)) < (1 << 20)
+    L = B.lib()
+    import ctypes
+    vpp = ctypes.POINTER(ctypes.c_void_p)
+    one = (ctypes.c_void_p * 1)(P)
+    sh = (ctypes.c_int64 * 2)(16, 16); h = (ctypes.c_double * 2)(0.1, 0.1); bc = (ctypes.c_int * 2)(1, 1)
+    st = L.fpde_fwd_f64(1, ctypes.cast(one, vpp), ctypes.cast(one, vpp), None, None, 2, sh, h, None, 0, bc, None, 0, None)
+    assert st == 2                                        # residuals missing
+    st = L.fpde_bwd_f64(1, ctypes.cast(one, vpp), None, None, ctypes.cast(one, vpp), 2, sh, h, None, 0, bc, None)
+    assert st == 2
+    st = L.fpde_bwd_f64(1, ctypes.cast(one, vpp), ctypes.cast(one, vpp), None, ctypes.cast(one, vpp), 3, sh, h, None, 0, bc, None)
+    assert st == 3
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
     monkeypatch.setattr(B, "_lib", None)
