@@ -314,7 +314,12 @@ static int sm_count() {
     return n;
 }
 
-static int fused2d_blocks_per_sm(int op) { return op == 1 ? 4 : (op == 2 ? 3 : 2); }
+static int fused2d_minb(int op) {                   // resident blocks per SM the kernel is compiled for
+    const int dflt = op == 1 ? 4 : (op == 2 ? 4 : 3);
+    const int v = env_int("FPDE_FUSED2D_MINB", dflt);
+    return op == 1 ? 4 : (op == 2 ? (v == 3 ? 3 : 4) : (v == 2 ? 2 : 3));
+}
+static int fused2d_blocks_per_sm(int op) { return fused2d_minb(op); }
 
 // Rows per work item: every item recomputes r on two extra rows, and the last wave of items
 // should be nearly full; pick the row count with the smallest (waves x rows marched per item).
@@ -369,11 +374,13 @@ cudaError_t launch_fused2d(const Problem& q, float* const* res) {
         for (int k = 0; k < 2; ++k) { p.f[k] = q.in[k]; p.g[k] = q.out[k]; p.res[k] = res ? res[k] : nullptr; }
         p.c[0] = sp(1.0 / (h0 * h0)); p.c[1] = sp(1.0 / (h1 * h1));
         p.c[2] = sp(q.coef[0]); p.c[3] = sp(q.coef[1]); p.c[4] = sp(q.coef[2]); p.c[5] = sp(q.coef[2] + q.coef[3]);
-        return launch_kernel(fused2d_kernel<FusedGrayScott, 3>, dim3(p.nitems), dim3(128), q.stream, p);
+        if (fused2d_minb(2) == 3) return launch_kernel(fused2d_kernel<FusedGrayScott, 3>, dim3(p.nitems), dim3(128), q.stream, p);
+        return launch_kernel(fused2d_kernel<FusedGrayScott, 4>, dim3(p.nitems), dim3(128), q.stream, p);
     case 5:
         for (int k = 0; k < 3; ++k) { p.f[k] = q.in[k]; p.g[k] = q.out[k]; p.res[k] = res ? res[k] : nullptr; }
         p.c[0] = sp(0.5 / h0); p.c[1] = sp(0.5 / h1);
         p.c[2] = sp(-q.coef[0] / (h0 * h0)); p.c[3] = sp(-q.coef[0] / (h1 * h1));
+        if (fused2d_minb(5) == 3) return launch_kernel(fused2d_kernel<FusedNs2d, 3>, dim3(p.nitems), dim3(128), q.stream, p);
         return launch_kernel(fused2d_kernel<FusedNs2d, 2>, dim3(p.nitems), dim3(128), q.stream, p);
     }
     return cudaErrorInvalidValue;
