@@ -51,6 +51,16 @@ def test_near_max_size_sampled_windows(op, shape, h, c, bc, ext):
     B.fpde_fwd(op, fields, sources, res, loss, shape, h, c, bc, ws)
     B.fpde_bwd(op, fields, res, gs, grads, shape, h, c, bc)
     torch.cuda.synchronize()
+    grad_sets = [("pair", grads)]
+    if B.has_single_pass(op) and torch.cuda.mem_get_info()[0] > info.nfields * need + (2 << 30):
+        # the single-pass kernel on the same grid: same loss, gradients checked on the same windows
+        grads1 = [torch.empty(shape, dtype=torch.float32, device="cuda") for _ in range(info.nfields)]
+        loss1 = torch.zeros(info.nresiduals + 1, dtype=torch.float64, device="cuda")
+        ws1 = torch.empty(B.fwd_bwd_workspace_bytes(op, shape), dtype=torch.uint8, device="cuda")
+        B.fpde_fwd_bwd(op, fields, sources, None, grads1, loss1, shape, h, c, bc, ws1)
+        torch.cuda.synchronize()
+        assert torch.all((loss1 - loss).abs() <= 1e-6 * loss.abs())
+        grad_sets.append(("single pass", grads1))
     # the reducer against a library reduction of the residuals it was given
     for e, r in enumerate(res):
         ref = float((r.double() ** 2).sum().item()) / rows
@@ -87,10 +97,11 @@ def test_near_max_size_sampled_windows(op, shape, h, c, bc, ext):
                 keep = (idx >= 2 * info.radius) & (idx < n - 2 * info.radius)
                 shp = [1] * len(ext); shp[a] = ext[a]
                 band_free &= keep.reshape(shp)
-        for f, (g, gg) in enumerate(zip(grads, G)):
-            got = g[sl].cpu().numpy()
-            mask = band_free[inner]
-            if mask.any():
-                assert_close(got[inner][mask], gg[inner][mask], "window %s gradient %d" % (w0, f))
-    del fields, sources, res, grads
+        for tag, gset in grad_sets:
+            for f, (g, gg) in enumerate(zip(gset, G)):
+                got = g[sl].cpu().numpy()
+                mask = band_free[inner]
+                if mask.any():
+                    assert_close(got[inner][mask], gg[inner][mask], "%s: window %s gradient %d" % (tag, w0, f))
+    del fields, sources, res, grads, grad_sets
     torch.cuda.empty_cache()
