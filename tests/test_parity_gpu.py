@@ -124,7 +124,7 @@ def test_unequal_spacing():
 
 @pytest.mark.parametrize("name,shape", FULL)
 def test_full_size_configs(name, shape):
-    """BASELINE's full sizes in the launch configuration the bench times; the C oracle is fast
+    """The configurations' full sizes in the launch configuration the bench times; the C oracle is fast
     enough to check every element."""
     _check_case(W.make(name, seed=42), name + " full size")
 
