@@ -270,6 +270,12 @@ int fpde_bwd_f64(int op,
  *   d_arena    DEVICE scratch of at least fpde_host_arena_bytes() bytes, 256-byte aligned, owned
  *              by the caller (staging for fields, sources, residuals, gradients, loss, workspace)
  * Same status codes as fpde_fwd / fpde_bwd; FPDE_ERR_WORKSPACE if the arena is too small.
+ * For FPDE_OP_NS_3D_T on grids of six or more 8-plane chunks the call is pipelined: chunks of
+ * x-planes are copied up on one internal stream, run through forward and adjoint launches over
+ * chunk ranges on `stream`, and copied down on a second internal stream, so the two copy
+ * directions overlap; `stream` waits for both internal streams before the call's work counts as
+ * done on it, so synchronising `stream` is still all a caller has to do.  (FPDE_HOST_PIPELINE=0
+ * in the environment selects the plain one-stream form.)
  */
 size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape);
 int fpde_loss_grad_host(int op,

@@ -9,12 +9,13 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 namespace fpde {
 
 int lap2d_items(const int* n);
 int star3d_items(const int* n);
-int ns_items(const int* n, bool xint);
+int ns_items(const int* n, bool xint, int planes_per_item = 0);
 int burgers_items(const int* n);
 int ns2d_items(const int* n);
 int ns3d_items(const int* n);
@@ -462,13 +463,150 @@ int fpde_bwd_f64(int op, const double* const* fields, const double* const* gres,
 
 static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 
+// scratch the host-buffer call needs: the loss partial sums of whichever launch shape it uses
+static size_t host_workspace_bytes(int op, int ndim, const int64_t* shape) {
+    size_t need = fpde_fwd_bwd_workspace_bytes(op, ndim, shape);
+    int n[MAX_D] = {0, 0, 0, 0};
+    if (op == FPDE_OP_NS_3D_T && check_shape(op, ndim, shape, n, nullptr, nullptr) == FPDE_OK)
+        need = std::max(need, round256((size_t)ns_items(n, false, 4) * REGISTRY[op].ne * sizeof(float)) + 4096);
+    return need;
+}
+
 size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape) {
     int64_t N = 0;
     if (check_shape(op, ndim, shape, nullptr, &N, nullptr) != FPDE_OK) return 0;
     const OpEntry& e = REGISTRY[op];
     const size_t arr = round256((size_t)N * sizeof(float));
     return arr * (size_t)(2 * e.nf + e.ns + e.ne) + round256((e.ne + 1) * sizeof(double))
-         + fpde_fwd_bwd_workspace_bytes(op, ndim, shape);
+         + host_workspace_bytes(op, ndim, shape);
+}
+
+// ------------------------------------------------------------------------------------------
+// fpde_loss_grad_host, pipelined form for the unsteady Navier-Stokes operator.
+//
+// The plain form queues H2D(all fields) -> kernels -> D2H(all gradients) on one stream, so the two
+// copy directions never overlap and the step costs T_in + T_out.  Here the grid is cut into K
+// chunks of x-planes: the fields of a chunk go up on a copy stream, the forward kernel of chunk c
+// runs (on the caller's stream) as soon as chunks c-1, c, c+1 have arrived, the adjoint of chunk c
+// as soon as the residuals of c-1, c, c+1 exist, and its gradients go down on a second copy
+// stream while later chunks are still coming up.  Kernels are the ordinary ones launched over a
+// range of plane chunks (they read their x neighbours from the full arrays, periodic wrap
+// included, and write only their own planes), so nothing is copied or recomputed on the device.
+// Because of the periodic wrap the last chunk is sent first; the adjoint of the first and the
+// last two chunks has to wait for the last forward launch, so about 4/K of the D2H time stays
+// exposed.  The caller's stream waits for both copy streams at the end: synchronising it covers
+// everything, as in the plain form.
+// ------------------------------------------------------------------------------------------
+static constexpr int HOST_PIPE_MIN_PLANES = 4;      // smallest chunk the pipeline may use (host_workspace_bytes sizes for it)
+static int host_pipe_planes() {                     // planes per work item and per chunk
+    const char* s = std::getenv("FPDE_HOST_PIPE_PLANES");
+    const int v = s && *s ? std::atoi(s) : 8;
+    return std::max(HOST_PIPE_MIN_PLANES, std::min(64, v));
+}
+static std::mutex g_pipe_mutex;
+static cudaStream_t g_pipe_in[64], g_pipe_out[64];
+
+static bool host_pipeline_wanted(int op, const int* n) {
+    const char* s = std::getenv("FPDE_HOST_PIPELINE");
+    if (s && s[0] == '0') return false;
+    const int P = host_pipe_planes();
+    return op == FPDE_OP_NS_3D_T && (n[0] + P - 1) / P >= 6;
+}
+
+static cudaError_t host_pipeline_streams(cudaStream_t* in, cudaStream_t* out) {
+    int dev = 0;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce != cudaSuccess) return ce;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    if (g_pipe_in[dev] == nullptr) {
+        cudaStream_t a = nullptr, b = nullptr;
+        ce = cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking);
+        if (ce != cudaSuccess) return ce;
+        ce = cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking);
+        if (ce != cudaSuccess) { cudaStreamDestroy(a); return ce; }
+        g_pipe_in[dev] = a; g_pipe_out[dev] = b;
+    }
+    *in = g_pipe_in[dev]; *out = g_pipe_out[dev];
+    return cudaSuccess;
+}
+
+// q: validated problem with device arrays set (in = fields, out unused); d_r / d_g device arrays
+static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, float* const* h_gfields, double* h_loss,
+                                    float* const* d_f, float* const* d_r, float* const* d_g, double* d_loss,
+                                    void* d_ws, int nf, int ne) {
+    cudaStream_t cs = q.stream, s_in = nullptr, s_out = nullptr;
+    if (host_pipeline_streams(&s_in, &s_out) != cudaSuccess) return FPDE_ERR_CUDA;
+    const int n0 = q.n[0];
+    const int64_t plane = (int64_t)q.n[1] * q.n[2] * q.n[3];
+    const int HOST_PIPE_PLANES = host_pipe_planes();
+    const int K = (n0 + HOST_PIPE_PLANES - 1) / HOST_PIPE_PLANES;
+    std::vector<cudaEvent_t> ev(2 * K + 2, nullptr);
+    auto cleanup = [&]() { for (cudaEvent_t e : ev) if (e) cudaEventDestroy(e); };
+    for (auto& e : ev)
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cleanup(); return FPDE_ERR_CUDA; }
+    cudaEvent_t* e_in = ev.data();           // chunk c has arrived
+    cudaEvent_t* e_bwd = ev.data() + K;      // gradients of chunk c are complete
+    cudaEvent_t e_start = ev[2 * K], e_done = ev[2 * K + 1];
+    bool ok = true;
+    auto chk = [&](cudaError_t ce) { ok = ok && ce == cudaSuccess; };
+    auto p0 = [&](int c) { return (int64_t)c * HOST_PIPE_PLANES; };
+    auto np = [&](int c) { return (int64_t)std::min(HOST_PIPE_PLANES, n0 - c * HOST_PIPE_PLANES); };
+
+    // the copy streams start after whatever the caller queued before this call
+    chk(cudaEventRecord(e_start, cs));
+    chk(cudaStreamWaitEvent(s_in, e_start, 0));
+    chk(cudaStreamWaitEvent(s_out, e_start, 0));
+    // fields up: last chunk first (the first chunk's forward needs it through the periodic wrap)
+    for (int i = 0; i < K; ++i) {
+        const int c = i == 0 ? K - 1 : i - 1;
+        const size_t off = (size_t)(p0(c) * plane), bytes = (size_t)(np(c) * plane) * sizeof(float);
+        for (int f = 0; f < nf; ++f)
+            chk(cudaMemcpyAsync(d_f[f] + off, h_fields[f] + off, bytes, cudaMemcpyHostToDevice, s_in));
+        chk(cudaEventRecord(e_in[c], s_in));
+    }
+    q.planes_per_item = HOST_PIPE_PLANES;
+    q.partials = static_cast<float*>(d_ws);
+    q.loss_out = d_loss;
+    for (int f = 0; f < nf; ++f) q.in[f] = d_f[f];
+    auto fwd = [&](int c) {
+        for (int d = -1; d <= 1; ++d) chk(cudaStreamWaitEvent(cs, e_in[(c + d + K) % K], 0));
+        Problem r = q;
+        for (int e = 0; e < ne; ++e) r.out[e] = d_r[e];
+        r.chunk_lo = c; r.chunk_hi = c + 1;
+        chk(launch_ns_fwd(r));
+    };
+    auto bwd = [&](int c) {
+        Problem r = q;
+        for (int e = 0; e < ne; ++e) { r.aux[e] = d_r[e]; r.gscale[e] = 2.0 / (double)q.rows; }
+        for (int f = 0; f < nf; ++f) r.out[f] = d_g[f];
+        r.partials = nullptr;
+        r.chunk_lo = c; r.chunk_hi = c + 1;
+        chk(launch_ns_bwd(r));
+        chk(cudaEventRecord(e_bwd[c], cs));
+        chk(cudaStreamWaitEvent(s_out, e_bwd[c], 0));
+        const size_t off = (size_t)(p0(c) * plane), bytes = (size_t)(np(c) * plane) * sizeof(float);
+        for (int f = 0; f < nf; ++f)
+            chk(cudaMemcpyAsync(h_gfields[f] + off, d_g[f] + off, bytes, cudaMemcpyDeviceToHost, s_out));
+    };
+    // forward of chunk c once c+1 is there; adjoint of chunk c once the forward of c+1 is queued
+    // (chunk 0's adjoint needs the last chunk's residuals and comes at the end)
+    fwd(0);
+    for (int c = 1; c <= K - 2; ++c) {
+        fwd(c);
+        if (c >= 2) bwd(c - 1);
+    }
+    fwd(K - 1);
+    chk(launch_loss_finalize(q.partials, ns_items(q.n, false, HOST_PIPE_PLANES), ne, q.rows, d_loss, cs));
+    bwd(K - 2);
+    bwd(K - 1);
+    bwd(0);
+    chk(cudaMemcpyAsync(h_loss, d_loss, (ne + 1) * sizeof(double), cudaMemcpyDeviceToHost, cs));
+    // the caller's stream covers the copy streams
+    chk(cudaEventRecord(e_done, s_out));
+    chk(cudaStreamWaitEvent(cs, e_done, 0));
+    cleanup();
+    return ok ? FPDE_OK : FPDE_ERR_CUDA;
 }
 
 int fpde_loss_grad_host(int op, const float* const* h_fields, const float* const* h_sources,
@@ -502,8 +640,20 @@ int fpde_loss_grad_host(int op, const float* const* h_fields, const float* const
     for (int f = 0; f < e.nf; ++f) { d_g[f] = reinterpret_cast<float*>(base); base += arr; }
     double* d_loss = reinterpret_cast<double*>(base); base += round256((e.ne + 1) * sizeof(double));
     void* d_ws = base;
-    const size_t ws_bytes = fpde_fwd_bwd_workspace_bytes(op, ndim, shape);
+    const size_t ws_bytes = host_workspace_bytes(op, ndim, shape);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    {
+        int n[MAX_D] = {0, 0, 0, 0};
+        check_shape(op, ndim, shape, n, nullptr, nullptr);
+        if (host_pipeline_wanted(op, n)) {
+            Problem q;
+            std::memset(&q, 0, sizeof(q));
+            st = validate(op, d_f, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
+            if (st != FPDE_OK) return st;
+            q.stream = cs;
+            return loss_grad_host_pipelined(q, h_fields, h_gfields, h_loss, d_f, d_r, d_g, d_loss, d_ws, e.nf, e.ne);
+        }
+    }
     for (int f = 0; f < e.nf; ++f)
         if (cudaMemcpyAsync(d_f[f], h_fields[f], bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FPDE_ERR_CUDA;
     for (int s = 0; s < e.ns; ++s)

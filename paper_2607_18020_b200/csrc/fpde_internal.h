@@ -26,6 +26,10 @@ struct Problem {
     int64_t rows;            // N_r
     cudaStream_t stream;
     bool bc0_interior;       // unsteady NS only: x axis not periodic (the slab form of the operator)
+    // unsteady NS only: planes per work item (0 = the launcher's default) and the range of plane
+    // chunks this launch covers (chunk_hi <= chunk_lo = all); the loss partial sums keep their
+    // global slots, so several ranged launches add up to one full launch
+    int planes_per_item, chunk_lo, chunk_hi;
 };
 
 // The same for the double-precision verification path (ops_f64.cu).

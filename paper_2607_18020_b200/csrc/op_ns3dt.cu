@@ -38,6 +38,7 @@ struct NsParams {
     int n0, n1, n3;       // x, y extents; t extent
     int C, C4, nt4;       // row length in floats / float4, float4 per z
     int planes_per_item, ncb, nmb, nitems;
+    int item_offset;      // first work item of this launch (launches over a range of plane chunks)
     NsConsts k;
     float* partials;
     int prefetch;         // planes ahead of the window to prefetch into L2 (0 = off)
@@ -74,7 +75,7 @@ __device__ __forceinline__ void prefetch_l2(const float* ptr) {
 
 __device__ __forceinline__ NsIndex ns_index(const NsParams& p, int& a0, int& a1) {
     NsIndex ix;
-    int item = blockIdx.x;
+    int item = blockIdx.x + p.item_offset;
     const int cb = item % p.ncb; item /= p.ncb;
     const int mb = item % p.nmb;
     const int ab = item / p.nmb;
@@ -184,7 +185,7 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
         float s[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) s[e] = acc[e].x + acc[e].y;
-        block_reduce_store<4>(s, p.partials, p.nitems, blockIdx.x);
+        block_reduce_store<4>(s, p.partials, p.nitems, blockIdx.x + p.item_offset);
     }
 }
 
@@ -199,8 +200,8 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
 //   g_p(P) = sum_q [ G_q(P-a_q) - G_q(P+a_q) ] / (2 h_{a_q})
 // G_e = gscale_e * gres_e; the scales are folded into the constants.
 // ------------------------------------------------------------------------------------------
-template <bool TSAFE, int MINB, int THREADS = 128>
-__global__ void __launch_bounds__(THREADS, MINB) ns_bwd_kernel(const NsParams p) {
+template <bool TSAFE, int MINB>
+__global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
     pdl_wait_then_trigger();
     int a0, a1;
     const NsIndex ix = ns_index(p, a0, a1);
@@ -268,16 +269,15 @@ static int env_int(const char* name, int dflt) {
     return v > 0 ? v : dflt;
 }
 
-static void ns_geometry(const Problem& q, NsParams& p, dim3& block, int ty_override = 0) {
+static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n3 = q.n[3];
     p.C = q.n[2] * q.n[3]; p.C4 = p.C / 4; p.nt4 = q.n[3] / 4;
     int tx = env_int("FPDE_NS_TX", p.C4 % 64 == 0 ? 64 : 32);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
     int ty = env_int("FPDE_NS_TY", 128 / tx);
     ty = std::max(1, std::min(128 / tx, ty));
-    if (ty_override > 0) ty = ty_override;
     block = dim3(tx, ty, 1);
-    p.planes_per_item = env_int("FPDE_NS_PLANES", 24);
+    p.planes_per_item = q.planes_per_item > 0 ? q.planes_per_item : env_int("FPDE_NS_PLANES", 24);
     p.ncb = (p.C4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
@@ -289,18 +289,31 @@ static void ns_geometry(const Problem& q, NsParams& p, dim3& block, int ty_overr
 
 static bool ns_tsafe(const NsParams& p) { return 32 % p.nt4 == 0; }
 
-int ns_items(const int* n, bool xint) {
-    if (!xint && ns_tma_wanted(n)) return ns_tma_items(n);
+// Grid of a launch: all work items, or those of the plane chunks [chunk_lo, chunk_hi) of the
+// problem (items are ordered with the plane chunk slowest, so a chunk range is an item range).
+static dim3 ns_range(const Problem& q, NsParams& p) {
+    const int per_chunk = p.ncb * p.nmb;
+    if (q.chunk_hi > q.chunk_lo) {
+        p.item_offset = q.chunk_lo * per_chunk;
+        return dim3((q.chunk_hi - q.chunk_lo) * per_chunk);
+    }
+    p.item_offset = 0;
+    return dim3(p.nitems);
+}
+
+int ns_items(const int* n, bool xint, int planes_per_item) {
+    if (!xint && planes_per_item == 0 && ns_tma_wanted(n)) return ns_tma_items(n);
     Problem q{};
     for (int a = 0; a < 4; ++a) { q.n[a] = n[a]; q.h[a] = 1.0; }
     q.bc0_interior = xint;
+    q.planes_per_item = planes_per_item;
     NsParams p{}; dim3 block;
     ns_geometry(q, p, block);
     return p.nitems;
 }
 
 cudaError_t launch_ns_fwd(const Problem& q) {
-    if (!q.bc0_interior) {
+    if (!q.bc0_interior && q.planes_per_item == 0) {
         bool launched = false;
         const cudaError_t ce = launch_ns_fwd_tma(q, launched);
         if (launched || ce != cudaSuccess) return ce;
@@ -313,30 +326,30 @@ cudaError_t launch_ns_fwd(const Problem& q) {
     p.partials = q.partials;
     const int minb = env_int("FPDE_NS_MINB_F", 3);
     cudaError_t ce;
-    if (!ns_tsafe(p)) ce = launch_kernel(ns_fwd_kernel<false, 3>, dim3(p.nitems), block, q.stream, p);
-    else if (minb == 3) ce = launch_kernel(ns_fwd_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
-    else ce = launch_kernel(ns_fwd_kernel<true, 4>, dim3(p.nitems), block, q.stream, p);
+    const dim3 grid = ns_range(q, p);
+    if (!ns_tsafe(p)) ce = launch_kernel(ns_fwd_kernel<false, 3>, grid, block, q.stream, p);
+    else if (minb == 3) ce = launch_kernel(ns_fwd_kernel<true, 3>, grid, block, q.stream, p);
+    else ce = launch_kernel(ns_fwd_kernel<true, 4>, grid, block, q.stream, p);
     return ce;
 }
 
 cudaError_t launch_ns_bwd(const Problem& q) {
-    if (!q.bc0_interior) {
+    if (!q.bc0_interior && q.planes_per_item == 0) {
         bool launched = false;
         const cudaError_t ce = launch_ns_bwd_tma(q, launched);
         if (launched || ce != cudaSuccess) return ce;
     }
     NsParams p{}; dim3 block;
-    const int ty_b = env_int("FPDE_NS_BWD_TY", 0);        // 8: one 256-thread block per SM (experiment)
-    ns_geometry(q, p, block, ty_b == 8 ? 8 : 0);
+    ns_geometry(q, p, block);
     for (int k = 0; k < 4; ++k) { p.f[k] = q.in[k]; p.g[k] = q.aux[k]; p.out[k] = q.out[k]; }
     ns_fill_consts(p.k, q.h, q.coef[0], q.gscale);
     p.partials = nullptr;
     const int minb = env_int("FPDE_NS_MINB_B", 2);
     cudaError_t ce;
-    if (ty_b == 8 && ns_tsafe(p) && block.x == 32) return launch_kernel(ns_bwd_kernel<true, 1, 256>, dim3(p.nitems), block, q.stream, p);
-    if (!ns_tsafe(p)) ce = launch_kernel(ns_bwd_kernel<false, 2>, dim3(p.nitems), block, q.stream, p);
-    else if (minb == 3) ce = launch_kernel(ns_bwd_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
-    else ce = launch_kernel(ns_bwd_kernel<true, 2>, dim3(p.nitems), block, q.stream, p);
+    const dim3 grid = ns_range(q, p);
+    if (!ns_tsafe(p)) ce = launch_kernel(ns_bwd_kernel<false, 2>, grid, block, q.stream, p);
+    else if (minb == 3) ce = launch_kernel(ns_bwd_kernel<true, 3>, grid, block, q.stream, p);
+    else ce = launch_kernel(ns_bwd_kernel<true, 2>, grid, block, q.stream, p);
     return ce;
 }
 
