@@ -259,11 +259,21 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     return FPDE_OK;
 }
 
+static int bwd_impl(int op, const float* const* fields, const float* const* gres, const double* gscale,
+                    float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
+                    const double* coeffs, int ncoeffs, const int* bc, void* stream, bool gres_zero_off_rows);
+
 int fpde_bwd(int op, const float* const* fields, const float* const* gres, const double* gscale,
              float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
              const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
              void* stream) {
     (void)workspace; (void)workspace_bytes;
+    return bwd_impl(op, fields, gres, gscale, gfields, ndim, shape, spacing, coeffs, ncoeffs, bc, stream, false);
+}
+
+static int bwd_impl(int op, const float* const* fields, const float* const* gres, const double* gscale,
+                    float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
+                    const double* coeffs, int ncoeffs, const int* bc, void* stream, bool gres_zero_off_rows) {
     Problem q;
     std::memset(&q, 0, sizeof(q));
     int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
@@ -283,6 +293,7 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
         q.out[f] = gfields[f];
     }
     q.stream = static_cast<cudaStream_t>(stream);
+    q.gres_zero_off_rows = gres_zero_off_rows;
     cudaError_t ce = cudaSuccess;
     switch (op) {
     case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_bwd(q); break;
@@ -331,8 +342,8 @@ int fpde_fwd_bwd(int op, const float* const* fields, const float* const* sources
         if (st != FPDE_OK) return st;
         double gscale[MAX_F];
         for (int r = 0; r < e.ne; ++r) gscale[r] = 2.0 / (double)q.rows;
-        return fpde_bwd(op, fields, residuals, gscale, gfields, ndim, shape, spacing, coeffs, ncoeffs, bc, nullptr, 0,
-                        stream);
+        // the upstream arrays are the residual arrays the forward kernel just wrote
+        return bwd_impl(op, fields, residuals, gscale, gfields, ndim, shape, spacing, coeffs, ncoeffs, bc, stream, true);
     }
     if (e.ns > 0 && !sources) return FPDE_ERR_NULL;
     for (int s = 0; s < e.ns; ++s) {

@@ -30,6 +30,9 @@ struct Problem {
     // chunks this launch covers (chunk_hi <= chunk_lo = all); the loss partial sums keep their
     // global slots, so several ranged launches add up to one full launch
     int planes_per_item, chunk_lo, chunk_hi;
+    // bwd: the upstream arrays are residual arrays a forward kernel of this library wrote (exactly
+    // zero at nodes without a row), so the adjoint need not zero-extend them itself
+    bool gres_zero_off_rows;
 };
 
 // The same for the double-precision verification path (ops_f64.cu).

@@ -42,8 +42,13 @@ __device__ __forceinline__ void prefetch_l2_line(const float* ptr) {
 // EDGE: the block touches the two-cell band in x or y, where (adjoint) rows and planes of the
 // upstream array read as zero; blocks away from the band run without those selects.  The first
 // and last float4 of a row (the band in z) are handled in every block.
-template <bool FWD, bool EDGE, int MINB>
+// MODE 0: forward.  MODE 1: adjoint of an arbitrary upstream array (zero-extended here).  MODE 2:
+// adjoint of an upstream array that is already zero off the rows (the residual array the forward
+// kernel of the same call wrote): the star itself, nothing to mask; clamped reads beyond the
+// array land in the zero band.
+template <int MODE, bool EDGE, int MINB>
 __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int mb, int ab) {
+    constexpr bool FWD = MODE == 0;
     const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
     const int c4 = cb * blockDim.x + threadIdx.x;
     const int m = mb * blockDim.y + threadIdx.y;
@@ -55,7 +60,7 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     const int a0 = ab * p.planes_per_item;
     const int a1 = min(a0 + p.planes_per_item, n0);
     const int PS = n1 * n2;
-    constexpr bool MASK_IN = !FWD;                  // the adjoint zero-extends its input outside the rows
+    constexpr bool MASK_IN = MODE == 1;             // the adjoint zero-extends its input outside the rows
     constexpr bool ROWMASK = MASK_IN && EDGE;
     const float* __restrict__ hin = p.hin;
 
@@ -163,7 +168,7 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     }
 }
 
-template <bool FWD, int MINB>
+template <int MODE, int MINB>
 __global__ void __launch_bounds__(256, MINB) star3d_kernel(const Star3dParams p) {
     pdl_wait_then_trigger();
     int item = blockIdx.x;
@@ -173,8 +178,8 @@ __global__ void __launch_bounds__(256, MINB) star3d_kernel(const Star3dParams p)
     const int m0 = mb * blockDim.y, a0 = ab * p.planes_per_item;
     // away from the band: every row m0-2 .. m0+TY+1 and plane a0-2 .. a1+1 is a row of the operator
     const bool interior = m0 >= 4 && m0 + (int)blockDim.y + 4 <= p.n1 && a0 >= 4 && a0 + p.planes_per_item + 4 <= p.n0;
-    if (interior) star3d_body<FWD, false, MINB>(p, cb, mb, ab);
-    else star3d_body<FWD, true, MINB>(p, cb, mb, ab);
+    if (interior) star3d_body<MODE, false, MINB>(p, cb, mb, ab);
+    else star3d_body<MODE, true, MINB>(p, cb, mb, ab);
 }
 
 static int env_int(const char* name, int dflt) {
@@ -224,8 +229,8 @@ cudaError_t launch_helmholtz_fwd(const Problem& q) {
     star3d_geometry(q, p, block, 1.0, true);
     p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0];
     p.partials = q.partials;
-    if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<true, 4>, dim3(p.nitems), block, q.stream, p);
-    return launch_kernel(star3d_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
+    if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<0, 4>, dim3(p.nitems), block, q.stream, p);
+    return launch_kernel(star3d_kernel<0, 3>, dim3(p.nitems), block, q.stream, p);
 }
 
 cudaError_t launch_helmholtz_bwd(const Problem& q) {
@@ -233,8 +238,13 @@ cudaError_t launch_helmholtz_bwd(const Problem& q) {
     star3d_geometry(q, p, block, q.gscale[0], false);      // the operator is linear: the scale goes into the weights
     p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0];
     p.partials = nullptr;
-    if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<false, 4>, dim3(p.nitems), block, q.stream, p);
-    return launch_kernel(star3d_kernel<false, 3>, dim3(p.nitems), block, q.stream, p);
+    const bool m4 = env_int("FPDE_STAR3D_MINB", 4) >= 4;
+    if (q.gres_zero_off_rows) {
+        if (m4) return launch_kernel(star3d_kernel<2, 4>, dim3(p.nitems), block, q.stream, p);
+        return launch_kernel(star3d_kernel<2, 3>, dim3(p.nitems), block, q.stream, p);
+    }
+    if (m4) return launch_kernel(star3d_kernel<1, 4>, dim3(p.nitems), block, q.stream, p);
+    return launch_kernel(star3d_kernel<1, 3>, dim3(p.nitems), block, q.stream, p);
 }
 
 }  // namespace fpde

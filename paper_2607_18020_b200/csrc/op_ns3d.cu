@@ -57,11 +57,11 @@ __device__ __forceinline__ V4 ns3d_zmask(const Ns3dThread& t, V4 v) {
 
 // array k at plane r (clamped into the array) at the thread's own float4; with `check`, an
 // upstream float4 whose plane or row is outside the rows reads as zero
-template <bool BWD>
+template <bool BWD, bool PRE>
 __device__ __forceinline__ V4 ns3d_load_own(const Ns3dParams& p, const Ns3dThread& t, int k, int r, bool check) {
     const int rr = max(0, min(t.n0 - 1, r));
     V4 v = ldv4(p.a[k] + rr * t.PS + t.rowoff);
-    if (BWD && k >= 3) {
+    if (BWD && !PRE && k >= 3) {
         v = ns3d_zmask(t, v);
         if (check && (t.y_dead || r < 1 || r > t.n0 - 2)) v = v4zero();
     }
@@ -71,7 +71,10 @@ __device__ __forceinline__ V4 ns3d_load_own(const Ns3dParams& p, const Ns3dThrea
 // One x step: W0 = plane a-1, W1 = plane a, W2 receives plane a+1.  EDGE: some float4 the block
 // reads in this step lies outside the rows (a block-uniform property), so the whole-vector
 // zero extension has to be looked at; the other steps skip those selects.
-template <bool BWD, bool EDGE, int NA>
+// PRE (adjoint only): the upstream arrays are already zero off the rows (residual arrays the
+// forward kernel of the same call wrote), so nothing is zero-extended here; clamped reads beyond
+// the array land in the zero shell.
+template <bool BWD, bool EDGE, int NA, bool PRE>
 __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread& t, int a, const V4 (&W0)[NA],
                                           const V4 (&W1)[NA], V4 (&W2)[NA], float2 (&acc)[4]) {
     constexpr int G0 = 3;                            // adjoint: first upstream array
@@ -86,7 +89,7 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
     float E[NA];
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
-        W2[k] = ns3d_load_own<BWD>(p, t, k, a + 1, EDGE);
+        W2[k] = ns3d_load_own<BWD, PRE>(p, t, k, a + 1, EDGE);
         Ym[k] = ldv4(p.a[k] + pl + t.ymoff);
         Yp[k] = ldv4(p.a[k] + pl + t.ypoff);
         E[k] = 0.f;
@@ -94,7 +97,7 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
     }
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
-        if (BWD && k >= G0) {
+        if (BWD && !PRE && k >= G0) {
             Ym[k] = ns3d_zmask(t, Ym[k]); Yp[k] = ns3d_zmask(t, Yp[k]);
             if (EDGE) {
                 if (x_dead || t.ym_dead) Ym[k] = v4zero();
@@ -141,7 +144,7 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
     }
 }
 
-template <bool BWD, int MINB>
+template <bool BWD, int MINB, bool PRE = false>
 __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     constexpr int NA = BWD ? 7 : 4;
     pdl_wait_then_trigger();
@@ -187,16 +190,16 @@ __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     V4 A[NA], B[NA], Cc[NA];
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
-        A[k] = ns3d_load_own<BWD>(p, t, k, a0 - 1, true);
-        B[k] = ns3d_load_own<BWD>(p, t, k, a0, true);
+        A[k] = ns3d_load_own<BWD, PRE>(p, t, k, a0 - 1, true);
+        B[k] = ns3d_load_own<BWD, PRE>(p, t, k, a0, true);
     }
     float2 acc[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
 
     auto step = [&](int a, const V4 (&W0)[NA], const V4 (&W1)[NA], V4 (&W2)[NA]) {
-        if (y_edge_block || a <= 1 || a >= p.n0 - 2) ns3d_step<BWD, true, NA>(p, t, a, W0, W1, W2, acc);
-        else ns3d_step<BWD, false, NA>(p, t, a, W0, W1, W2, acc);
+        if (!PRE && (y_edge_block || a <= 1 || a >= p.n0 - 2)) ns3d_step<BWD, true, NA, PRE>(p, t, a, W0, W1, W2, acc);
+        else ns3d_step<BWD, false, NA, PRE>(p, t, a, W0, W1, W2, acc);
     };
     for (int a = a0; a < a1; a += 3) {
         step(a, A, B, Cc);
@@ -266,6 +269,7 @@ cudaError_t launch_ns3d_bwd(const Problem& q) {
     for (int k = 0; k < 4; ++k) { p.a[3 + k] = q.aux[k]; p.out[k] = q.out[k]; }
     ns3d_consts(q, q.gscale, p.k);
     p.partials = nullptr;
+    if (q.gres_zero_off_rows) return launch_kernel(ns3d_kernel<true, 2, true>, dim3(p.nitems), block, q.stream, p);
     if (env_int("FPDE_NS3D_MINB_B", 2) == 3) return launch_kernel(ns3d_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
     return launch_kernel(ns3d_kernel<true, 2>, dim3(p.nitems), block, q.stream, p);
 }

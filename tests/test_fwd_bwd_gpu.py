@@ -33,8 +33,12 @@ SINGLE_PASS = [
 TWO_KERNEL = [
     ("burgers_256x128", (37, 23)),
     ("helmholtz_256", (12, 20, 24)),
+    ("helmholtz_256", (70, 45, 136)),              # ragged z line: the adjoint runs without zero-extension here
+    ("helmholtz_256", (5, 5, 8)),
     ("ns_tgv_128x16", (8, 12, 16, 8)),
     ("ns3d_steady_256", (7, 5, 132)),
+    ("ns3d_steady_256", (37, 22, 136)),
+    ("ns3d_steady_256", (3, 3, 4)),
 ]
 
 
