@@ -7,9 +7,9 @@
 `fused_residual` runs `fpde_fwd` (no loss) in the forward pass and `fpde_bwd` on the upstream
 sensitivities autograd hands back.  `fused_residual_loss` also fuses the mean-square loss: the
 forward pass is `fpde_fwd` with the loss, the backward pass is `fpde_bwd` on the residual
-arrays with scale 2/N_r, times the incoming scalar gradient; where the operator has a
-single-pass kernel and a gradient is wanted, the forward pass is `fpde_fwd_bwd` (loss and
-dL/dfield from one kernel) and the backward pass only applies the incoming scalar.  Everything runs in the library's
+arrays with scale 2/N_r, times the incoming scalar gradient; in fp32, when a gradient is wanted,
+the forward pass is `fpde_fwd_bwd` (loss and dL/dfield from one call, one kernel where the
+operator has a single-pass kernel) and the backward pass only applies the incoming scalar.  Everything runs in the library's
 kernels on the current CUDA stream; torch allocates the outputs and nothing else.  fp64 tensors go
 through the double-precision verification kernels (`fpde_fwd_f64` / `fpde_bwd_f64`), which makes
 `torch.autograd.gradcheck` usable on the operators.
@@ -83,12 +83,15 @@ class _FusedResidualLoss(torch.autograd.Function):
         ne = B.op_info(op).nresiduals
         loss = torch.empty(ne + 1, dtype=torch.float64, device=dev)
         ctx.op, ctx.shape, ctx.spacing, ctx.coeffs, ctx.bc, ctx.ne, ctx.dt = op, shape, spacing, coeffs, bc, ne, dt
-        ctx.single_pass = dt == torch.float32 and B.has_single_pass(op) and any(ctx.needs_input_grad[5:])
+        ctx.single_pass = dt == torch.float32 and any(ctx.needs_input_grad[5:])
         if ctx.single_pass:
-            # one kernel: the loss and dL/dfield together, no residual arrays kept for backward
+            # one call: the loss and dL/dfield together (one kernel where the operator has a
+            # single-pass kernel; forward + adjoint with scratch residual arrays elsewhere);
+            # nothing but the gradients is kept for backward
             grads = [torch.empty(shape, dtype=torch.float32, device=dev) for _ in fields]
             ws = torch.empty(B.fwd_bwd_workspace_bytes(op, shape), dtype=torch.uint8, device=dev)
-            B.fpde_fwd_bwd(op, fields, sources, None, grads, loss, shape, spacing, coeffs, bc, ws)
+            res = None if B.has_single_pass(op) else [torch.empty(shape, dtype=torch.float32, device=dev) for _ in range(ne)]
+            B.fpde_fwd_bwd(op, fields, sources, res, grads, loss, shape, spacing, coeffs, bc, ws)
             ctx.save_for_backward(*grads)
             return loss[ne]
         res = [torch.empty(shape, dtype=dt, device=dev) for _ in range(ne)]
