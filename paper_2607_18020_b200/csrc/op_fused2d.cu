@@ -303,14 +303,13 @@ bool fused2d_supported(int op) {
     return op == 1 || op == 2 || op == 5;            // Poisson 2-D, Gray-Scott, steady 2-D Navier-Stokes
 }
 
-static int sm_count() {
-    static int n = 0;
-    if (n == 0) {
+static int sm_count() {                              // initialised once, thread-safe
+    static const int n = [] {
         int dev = 0, v = 0;
         if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else n = 148;
-    }
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) return v;
+        return 148;
+    }();
     return n;
 }
 
