@@ -23,7 +23,7 @@ _SRC = os.path.join(_HERE, "fpde_oracle.c")
 _LIB = os.path.join(_HERE, "libfpde_oracle.so")
 
 OP_IDS = {"burgers_1d_t": 0, "poisson_2d": 1, "grayscott_2d": 2, "helmholtz_3d_o4": 3, "ns_3d_t": 4, "ns_2d_steady": 5, "ns_3d_steady": 6,
-          "ns_3d_t_xslab": 7}
+          "ns_3d_t_xslab": 7, "grayscott_2d_xslab": 8}
 
 _lib = None
 
@@ -71,7 +71,7 @@ def fwd(op: str, fields, sources, shape, spacing, coeffs) -> Tuple[List[np.ndarr
     F, S = _f64(fields), _f64(sources)
     for a in F + S:
         assert a.shape == shape, (a.shape, shape)
-    ne = {0: 1, 1: 1, 2: 2, 3: 1, 4: 4, 5: 3, 6: 4, 7: 4}[opi]
+    ne = {0: 1, 1: 1, 2: 2, 3: 1, 4: 4, 5: 3, 6: 4, 7: 4, 8: 2}[opi]
     R = [np.empty(shape, dtype=np.float64) for _ in range(ne)]
     loss = np.zeros(ne + 1, dtype=np.float64)
     shp = np.asarray(shape, dtype=np.int64)

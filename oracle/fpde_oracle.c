@@ -34,7 +34,8 @@ typedef long long i64;
 
 enum { OP_BURGERS_1D_T = 0, OP_POISSON_2D = 1, OP_GRAYSCOTT_2D = 2, OP_HELMHOLTZ_3D_O4 = 3,
        OP_NS_3D_T = 4, OP_NS_2D_STEADY = 5, OP_NS_3D_STEADY = 6, OP_NS_3D_T_XSLAB = 7,
-       OP_COUNT = 8 };
+       OP_GRAYSCOTT_2D_XSLAB = 8,
+       OP_COUNT = 9 };
 enum { BC_PERIODIC = 0, BC_INTERIOR = 1, BC_ONE_SIDED = 2 };
 
 /* A 1-D difference formula at one node: value = sum_k w[k] * q[idx[k]] along one axis. */
@@ -115,11 +116,11 @@ static void scatter(const stencil* s, double* line, i64 stride, double a) {
     for (k = 0; k < s->n; ++k) line[s->idx[k] * stride] += a * s->w[k];
 }
 
-static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2, 3, 4 };
-static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4, 4 };
-static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0, 0, 0 };
-static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4, 4 };
-static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1, 1, 1 };
+static const int OP_NDIM[OP_COUNT] = { 2, 2, 2, 3, 4, 2, 3, 4, 2 };
+static const int OP_NF[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4, 4, 2 };
+static const int OP_NS[OP_COUNT] = { 0, 1, 0, 1, 0, 0, 0, 0, 0 };
+static const int OP_NE[OP_COUNT] = { 1, 1, 2, 1, 4, 3, 4, 4, 2 };
+static const int OP_NC[OP_COUNT] = { 1, 0, 4, 1, 1, 1, 1, 1, 4 };
 static const int OP_BC[OP_COUNT][4] = {
     { BC_ONE_SIDED, BC_ONE_SIDED, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
@@ -129,6 +130,7 @@ static const int OP_BC[OP_COUNT][4] = {
     { BC_INTERIOR, BC_INTERIOR, 0, 0 },
     { BC_INTERIOR, BC_INTERIOR, BC_INTERIOR, 0 },
     { BC_INTERIOR, BC_PERIODIC, BC_PERIODIC, BC_INTERIOR },
+    { BC_INTERIOR, BC_PERIODIC, 0, 0 },
 };
 
 int fpde_oracle_info(int op, int* ndim, int* nf, int* ns, int* ne, int* nc) {
@@ -197,13 +199,13 @@ static i64 poisson(int mode, const double* u, const double* f, double* r, const 
  * r_v = Dv*Lap v + u v^2 - (F+k) v, Lap = d_xx + d_yy (five points). */
 static i64 grayscott(int mode, const double* u, const double* v, double* ru, double* rv,
                      const double* Gu, const double* Gv, double* gu, double* gv,
-                     const i64* n, const double* h, const double* c) {
+                     const i64* n, const double* h, const double* c, int bcx) {
     i64 nx = n[0], ny = n[1], i, j, rows = 0;
     double Du = c[0], Dv = c[1], F = c[2], k = c[3];
     for (i = 0; i < nx; ++i) for (j = 0; j < ny; ++j) {
         stencil sx, sy;
         i64 p = i * ny + j;
-        d2(BC_PERIODIC, i, nx, h[0], &sx);
+        if (!d2(bcx, i, nx, h[0], &sx)) continue;    /* bcx = BC_INTERIOR: the slab form, rows at x-index 1..nx-2 */
         d2(BC_PERIODIC, j, ny, h[1], &sy);
         ++rows;
         if (mode == 0) {
@@ -445,7 +447,8 @@ i64 fpde_oracle_fwd(int op, const double* const* fields, const double* const* so
     switch (op) {
     case OP_BURGERS_1D_T: rows = burgers(0, fields[0], residuals[0], NULL, NULL, shape, spacing, coeffs); break;
     case OP_POISSON_2D: rows = poisson(0, fields[0], sources[0], residuals[0], NULL, NULL, shape, spacing); break;
-    case OP_GRAYSCOTT_2D: rows = grayscott(0, fields[0], fields[1], residuals[0], residuals[1], NULL, NULL, NULL, NULL, shape, spacing, coeffs); break;
+    case OP_GRAYSCOTT_2D: rows = grayscott(0, fields[0], fields[1], residuals[0], residuals[1], NULL, NULL, NULL, NULL, shape, spacing, coeffs, BC_PERIODIC); break;
+    case OP_GRAYSCOTT_2D_XSLAB: rows = grayscott(0, fields[0], fields[1], residuals[0], residuals[1], NULL, NULL, NULL, NULL, shape, spacing, coeffs, BC_INTERIOR); break;
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(0, fields[0], sources[0], residuals[0], NULL, NULL, shape, spacing, coeffs); break;
     case OP_NS_3D_T: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs, BC_PERIODIC); break;
     case OP_NS_3D_T_XSLAB: rows = ns3dt(0, fields, residuals, NULL, NULL, shape, spacing, coeffs, BC_INTERIOR); break;
@@ -476,7 +479,8 @@ i64 fpde_oracle_bwd(int op, const double* const* fields, const double* const* G,
     switch (op) {
     case OP_BURGERS_1D_T: rows = burgers(1, fields[0], NULL, G[0], gfields[0], shape, spacing, coeffs); break;
     case OP_POISSON_2D: rows = poisson(1, fields[0], NULL, NULL, G[0], gfields[0], shape, spacing); break;
-    case OP_GRAYSCOTT_2D: rows = grayscott(1, fields[0], fields[1], NULL, NULL, G[0], G[1], gfields[0], gfields[1], shape, spacing, coeffs); break;
+    case OP_GRAYSCOTT_2D: rows = grayscott(1, fields[0], fields[1], NULL, NULL, G[0], G[1], gfields[0], gfields[1], shape, spacing, coeffs, BC_PERIODIC); break;
+    case OP_GRAYSCOTT_2D_XSLAB: rows = grayscott(1, fields[0], fields[1], NULL, NULL, G[0], G[1], gfields[0], gfields[1], shape, spacing, coeffs, BC_INTERIOR); break;
     case OP_HELMHOLTZ_3D_O4: rows = helmholtz(1, fields[0], NULL, NULL, G[0], gfields[0], shape, spacing, coeffs); break;
     case OP_NS_3D_T: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs, BC_PERIODIC); break;
     case OP_NS_3D_T_XSLAB: rows = ns3dt(1, fields, NULL, G, gfields, shape, spacing, coeffs, BC_INTERIOR); break;

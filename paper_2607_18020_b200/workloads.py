@@ -35,7 +35,9 @@ NS_3D_T = "ns_3d_t"
 NS_2D_STEADY = "ns_2d_steady"
 NS_3D_STEADY = "ns_3d_steady"
 NS_3D_T_XSLAB = "ns_3d_t_xslab"     # NS_3D_T with a non-periodic x axis: the form of one slab of a grid split along x
-OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY, NS_3D_STEADY, NS_3D_T_XSLAB)
+GRAYSCOTT_2D_XSLAB = "grayscott_2d_xslab"   # the same for Gray-Scott
+OPS = (BURGERS_1D_T, POISSON_2D, GRAYSCOTT_2D, HELMHOLTZ_3D_O4, NS_3D_T, NS_2D_STEADY, NS_3D_STEADY, NS_3D_T_XSLAB,
+       GRAYSCOTT_2D_XSLAB)
 
 # Boundary kinds per array axis.
 PERIODIC = "periodic"      # rows at every node, wrap-around neighbours
@@ -127,8 +129,11 @@ CONFIGS["ns3d_steady_256"] = dict(op=NS_3D_STEADY, shape=(256, 256, 256),
 CONFIGS["ns_tgv_xslab_34"] = dict(op=NS_3D_T_XSLAB, shape=(34, 128, 128, 16),
                                   domain=((0.0, 2 * math.pi * 33 / 128),) + ((0.0, 2 * math.pi),) * 2 + ((0.0, 1.0),),
                                   bc=(INTERIOR, PERIODIC, PERIODIC, INTERIOR))
+# one of four x-slabs of the 4096^2 Gray-Scott grid, with its two halo rows
+CONFIGS["grayscott_xslab_1026"] = dict(op=GRAYSCOTT_2D_XSLAB, shape=(1026, 4096),
+                                       domain=((0.0, 1025.0 / 4096.0), (0.0, 1.0)), bc=(INTERIOR, PERIODIC))
 EXTRA_CONFIGS = ("ns2d_steady_4096", "ns3d_steady_256")
-SLAB_CONFIGS = ("ns_tgv_xslab_34",)
+SLAB_CONFIGS = ("ns_tgv_xslab_34", "grayscott_xslab_1026")
 CONFIG_ORDER = ("burgers_256x128", "poisson_1024", "grayscott_4096", "helmholtz_256", "ns_tgv_128x16")
 
 OP_META = {
@@ -143,6 +148,7 @@ OP_META = {
                        residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
     NS_3D_T_XSLAB: dict(fields=("u", "v", "w", "p"), sources=(),
                         residuals=("mom_x", "mom_y", "mom_z", "continuity"), ncoeffs=1),
+    GRAYSCOTT_2D_XSLAB: dict(fields=("u", "v"), sources=(), residuals=("r_u", "r_v"), ncoeffs=4),
 }
 DEFAULT_COEFFS = {
     BURGERS_1D_T: (0.01 / math.pi,),
@@ -153,6 +159,7 @@ DEFAULT_COEFFS = {
     NS_2D_STEADY: (0.01,),
     NS_3D_STEADY: (0.01,),
     NS_3D_T_XSLAB: (0.01,),
+    GRAYSCOTT_2D_XSLAB: (2e-5, 1e-5, 0.04, 0.06),
 }
 
 
@@ -187,7 +194,7 @@ def analytic_fields(op: str, axes: Sequence[np.ndarray], coeffs: Sequence[float]
         x, y = _bcast(axes, 0), _bcast(axes, 1)
         us = np.sin(math.pi * x) * np.sin(math.pi * y)
         return [us.copy()], [2 * math.pi ** 2 * us]
-    if op == GRAYSCOTT_2D:
+    if op in (GRAYSCOTT_2D, GRAYSCOTT_2D_XSLAB):
         return [np.full(shape, 0.95), np.full(shape, 0.05)], []
     if op == HELMHOLTZ_3D_O4:
         x, y, z = (_bcast(axes, a) for a in range(3))
@@ -255,7 +262,7 @@ def make(name: str, seed: int = 42, shape: Optional[Sequence[int]] = None, kind:
         sources = [_noise(seed, 50 + i, shape, 1.0) for i in range(ns)]
     elif kind == "config":
         fields, sources = analytic_fields(op, axes, coeffs)
-        if op == GRAYSCOTT_2D:
+        if op in (GRAYSCOTT_2D, GRAYSCOTT_2D_XSLAB):
             n = int(np.prod(shape))
             fields = [0.9 + 0.1 * uniform01(seed, 10, n).reshape(shape),
                       0.1 * uniform01(seed, 11, n).reshape(shape)]

@@ -300,6 +300,7 @@ CASES = [
     (W.NS_2D_STEADY, (8, 9), (0.2, 0.3), (0.17,)),
     (W.NS_3D_STEADY, (6, 7, 5), (0.2, 0.3, 0.25), (0.17,)),
     (W.NS_3D_T_XSLAB, (6, 5, 4, 6), (0.3, 0.2, 0.25, 0.15), (0.13,)),
+    (W.GRAYSCOTT_2D_XSLAB, (7, 6), (0.2, 0.3), (0.7, 0.3, 0.04, 0.06)),
 ]
 
 
@@ -348,6 +349,7 @@ TINY = [
     (W.NS_2D_STEADY, (6, 7), (0.2, 0.3), (0.17,)),
     (W.NS_3D_STEADY, (5, 4, 5), (0.2, 0.3, 0.25), (0.17,)),
     (W.NS_3D_T_XSLAB, (5, 4, 4, 5), (0.3, 0.2, 0.25, 0.15), (0.13,)),
+    (W.GRAYSCOTT_2D_XSLAB, (6, 5), (0.2, 0.3), (0.7, 0.3, 0.04, 0.06)),
 ]
 
 
@@ -628,5 +630,24 @@ def test_ns3dt_xslab_is_the_periodic_operator_on_its_inner_planes():
         g[0] = 0.0; g[-1] = 0.0
     gs = oracle.bwd(W.NS_3D_T_XSLAB, F, G, shape, h, c)          # outer planes of G are ignored
     gp = oracle.bwd(W.NS_3D_T, F, G0, shape, h, c)
+    for a, b in zip(gs, gp):
+        assert np.allclose(a, b, rtol=0, atol=1e-12)
+
+
+def test_grayscott_xslab_is_the_periodic_operator_on_its_inner_rows():
+    shape, h, c = (7, 8), (0.2, 0.3), (0.7, 0.3, 0.04, 0.06)
+    r = np.random.default_rng(78)
+    F = [r.standard_normal(shape) for _ in range(2)]
+    Rp, _, rows_p = oracle.fwd(W.GRAYSCOTT_2D, F, [], shape, h, c)
+    Rs, _, rows_s = oracle.fwd(W.GRAYSCOTT_2D_XSLAB, F, [], shape, h, c)
+    assert rows_p == 56 and rows_s == 40
+    for a, b in zip(Rp, Rs):
+        assert np.array_equal(a[1:-1], b[1:-1]) and np.all(b[0] == 0.0) and np.all(b[-1] == 0.0)
+    G = [r.standard_normal(shape) for _ in range(2)]
+    G0 = [g.copy() for g in G]
+    for g in G0:
+        g[0] = 0.0; g[-1] = 0.0
+    gs = oracle.bwd(W.GRAYSCOTT_2D_XSLAB, F, G, shape, h, c)
+    gp = oracle.bwd(W.GRAYSCOTT_2D, F, G0, shape, h, c)
     for a, b in zip(gs, gp):
         assert np.allclose(a, b, rtol=0, atol=1e-12)
