@@ -85,6 +85,8 @@ typedef enum {
  *        x-plane are data.  This is the form one slab of a grid split along x takes: its outer
  *        planes are copies of the neighbouring slabs' planes, and on the planes that carry rows
  *        the residuals are those of the periodic operator on the whole grid.
+ *  FPDE_OP_GRAYSCOTT_2D_XSLAB  the same for FPDE_OP_GRAYSCOTT_2D, bc = (INTERIOR, PERIODIC): rows
+ *        at x-index 1..n_x-2, the first and last row of the array are data.
  *
  * Shape rules: the contiguous extent must be a multiple of 4 (float4 path) except for
  * BURGERS_1D_T; PERIODIC / INTERIOR axes need n >= 2*radius+1, ONE_SIDED axes n >= 4; the
@@ -99,7 +101,8 @@ typedef enum {
     FPDE_OP_NS_2D_STEADY = 5,
     FPDE_OP_NS_3D_STEADY = 6,
     FPDE_OP_NS_3D_T_XSLAB = 7,
-    FPDE_OP_COUNT = 8
+    FPDE_OP_GRAYSCOTT_2D_XSLAB = 8,
+    FPDE_OP_COUNT = 9
 } fpde_op;
 
 /* Boundary kind of one array axis (Appendix A.4 names the three causes of boundary terms:

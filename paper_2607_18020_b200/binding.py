@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libfpde.so")
 
 # numeric ids of include/fpde.h
 OP_IDS = {_w.BURGERS_1D_T: 0, _w.POISSON_2D: 1, _w.GRAYSCOTT_2D: 2, _w.HELMHOLTZ_3D_O4: 3, _w.NS_3D_T: 4, _w.NS_2D_STEADY: 5,
-          _w.NS_3D_STEADY: 6, _w.NS_3D_T_XSLAB: 7}
+          _w.NS_3D_STEADY: 6, _w.NS_3D_T_XSLAB: 7, _w.GRAYSCOTT_2D_XSLAB: 8}
 BC_IDS = {_w.PERIODIC: 0, _w.INTERIOR: 1, _w.ONE_SIDED: 2}
 FPDE_OK = 0
 

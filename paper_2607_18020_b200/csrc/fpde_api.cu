@@ -35,6 +35,7 @@ static const OpEntry REGISTRY[FPDE_OP_COUNT] = {
     /* NS_2D_STEADY    */ {2, 3, 0, 3, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0, 0}, true},
     /* NS_3D_STEADY    */ {3, 4, 0, 4, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, FPDE_BC_INTERIOR, 0}, true},
     /* NS_3D_T_XSLAB   */ {4, 4, 0, 4, 1, 1, {FPDE_BC_INTERIOR, FPDE_BC_PERIODIC, FPDE_BC_PERIODIC, FPDE_BC_INTERIOR}, true},
+    /* GRAYSCOTT_XSLAB */ {2, 2, 0, 2, 4, 1, {FPDE_BC_INTERIOR, FPDE_BC_PERIODIC, 0, 0}, true},
 };
 
 static int check_shape(int op, int ndim, const int64_t* shape, int* n_out, int64_t* total, int64_t* rows) {
@@ -63,7 +64,8 @@ static size_t workspace_need(int op, const int* n) {
     switch (op) {
     case FPDE_OP_BURGERS_1D_T: items = burgers_items(n); break;
     case FPDE_OP_POISSON_2D:
-    case FPDE_OP_GRAYSCOTT_2D: items = lap2d_items(n); break;
+    case FPDE_OP_GRAYSCOTT_2D:
+    case FPDE_OP_GRAYSCOTT_2D_XSLAB: items = lap2d_items(n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: items = star3d_items(n); break;
     case FPDE_OP_NS_3D_T: items = ns_items(n, false); break;
     case FPDE_OP_NS_3D_T_XSLAB: items = ns_items(n, true); break;
@@ -244,7 +246,8 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     switch (op) {
     case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_fwd(q); items = burgers_items(q.n); break;
     case FPDE_OP_POISSON_2D:
-    case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_fwd(q); items = lap2d_items(q.n); break;
+    case FPDE_OP_GRAYSCOTT_2D:
+    case FPDE_OP_GRAYSCOTT_2D_XSLAB: ce = launch_lap2d_fwd(q); items = lap2d_items(q.n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q); items = star3d_items(q.n); break;
     case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n, false); break;
     case FPDE_OP_NS_3D_T_XSLAB: ce = launch_ns_fwd(q); items = ns_items(q.n, true); break;
@@ -298,7 +301,8 @@ static int bwd_impl(int op, const float* const* fields, const float* const* gres
     switch (op) {
     case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_bwd(q); break;
     case FPDE_OP_POISSON_2D:
-    case FPDE_OP_GRAYSCOTT_2D: ce = launch_lap2d_bwd(q); break;
+    case FPDE_OP_GRAYSCOTT_2D:
+    case FPDE_OP_GRAYSCOTT_2D_XSLAB: ce = launch_lap2d_bwd(q); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_bwd(q); break;
     case FPDE_OP_NS_3D_T:
     case FPDE_OP_NS_3D_T_XSLAB: ce = launch_ns_bwd(q); break;

@@ -90,13 +90,17 @@ struct GrayScottBwd {
     }
 };
 
-template <class F, bool PERIODIC, int U>
+// PX / PY: the row axis (x) / the column axis (y) is periodic.  Poisson: neither; Gray-Scott:
+// both; the slab form of Gray-Scott (x not periodic: rows at x-index 1..n0-2): PY only.
+template <class F, bool PX, bool PY, int U>
 __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
     constexpr int NH = F::NH, NC = F::NC, NO = F::NO;
     constexpr int NCA = NC > 0 ? NC : 1;
     constexpr bool BWD = F::BWD;
-    constexpr bool MASK_IN = BWD && !PERIODIC;     // upstream array is zero outside the rows
-    constexpr bool MASK_OUT = !BWD && !PERIODIC;   // ring nodes carry no row
+    constexpr bool ROWS_MASK_IN = BWD && !PX;      // upstream array is zero on the first / last row and beyond
+    constexpr bool COLS_MASK_IN = BWD && !PY;      // ... and on the first / last column and beyond
+    constexpr bool ROWS_MASK_OUT = !BWD && !PX;    // nodes of the first / last row carry no residual row
+    constexpr bool COLS_MASK_OUT = !BWD && !PY;    // nor do those of the first / last column
     pdl_wait_then_trigger();
     const int n0 = p.n0, n1 = p.n1, nc4 = p.nc4;
     const int item = blockIdx.x;
@@ -111,23 +115,23 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
 
     // columns the first / last lane of a warp fetch from memory (the others use shuffles)
     int lcol = col - 1, rcol = col + 4;
-    if (PERIODIC) { if (lcol < 0) lcol += n1; if (rcol >= n1) rcol -= n1; }
+    if (PY) { if (lcol < 0) lcol += n1; if (rcol >= n1) rcol -= n1; }
     const bool lfetch = cvalid && (lane == 0 || first_col) && lcol >= 0;
     const bool rfetch = cvalid && (lane == 31 || last_col) && rcol < n1;
-    const bool lzero = !PERIODIC && first_col, rzero = !PERIODIC && last_col;
+    const bool lzero = !PY && first_col, rzero = !PY && last_col;
 
     // row index a halo-input row is read from, or -1 if it reads as zero
     auto in_row = [&](int r) -> int {
-        if (PERIODIC) return r < 0 ? r + n0 : (r >= n0 ? r - n0 : r);
-        if (MASK_IN) return (r < 1 || r > n0 - 2) ? -1 : r;
+        if (PX) return r < 0 ? r + n0 : (r >= n0 ? r - n0 : r);
+        if (ROWS_MASK_IN) return (r < 1 || r > n0 - 2) ? -1 : r;
         return max(0, min(n0 - 1, r));              // forward: out-of-range rows only feed masked outputs
     };
     auto load_h = [&](int k, int r) -> V4 {
         const int rr = in_row(r);
-        if (MASK_IN && rr < 0) return v4zero();
+        if (ROWS_MASK_IN && rr < 0) return v4zero();
         V4 v = ldv4(p.hin[k] + rr * n1 + col);
         if (BWD) v = v4mul(v, p.hscale[k]);
-        if (MASK_IN) {
+        if (COLS_MASK_IN) {
             if (first_col) v.lo.x = 0.f;
             if (last_col) v.hi.y = 0.f;
         }
@@ -154,7 +158,7 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
                 nxt[u][k] = load_h(k, row + 1);
                 const int rr = in_row(row);
                 le[u][k] = 0.f; re[u][k] = 0.f;
-                if (!(MASK_IN && rr < 0)) {
+                if (!(ROWS_MASK_IN && rr < 0)) {
                     const float* rp = p.hin[k] + rr * n1;
                     if (lfetch) le[u][k] = __ldg(rp + lcol);
                     if (rfetch) re[u][k] = __ldg(rp + rcol);
@@ -191,13 +195,13 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
                 for (int k = 0; k < NC; ++k) { cc_lo[k] = cen[u][k].lo; cc_hi[k] = cen[u][k].hi; }
                 F::eval(v_lo, lap_lo, cc_lo, p.c, o_lo);
                 F::eval(v_hi, lap_hi, cc_hi, p.c, o_hi);
-                if (MASK_OUT) {
-                    const bool rowless = row < 1 || row > n0 - 2;
+                if (ROWS_MASK_OUT || COLS_MASK_OUT) {
+                    const bool rowless = ROWS_MASK_OUT && (row < 1 || row > n0 - 2);
 #pragma unroll
                     for (int e = 0; e < NO; ++e) {
                         if (rowless) { o_lo[e] = make_float2(0.f, 0.f); o_hi[e] = o_lo[e]; }
-                        if (first_col) o_lo[e].x = 0.f;
-                        if (last_col) o_hi[e].y = 0.f;
+                        if (COLS_MASK_OUT && first_col) o_lo[e].x = 0.f;
+                        if (COLS_MASK_OUT && last_col) o_hi[e].y = 0.f;
                     }
                 }
                 if (cvalid) {
@@ -246,9 +250,9 @@ int lap2d_items(const int* n) {
     return p.nitems;
 }
 
-template <class F, bool PERIODIC>
+template <class F, bool PX, bool PY>
 static cudaError_t launch(const Lap2dParams& p, int block, cudaStream_t s) {
-    return launch_kernel(lap2d_kernel<F, PERIODIC, 4>, dim3(p.nitems), dim3(block), s, p);
+    return launch_kernel(lap2d_kernel<F, PX, PY, 4>, dim3(p.nitems), dim3(block), s, p);
 }
 
 static float2 sp(double v) { return make_float2((float)v, (float)v); }
@@ -258,13 +262,14 @@ cudaError_t launch_lap2d_fwd(const Problem& q) {
     lap2d_geometry(q, p, block);
     p.partials = q.partials;
     p.hin[0] = q.in[0]; p.out[0] = q.out[0];
-    if (q.op == 2) {
+    if (q.op != 1) {                                 // Gray-Scott: 2 periodic, 8 its slab form
         p.hin[1] = q.in[1]; p.out[1] = q.out[1];
         p.c[0] = sp(q.coef[0]); p.c[1] = sp(q.coef[1]); p.c[2] = sp(q.coef[2]); p.c[3] = sp(q.coef[2] + q.coef[3]);
-        return launch<GrayScottFwd, true>(p, block, q.stream);
+        if (q.op == 2) return launch<GrayScottFwd, true, true>(p, block, q.stream);
+        return launch<GrayScottFwd, false, true>(p, block, q.stream);
     }
     p.cin[0] = q.aux[0];
-    return launch<PoissonFwd, false>(p, block, q.stream);
+    return launch<PoissonFwd, false, false>(p, block, q.stream);
 }
 
 cudaError_t launch_lap2d_bwd(const Problem& q) {
@@ -272,13 +277,14 @@ cudaError_t launch_lap2d_bwd(const Problem& q) {
     lap2d_geometry(q, p, block);
     p.partials = nullptr;
     p.hin[0] = q.aux[0]; p.out[0] = q.out[0]; p.hscale[0] = sp(q.gscale[0]);
-    if (q.op == 2) {
+    if (q.op != 1) {
         p.hin[1] = q.aux[1]; p.out[1] = q.out[1]; p.hscale[1] = sp(q.gscale[1]);
         p.cin[0] = q.in[0]; p.cin[1] = q.in[1];
         p.c[0] = sp(q.coef[0]); p.c[1] = sp(q.coef[1]); p.c[2] = sp(q.coef[2]); p.c[3] = sp(q.coef[2] + q.coef[3]);
-        return launch<GrayScottBwd, true>(p, block, q.stream);
+        if (q.op == 2) return launch<GrayScottBwd, true, true>(p, block, q.stream);
+        return launch<GrayScottBwd, false, true>(p, block, q.stream);
     }
-    return launch<PoissonBwd, false>(p, block, q.stream);
+    return launch<PoissonBwd, false, false>(p, block, q.stream);
 }
 
 }  // namespace fpde

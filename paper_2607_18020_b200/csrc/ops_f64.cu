@@ -161,7 +161,7 @@ __device__ void residual_at(const F64Params& p, const Node& q, double* r) {
     case 1:                                               // Poisson
         r[0] = -(d2c(p, p.in[0], q, 0) + d2c(p, p.in[0], q, 1)) - p.aux[0][q.idx];
         break;
-    case 2: {                                             // Gray-Scott: coef = D_u, D_v, F, k
+    case 2: case 8: {                                     // Gray-Scott (8: its slab form): coef = D_u, D_v, F, k
         const double u = p.in[0][q.idx], v = p.in[1][q.idx];
         r[0] = p.coef[0] * (d2c(p, p.in[0], q, 0) + d2c(p, p.in[0], q, 1)) - u * v * v + p.coef[2] * (1.0 - u);
         r[1] = p.coef[1] * (d2c(p, p.in[1], q, 0) + d2c(p, p.in[1], q, 1)) + u * v * v - (p.coef[2] + p.coef[3]) * v;
@@ -255,7 +255,7 @@ __device__ void adjoint_at(const F64Params& p, const Node& q, double* g) {
     case 1:
         g[0] = -(G_d2c(p, 0, q, 0) + G_d2c(p, 0, q, 1));
         break;
-    case 2: {
+    case 2: case 8: {
         const double u = p.in[0][q.idx], v = p.in[1][q.idx];
         const double a = G(p, 0, q, 0, 0), b = G(p, 1, q, 0, 0);
         g[0] = p.coef[0] * (G_d2c(p, 0, q, 0) + G_d2c(p, 0, q, 1)) + a * (-v * v - p.coef[2]) + b * v * v;

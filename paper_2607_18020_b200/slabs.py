@@ -16,8 +16,8 @@ those rows' own neighbours).  So per step a rank
 Every array is stored once per rank with the widest halo; the forward call is handed a
 sub-range of planes (contiguous, because x is the slowest axis), so nothing is copied locally.
 An operator whose x axis is an interior axis is its own slab form (at the two ends of the
-domain the halo is simply absent); the periodic unsteady Navier-Stokes operator has a slab form
-with a non-periodic x axis (`ns_3d_t_xslab`).  The kernels are the single-GPU kernels; this
+domain the halo is simply absent); the periodic operators (unsteady Navier-Stokes, Gray-Scott) have
+slab forms with a non-periodic x axis (`ns_3d_t_xslab`, `grayscott_2d_xslab`).  The kernels are the single-GPU kernels; this
 module only plans the ranges and moves the halo planes (torch.distributed point-to-point, or
 plain copies when several slabs live in one process).
 """
@@ -35,8 +35,9 @@ SLAB_OP = {
     W.NS_2D_STEADY: W.NS_2D_STEADY,
     W.NS_3D_STEADY: W.NS_3D_STEADY,
     W.NS_3D_T: W.NS_3D_T_XSLAB,
+    W.GRAYSCOTT_2D: W.GRAYSCOTT_2D_XSLAB,
 }
-RADIUS = {W.POISSON_2D: 1, W.HELMHOLTZ_3D_O4: 2, W.NS_2D_STEADY: 1, W.NS_3D_STEADY: 1, W.NS_3D_T: 1}
+RADIUS = {W.POISSON_2D: 1, W.HELMHOLTZ_3D_O4: 2, W.NS_2D_STEADY: 1, W.NS_3D_STEADY: 1, W.NS_3D_T: 1, W.GRAYSCOTT_2D: 1}
 
 
 @dataclass(frozen=True)

@@ -40,7 +40,7 @@ def test_registry():
     expect = {W.BURGERS_1D_T: (2, 1, 0, 1, 1, 1), W.POISSON_2D: (2, 1, 1, 1, 0, 1), W.GRAYSCOTT_2D: (2, 2, 0, 2, 4, 1),
               W.HELMHOLTZ_3D_O4: (3, 1, 1, 1, 1, 2), W.NS_3D_T: (4, 4, 0, 4, 1, 1),
               W.NS_2D_STEADY: (2, 3, 0, 3, 1, 1), W.NS_3D_STEADY: (3, 4, 0, 4, 1, 1),
-              W.NS_3D_T_XSLAB: (4, 4, 0, 4, 1, 1)}
+              W.NS_3D_T_XSLAB: (4, 4, 0, 4, 1, 1), W.GRAYSCOTT_2D_XSLAB: (2, 2, 0, 2, 4, 1)}
     for op, e in expect.items():
         i = B.op_info(op)
         assert (i.ndim, i.nfields, i.nsources, i.nresiduals, i.ncoeffs, i.radius) == e
@@ -62,6 +62,7 @@ def test_row_counts_and_workspace():
     assert B.row_count(W.NS_2D_STEADY, (128, 128)) == 126 * 126
     assert B.row_count(W.NS_3D_STEADY, (64, 32, 16)) == 62 * 30 * 14
     assert B.row_count(W.NS_3D_T_XSLAB, (34, 8, 8, 16)) == 32 * 8 * 8 * 14
+    assert B.row_count(W.GRAYSCOTT_2D_XSLAB, (18, 32)) == 16 * 32
     for name in W.CONFIG_ORDER + W.EXTRA_CONFIGS + W.SLAB_CONFIGS:
         c = W.CONFIGS[name]
         assert 0 < B.workspace_bytes(c["op"], c["shape"]) < (64 << 20)

@@ -21,6 +21,7 @@ CASES = [
     ("ns2d_steady_4096", (3, 4)), ("ns2d_steady_4096", (36, 40)),
     ("ns3d_steady_256", (3, 3, 4)), ("ns3d_steady_256", (7, 5, 12)),
     ("ns_tgv_xslab_34", (3, 3, 3, 4)), ("ns_tgv_xslab_34", (6, 5, 4, 8)),
+    ("grayscott_xslab_1026", (3, 4)), ("grayscott_xslab_1026", (9, 12)),
 ]
 
 

@@ -28,6 +28,7 @@ MEDIUM = [
     ("ns3d_steady_256", (20, 9, 260)),      # warp edges inside a z line, a ragged column block
     ("ns_tgv_xslab_34", (34, 21, 20, 16)),  # slab form: first / last x-plane without rows, three plane chunks
     ("ns_tgv_xslab_34", (17, 8, 8, 12)),    # t groups that straddle warps
+    ("grayscott_xslab_1026", (203, 300)),   # slab form: first / last row without residual rows, periodic columns
 ]
 TINY = [
     ("burgers_256x128", (4, 4)),
@@ -48,6 +49,8 @@ TINY = [
     ("ns3d_steady_256", (7, 5, 132)),
     ("ns_tgv_xslab_34", (3, 3, 3, 4)),
     ("ns_tgv_xslab_34", (5, 6, 7, 12)),
+    ("grayscott_xslab_1026", (3, 4)),
+    ("grayscott_xslab_1026", (17, 12)),
 ]
 FULL = [
     ("grayscott_4096", None),

@@ -22,6 +22,8 @@ CASES = [
     ("poisson_1024", (40, 36), 4),
     ("ns2d_steady_4096", (30, 40), 2),
     ("ns3d_steady_256", (14, 6, 8), 3),
+    ("grayscott_4096", (64, 96), 1),
+    ("grayscott_4096", (67, 200), 3),
 ]
 
 

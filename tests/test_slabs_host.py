@@ -20,7 +20,8 @@ def _expected_plane(plan, local):
 
 @pytest.mark.parametrize("op,shape,world", [(W.NS_3D_T, (16, 4, 4, 8), 1), (W.NS_3D_T, (16, 4, 4, 8), 2),
                                             (W.NS_3D_T, (17, 4, 4, 8), 3), (W.HELMHOLTZ_3D_O4, (19, 6, 8), 3),
-                                            (W.POISSON_2D, (11, 8), 4), (W.NS_3D_STEADY, (9, 5, 8), 2)])
+                                            (W.POISSON_2D, (11, 8), 4), (W.NS_3D_STEADY, (9, 5, 8), 2),
+                                            (W.GRAYSCOTT_2D, (10, 8), 2)])
 def test_ranges_and_transfers(op, shape, world):
     ps = S.plans(op, shape, world)
     R = ps[0].radius
@@ -53,7 +54,7 @@ def test_too_thin_slabs_are_refused():
     with pytest.raises(ValueError):
         S.plans(W.HELMHOLTZ_3D_O4, (12, 6, 8), 4)       # 3 planes per rank < 2 * radius
     with pytest.raises(ValueError):
-        S.plans(W.GRAYSCOTT_2D, (16, 8), 2)             # no slab form
+        S.plans(W.BURGERS_1D_T, (16, 8), 2)             # no slab form
 
 
 def test_local_exchange_on_cpu_tensors():
