@@ -48,10 +48,11 @@ constexpr int FUSED2D_OWN = 30;     // float4 columns a warp owns (lanes 1..30)
 
 struct FusedPoisson {       // r = -Lap u - f ; g = -Lap G
     static constexpr int NF = 1, NS = 1, NE = 1;
-    static constexpr bool PERIODIC = false, FIELD_LATERAL_IN_BWD = false;
-    __device__ static __forceinline__ float2 lap(const float2* c, float2 m, float2 z, float2 p, float2 l, float2 r) {
+    static constexpr bool PERIODIC = false, FIELD_LATERAL_IN_BWD = false, LATERAL_SUM = true;
+    // l: the SUM of the two lateral neighbours (LATERAL_SUM operators get it in fl / rl; fr / rr unused)
+    __device__ static __forceinline__ float2 lap(const float2* c, float2 m, float2 z, float2 p, float2 l, float2) {
         const float2 m2 = splat2(-2.f);
-        return fma2(fma2(z, m2, add2(m, p)), c[0], mul2(fma2(z, m2, add2(l, r)), c[1]));
+        return fma2(fma2(z, m2, add2(m, p)), c[0], mul2(fma2(z, m2, l), c[1]));
     }
     __device__ static __forceinline__ void fwd(const float2* c, const float2* fm, const float2* f0, const float2* fp,
                                                const float2* fl, const float2* fr, const float2* s, float2* r) {
@@ -67,7 +68,7 @@ struct FusedPoisson {       // r = -Lap u - f ; g = -Lap G
 
 struct FusedGrayScott {     // c: 1/h0^2, 1/h1^2, D_u, D_v, F, F+k
     static constexpr int NF = 2, NS = 0, NE = 2;
-    static constexpr bool PERIODIC = true, FIELD_LATERAL_IN_BWD = false;
+    static constexpr bool PERIODIC = true, FIELD_LATERAL_IN_BWD = false, LATERAL_SUM = true;
     __device__ static __forceinline__ void fwd(const float2* c, const float2* fm, const float2* f0, const float2* fp,
                                                const float2* fl, const float2* fr, const float2* s, float2* r) {
         const float2 u = f0[0], w = f0[1];
@@ -93,7 +94,7 @@ struct FusedGrayScott {     // c: 1/h0^2, 1/h1^2, D_u, D_v, F, F+k
 
 struct FusedNs2d {          // c: 1/(2 h0), 1/(2 h1), -nu/h0^2, -nu/h1^2 ; fields u,v,p ; residuals mom_x, mom_y, div
     static constexpr int NF = 3, NS = 0, NE = 3;
-    static constexpr bool PERIODIC = false, FIELD_LATERAL_IN_BWD = true;
+    static constexpr bool PERIODIC = false, FIELD_LATERAL_IN_BWD = true, LATERAL_SUM = false;
     __device__ static __forceinline__ void fwd(const float2* c, const float2* fm, const float2* f0, const float2* fp,
                                                const float2* fl, const float2* fr, const float2* s, float2* r) {
         const float2 us = mul2(f0[0], c[0]), vs = mul2(f0[1], c[1]);
@@ -185,8 +186,14 @@ __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams 
     auto lateral = [&](const V4& c, V4& L, V4& R) {
         const float l1 = __shfl_up_sync(FULL_MASK, c.hi.y, 1);
         const float r1 = __shfl_down_sync(FULL_MASK, c.lo.x, 1);
-        L = shift_left(c, l1);
-        R = shift_right(c, r1);
+        if (OP::LATERAL_SUM) {                           // only l + r is wanted: four scalar adds, no shifted copies
+            L.lo = make_float2(l1 + c.lo.y, c.lo.x + c.hi.x);
+            L.hi = make_float2(c.lo.y + c.hi.y, c.hi.x + r1);
+            R = L;
+        } else {
+            L = shift_left(c, l1);
+            R = shift_right(c, r1);
+        }
     };
     // r at row j from the field rows j-1, j, j+1; zero where the operator has no row
     auto residual_row = [&](int j, const V4 (&Fm)[NF], const V4 (&F0)[NF], const V4 (&Fp)[NF], const V4 (&S0)[NSA],
