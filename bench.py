@@ -549,6 +549,46 @@ def main():
                 "pair_frac": (fb + bb) * Nk * args.steps / (total_ms * 1e-3) / 1e9 / peak}
     if args.slabs:
         roofline["note"] = "per-call times include the halo exchange of the step (and the loss all-reduce)"
+    elif not args.single_pass:
+        # the dominant kernel launched K times back to back between ONE pair of events: its
+        # sustained per-launch time, with the ramp and tail of consecutive launches overlapping
+        # (programmatic dependent launch) as they do inside a step
+        call = prob.bwd if dom == 1 else prob.fwd
+        for _ in range(3):
+            call()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        s0.record()
+        for _ in range(args.steps):
+            call()
+        s1.record(); torch.cuda.synchronize()
+        sus_ms = s0.elapsed_time(s1) / args.steps
+        roofline["sustained"] = {"avg_ms": sus_ms, "achieved": dom_bytes / (sus_ms * 1e-3) / 1e9,
+                                 "frac": dom_bytes / (sus_ms * 1e-3) / 1e9 / peak,
+                                 "what": "%d consecutive launches of the dominant kernel between one event pair" % args.steps}
+
+    # The same step over about two seconds: on these parts the SM clock comes down from its boost
+    # value a few tenths of a second into a sustained load (power management), and these kernels
+    # are bound by instruction issue and latency, so the long-run figure is the lower one.
+    sustained = None
+    if world == 1 and not args.no_extras and not args.slabs:
+        s_sampler = ClockSampler(torch, local_rank)
+        n_sus = max(200, int(2000.0 / max(total_ms / args.steps, 1e-3)))
+        half = n_sus // 2
+        ea, eb, ec = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        torch.cuda.synchronize()
+        s_sampler.start()
+        ea.record()
+        for k in range(n_sus):
+            if k == half:
+                eb.record()
+            prob.fwd(); prob.bwd()
+        ec.record(); torch.cuda.synchronize()
+        s_sampler.stop()
+        sus_ms = eb.elapsed_time(ec) / (n_sus - half)
+        sustained = {"steps": n_sus, "seconds": ea.elapsed_time(ec) * 1e-3, "ms_per_step": sus_ms,
+                     "value": N / (sus_ms * 1e-3), "pair_frac": (fb + bb) * Nk / (sus_ms * 1e-3) / 1e9 / peak,
+                     "clocks": s_sampler.summary(), "what": "second half of a ~2 s back-to-back run of the same step"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -566,6 +606,7 @@ def main():
                 "what": "fpde_loss_grad_host from pinned host buffers: H2D fields, fwd, bwd, D2H gradients + loss, sync"},
         "gpu_launches": (2 if args.single_pass else LAUNCHES_PER_STEP) * args.steps,
         "roofline": roofline,
+        "sustained": sustained,
         "loss": float(prob.loss[-1].item()),
     }
     if world == 1 and not args.no_extras:
