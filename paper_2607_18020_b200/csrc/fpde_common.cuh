@@ -59,6 +59,21 @@ __device__ __forceinline__ V4 ldv4(const float* p) {
 __device__ __forceinline__ void stv4(float* p, float2 lo, float2 hi) {
     *reinterpret_cast<float4*>(p) = make_float4(lo.x, lo.y, hi.x, hi.y);
 }
+// The same accesses at an element offset from an array base.  OFF32: the byte offset is formed
+// as an unsigned 32-bit number (arrays of at most 2^30 floats), which lets the address be a
+// 64-bit base plus a 32-bit register instead of a 64-bit add per access; the kernels spend a
+// sixth of their issue slots on addresses otherwise.
+template <bool OFF32>
+__device__ __forceinline__ const float* at_off(const float* base, int eoff) {
+    if (OFF32) return reinterpret_cast<const float*>(reinterpret_cast<const char*>(base) + 4u * (unsigned)eoff);
+    return base + eoff;
+}
+template <bool OFF32>
+__device__ __forceinline__ float* at_off(float* base, int eoff) {
+    if (OFF32) return reinterpret_cast<float*>(reinterpret_cast<char*>(base) + 4u * (unsigned)eoff);
+    return base + eoff;
+}
+
 __device__ __forceinline__ V4 v4zero() { V4 v; v.lo = make_float2(0.f, 0.f); v.hi = v.lo; return v; }
 __device__ __forceinline__ V4 v4add(V4 a, V4 b) { V4 r; r.lo = add2(a.lo, b.lo); r.hi = add2(a.hi, b.hi); return r; }
 __device__ __forceinline__ V4 v4sub(V4 a, V4 b) { V4 r; r.lo = sub2(a.lo, b.lo); r.hi = sub2(a.hi, b.hi); return r; }

@@ -115,7 +115,7 @@ __device__ __forceinline__ void t_neighbours(const V4& c, const float* __restric
 // ------------------------------------------------------------------------------------------
 // forward
 // ------------------------------------------------------------------------------------------
-template <bool TSAFE, int MINB>
+template <bool TSAFE, int MINB, bool O32>
 __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
     pdl_wait_then_trigger();
     int a0, a1;
@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
         const int om = xplane(p, a0 - 1) * PS + ix.rowoff + ix.col;
         const int oc = a0 * PS + ix.rowoff + ix.col;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) { A[k] = ldv4(fp[k] + om); B[k] = ldv4(fp[k] + oc); }
+        for (int k = 0; k < 4; ++k) { A[k] = ldv4(at_off<O32>(fp[k], om)); B[k] = ldv4(at_off<O32>(fp[k], oc)); }
     }
     float2 acc[4];
 #pragma unroll
@@ -146,16 +146,16 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
             const int af = xplane(p, a + 1 + p.prefetch);
             const int po = af * PS + ix.rowoff + ix.col;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) prefetch_l2(fp[k] + po);
+            for (int k = 0; k < 4; ++k) prefetch_l2(at_off<O32>(fp[k], po));
         }
         V4 Ym[4], Yp[4], Zm[4], Zp[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            W2[k] = ldv4(fp[k] + ap + ix.rowoff + ix.col);
-            Ym[k] = ldv4(fp[k] + pl + ix.ymoff + ix.col);
-            Yp[k] = ldv4(fp[k] + pl + ix.ypoff + ix.col);
-            Zm[k] = ldv4(fp[k] + pl + ix.rowoff + ix.zmcol);
-            Zp[k] = ldv4(fp[k] + pl + ix.rowoff + ix.zpcol);
+            W2[k] = ldv4(at_off<O32>(fp[k], ap + ix.rowoff + ix.col));
+            Ym[k] = ldv4(at_off<O32>(fp[k], pl + ix.ymoff + ix.col));
+            Yp[k] = ldv4(at_off<O32>(fp[k], pl + ix.ypoff + ix.col));
+            Zm[k] = ldv4(at_off<O32>(fp[k], pl + ix.rowoff + ix.zmcol));
+            Zp[k] = ldv4(at_off<O32>(fp[k], pl + ix.rowoff + ix.zpcol));
         }
         float l1[3], r1[3];
 #pragma unroll
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
             const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                stv4(p.out[e] + off, o[e][0], o[e][1]);
+                stv4(at_off<O32>(p.out[e], off), o[e][0], o[e][1]);
                 acc[e] = fma2(o[e][0], o[e][0], fma2(o[e][1], o[e][1], acc[e]));
             }
         }
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(128, MINB) ns_fwd_kernel(const NsParams p) {
 //   g_p(P) = sum_q [ G_q(P-a_q) - G_q(P+a_q) ] / (2 h_{a_q})
 // G_e = gscale_e * gres_e; the scales are folded into the constants.
 // ------------------------------------------------------------------------------------------
-template <bool TSAFE, int MINB>
+template <bool TSAFE, int MINB, bool O32>
 __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
     pdl_wait_then_trigger();
     int a0, a1;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
         const int om = xplane(p, a0 - 1) * PS + ix.rowoff + ix.col;
         const int oc = a0 * PS + ix.rowoff + ix.col;
 #pragma unroll
-        for (int k = 0; k < 7; ++k) { A[k] = ldv4(ap[k] + om); B[k] = ldv4(ap[k] + oc); }
+        for (int k = 0; k < 7; ++k) { A[k] = ldv4(at_off<O32>(ap[k], om)); B[k] = ldv4(at_off<O32>(ap[k], oc)); }
         // upstream arrays count as zero on planes without rows
         if (xdead(p, a0 - 1)) zero_from<7>(A, 3);
         if (xdead(p, a0)) zero_from<7>(B, 3);
@@ -227,16 +227,16 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
             const int af = xplane(p, a + 1 + p.prefetch);
             const int po = af * PS + ix.rowoff + ix.col;
 #pragma unroll
-            for (int k = 0; k < 7; ++k) prefetch_l2(ap[k] + po);
+            for (int k = 0; k < 7; ++k) prefetch_l2(at_off<O32>(ap[k], po));
         }
         V4 Ym[7], Yp[7], Zm[7], Zp[7];
 #pragma unroll
         for (int k = 0; k < 7; ++k) {
-            W2[k] = ldv4(ap[k] + apl + ix.rowoff + ix.col);
-            Ym[k] = ldv4(ap[k] + pl + ix.ymoff + ix.col);
-            Yp[k] = ldv4(ap[k] + pl + ix.ypoff + ix.col);
-            Zm[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zmcol);
-            Zp[k] = ldv4(ap[k] + pl + ix.rowoff + ix.zpcol);
+            W2[k] = ldv4(at_off<O32>(ap[k], apl + ix.rowoff + ix.col));
+            Ym[k] = ldv4(at_off<O32>(ap[k], pl + ix.ymoff + ix.col));
+            Yp[k] = ldv4(at_off<O32>(ap[k], pl + ix.ypoff + ix.col));
+            Zm[k] = ldv4(at_off<O32>(ap[k], pl + ix.rowoff + ix.zmcol));
+            Zp[k] = ldv4(at_off<O32>(ap[k], pl + ix.rowoff + ix.zpcol));
         }
         if (xdead(p, a + 1)) zero_from<7>(W2, 3);
         if (xdead(p, a)) { zero_from<7>(Ym, 3); zero_from<7>(Yp, 3); zero_from<7>(Zm, 3); zero_from<7>(Zp, 3); }
@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(128, MINB) ns_bwd_kernel(const NsParams p) {
         if (ix.valid) {
             const int off = pl + ix.rowoff + ix.col;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) stv4(p.out[e] + off, o[e][0], o[e][1]);
+            for (int e = 0; e < 4; ++e) stv4(at_off<O32>(p.out[e], off), o[e][0], o[e][1]);
         }
     };
 
@@ -288,6 +288,13 @@ static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
 }
 
 static bool ns_tsafe(const NsParams& p) { return 32 % p.nt4 == 0; }
+
+// 32-bit byte offsets are enough for arrays of at most 2^30 floats (FPDE_NS_OFF32=0: never)
+static bool ns_off32(const Problem& q) {
+    const int64_t N = (int64_t)q.n[0] * q.n[1] * q.n[2] * q.n[3];
+    const char* s = std::getenv("FPDE_NS_OFF32");
+    return !(s && s[0] == '0') && N <= ((int64_t)1 << 30);
+}
 
 // Grid of a launch: all work items, or those of the plane chunks [chunk_lo, chunk_hi) of the
 // problem (items are ordered with the plane chunk slowest, so a chunk range is an item range).
@@ -327,9 +334,11 @@ cudaError_t launch_ns_fwd(const Problem& q) {
     const int minb = env_int("FPDE_NS_MINB_F", 3);
     cudaError_t ce;
     const dim3 grid = ns_range(q, p);
-    if (!ns_tsafe(p)) ce = launch_kernel(ns_fwd_kernel<false, 3>, grid, block, q.stream, p);
-    else if (minb == 3) ce = launch_kernel(ns_fwd_kernel<true, 3>, grid, block, q.stream, p);
-    else ce = launch_kernel(ns_fwd_kernel<true, 4>, grid, block, q.stream, p);
+    const bool o32 = ns_off32(q);
+    if (!ns_tsafe(p)) ce = launch_kernel(ns_fwd_kernel<false, 3, false>, grid, block, q.stream, p);
+    else if (minb != 3) ce = launch_kernel(ns_fwd_kernel<true, 4, false>, grid, block, q.stream, p);
+    else if (o32) ce = launch_kernel(ns_fwd_kernel<true, 3, true>, grid, block, q.stream, p);
+    else ce = launch_kernel(ns_fwd_kernel<true, 3, false>, grid, block, q.stream, p);
     return ce;
 }
 
@@ -347,9 +356,11 @@ cudaError_t launch_ns_bwd(const Problem& q) {
     const int minb = env_int("FPDE_NS_MINB_B", 2);
     cudaError_t ce;
     const dim3 grid = ns_range(q, p);
-    if (!ns_tsafe(p)) ce = launch_kernel(ns_bwd_kernel<false, 2>, grid, block, q.stream, p);
-    else if (minb == 3) ce = launch_kernel(ns_bwd_kernel<true, 3>, grid, block, q.stream, p);
-    else ce = launch_kernel(ns_bwd_kernel<true, 2>, grid, block, q.stream, p);
+    const bool o32 = ns_off32(q);
+    if (!ns_tsafe(p)) ce = launch_kernel(ns_bwd_kernel<false, 2, false>, grid, block, q.stream, p);
+    else if (minb == 3) ce = launch_kernel(ns_bwd_kernel<true, 3, false>, grid, block, q.stream, p);
+    else if (o32) ce = launch_kernel(ns_bwd_kernel<true, 2, true>, grid, block, q.stream, p);
+    else ce = launch_kernel(ns_bwd_kernel<true, 2, false>, grid, block, q.stream, p);
     return ce;
 }
 
