@@ -57,10 +57,10 @@ __device__ __forceinline__ V4 ns3d_zmask(const Ns3dThread& t, V4 v) {
 
 // array k at plane r (clamped into the array) at the thread's own float4; with `check`, an
 // upstream float4 whose plane or row is outside the rows reads as zero
-template <bool BWD, bool PRE>
+template <bool BWD, bool PRE, bool O32>
 __device__ __forceinline__ V4 ns3d_load_own(const Ns3dParams& p, const Ns3dThread& t, int k, int r, bool check) {
     const int rr = max(0, min(t.n0 - 1, r));
-    V4 v = ldv4(p.a[k] + rr * t.PS + t.rowoff);
+    V4 v = ldv4(at_off<O32>(p.a[k], rr * t.PS + t.rowoff));
     if (BWD && !PRE && k >= 3) {
         v = ns3d_zmask(t, v);
         if (check && (t.y_dead || r < 1 || r > t.n0 - 2)) v = v4zero();
@@ -74,7 +74,7 @@ __device__ __forceinline__ V4 ns3d_load_own(const Ns3dParams& p, const Ns3dThrea
 // PRE (adjoint only): the upstream arrays are already zero off the rows (residual arrays the
 // forward kernel of the same call wrote), so nothing is zero-extended here; clamped reads beyond
 // the array land in the zero shell.
-template <bool BWD, bool EDGE, int NA, bool PRE>
+template <bool BWD, bool EDGE, int NA, bool PRE, bool O32>
 __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread& t, int a, const V4 (&W0)[NA],
                                           const V4 (&W1)[NA], V4 (&W2)[NA], float2 (&acc)[4]) {
     constexpr int G0 = 3;                            // adjoint: first upstream array
@@ -83,17 +83,17 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
     if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 1 + p.prefetch <= min(t.a1, t.n0 - 1)) {
         const int po = (a + 1 + p.prefetch) * t.PS + t.rowoff;
 #pragma unroll
-        for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(p.a[k] + po);
+        for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(at_off<O32>(p.a[k], po));
     }
     V4 Ym[NA], Yp[NA], Zm[NA], Zp[NA];
     float E[NA];
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
-        W2[k] = ns3d_load_own<BWD, PRE>(p, t, k, a + 1, EDGE);
-        Ym[k] = ldv4(p.a[k] + pl + t.ymoff);
-        Yp[k] = ldv4(p.a[k] + pl + t.ypoff);
+        W2[k] = ns3d_load_own<BWD, PRE, O32>(p, t, k, a + 1, EDGE);
+        Ym[k] = ldv4(at_off<O32>(p.a[k], pl + t.ymoff));
+        Yp[k] = ldv4(at_off<O32>(p.a[k], pl + t.ypoff));
         E[k] = 0.f;
-        if (t.efetch) E[k] = __ldg(p.a[k] + pl + t.eoff);
+        if (t.efetch) E[k] = __ldg(at_off<O32>(p.a[k], pl + t.eoff));
     }
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
@@ -138,13 +138,15 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
         const int off = pl + t.rowoff;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            stv4(p.out[e] + off, o[e][0], o[e][1]);
+            stv4(at_off<O32>(p.out[e], off), o[e][0], o[e][1]);
             if (!BWD) acc[e] = fma2(o[e][0], o[e][0], fma2(o[e][1], o[e][1], acc[e]));
         }
     }
 }
 
-template <bool BWD, int MINB, bool PRE = false>
+// O32: 32-bit byte offsets from the array bases (arrays of at most 2^30 floats); used where the
+// build comes out without spills (forward, and the adjoint without zero-extension)
+template <bool BWD, int MINB, bool PRE = false, bool O32 = false>
 __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     constexpr int NA = BWD ? 7 : 4;
     pdl_wait_then_trigger();
@@ -184,22 +186,22 @@ __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
         for (int d = 1; d <= p.prefetch && a0 + d <= min(a1, p.n0 - 1); ++d) {
             const int po = (a0 + d) * t.PS + t.rowoff;
 #pragma unroll
-            for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(p.a[k] + po);
+            for (int k = 0; k < NA; ++k) ns3d_prefetch_l2(at_off<O32>(p.a[k], po));
         }
     }
     V4 A[NA], B[NA], Cc[NA];
 #pragma unroll
     for (int k = 0; k < NA; ++k) {
-        A[k] = ns3d_load_own<BWD, PRE>(p, t, k, a0 - 1, true);
-        B[k] = ns3d_load_own<BWD, PRE>(p, t, k, a0, true);
+        A[k] = ns3d_load_own<BWD, PRE, O32>(p, t, k, a0 - 1, true);
+        B[k] = ns3d_load_own<BWD, PRE, O32>(p, t, k, a0, true);
     }
     float2 acc[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
 
     auto step = [&](int a, const V4 (&W0)[NA], const V4 (&W1)[NA], V4 (&W2)[NA]) {
-        if (!PRE && (y_edge_block || a <= 1 || a >= p.n0 - 2)) ns3d_step<BWD, true, NA, PRE>(p, t, a, W0, W1, W2, acc);
-        else ns3d_step<BWD, false, NA, PRE>(p, t, a, W0, W1, W2, acc);
+        if (!PRE && (y_edge_block || a <= 1 || a >= p.n0 - 2)) ns3d_step<BWD, true, NA, PRE, O32>(p, t, a, W0, W1, W2, acc);
+        else ns3d_step<BWD, false, NA, PRE, O32>(p, t, a, W0, W1, W2, acc);
     };
     for (int a = a0; a < a1; a += 3) {
         step(a, A, B, Cc);
@@ -237,6 +239,12 @@ static void ns3d_geometry(const int* n, Ns3dParams& p, dim3& block) {
     if (p.prefetch < 0 || p.prefetch >= p.n0) p.prefetch = 0;
 }
 
+// 32-bit byte offsets are enough for arrays of at most 2^30 floats
+static bool ns3d_off32(const Problem& q) {
+    const char* s = std::getenv("FPDE_NS3D_OFF32");
+    return !(s && s[0] == '0') && (int64_t)q.n[0] * q.n[1] * q.n[2] <= ((int64_t)1 << 30);
+}
+
 int ns3d_items(const int* n) {
     Ns3dParams p{}; dim3 block;
     ns3d_geometry(n, p, block);
@@ -259,6 +267,7 @@ cudaError_t launch_ns3d_fwd(const Problem& q) {
     ns3d_consts(q, ones, p.k);
     p.partials = q.partials;
     if (env_int("FPDE_NS3D_MINB_F", 3) == 4) return launch_kernel(ns3d_kernel<false, 4>, dim3(p.nitems), block, q.stream, p);
+    if (ns3d_off32(q)) return launch_kernel(ns3d_kernel<false, 3, false, true>, dim3(p.nitems), block, q.stream, p);
     return launch_kernel(ns3d_kernel<false, 3>, dim3(p.nitems), block, q.stream, p);
 }
 
@@ -269,7 +278,10 @@ cudaError_t launch_ns3d_bwd(const Problem& q) {
     for (int k = 0; k < 4; ++k) { p.a[3 + k] = q.aux[k]; p.out[k] = q.out[k]; }
     ns3d_consts(q, q.gscale, p.k);
     p.partials = nullptr;
-    if (q.gres_zero_off_rows) return launch_kernel(ns3d_kernel<true, 2, true>, dim3(p.nitems), block, q.stream, p);
+    if (q.gres_zero_off_rows) {
+        if (ns3d_off32(q)) return launch_kernel(ns3d_kernel<true, 2, true, true>, dim3(p.nitems), block, q.stream, p);
+        return launch_kernel(ns3d_kernel<true, 2, true>, dim3(p.nitems), block, q.stream, p);
+    }
     if (env_int("FPDE_NS3D_MINB_B", 2) == 3) return launch_kernel(ns3d_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
     return launch_kernel(ns3d_kernel<true, 2>, dim3(p.nitems), block, q.stream, p);
 }
