@@ -148,7 +148,7 @@ struct FusedNs2d {          // c: 1/(2 h0), 1/(2 h1), -nu/h0^2, -nu/h1^2 ; field
 };
 
 // ---- engine ------------------------------------------------------------------------------------
-template <class OP, int MINB>
+template <class OP, int MINB, bool O32 = false>
 __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams p) {
     constexpr int NF = OP::NF, NS = OP::NS, NE = OP::NE;
     constexpr int NSA = NS > 0 ? NS : 1;
@@ -177,9 +177,9 @@ __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams 
     auto load_row = [&](int j, V4 (&F)[NF], V4 (&S)[NSA]) {
         const int off = row_of(j) * n1 + col;
 #pragma unroll
-        for (int k = 0; k < NF; ++k) F[k] = ldv4(p.f[k] + off);
+        for (int k = 0; k < NF; ++k) F[k] = ldv4(at_off<O32>(p.f[k], off));
 #pragma unroll
-        for (int k = 0; k < NS; ++k) S[k] = ldv4(p.src[k] + off);
+        for (int k = 0; k < NS; ++k) S[k] = ldv4(at_off<O32>(p.src[k], off));
     };
     // left / right neighbours along y of a row held in registers (lanes 0 / 31 get their own
     // value back on the outer side: what depends on it is never used)
@@ -244,9 +244,9 @@ __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams 
         if (p.prefetch > 0 && (lane & 7) == 0 && i + 3 + p.prefetch <= a1 + 1) {
             const int off = row_of(i + 3 + p.prefetch) * n1 + col;
 #pragma unroll
-            for (int k = 0; k < NF; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.f[k] + off));
+            for (int k = 0; k < NF; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(at_off<O32>(p.f[k], off)));
 #pragma unroll
-            for (int k = 0; k < NS; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.src[k] + off));
+            for (int k = 0; k < NS; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(at_off<O32>(p.src[k], off)));
         }
         residual_row(i + 1, F0, Fp, Fpp, Sp, Rp);
         V4 RL[NE], RR[NE], FL[NF], FR[NF];
@@ -272,10 +272,10 @@ __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams 
         if (own) {
             const int off = i * n1 + col;
 #pragma unroll
-            for (int k = 0; k < NF; ++k) stv4(p.g[k] + off, g[k][0], g[k][1]);
+            for (int k = 0; k < NF; ++k) stv4(at_off<O32>(p.g[k], off), g[k][0], g[k][1]);
 #pragma unroll
             for (int e = 0; e < NE; ++e) {
-                if (p.res[e] != nullptr) stv4(p.res[e] + off, R0[e].lo, R0[e].hi);
+                if (p.res[e] != nullptr) stv4(at_off<O32>(p.res[e], off), R0[e].lo, R0[e].hi);
                 acc[e] = fma2(R0[e].lo, R0[e].lo, fma2(R0[e].hi, R0[e].hi, acc[e]));
             }
         }
@@ -370,23 +370,31 @@ cudaError_t launch_fused2d(const Problem& q, float* const* res) {
     fused2d_geometry(q.op, q.n, p);
     p.partials = q.partials;
     p.gs = sp(2.0 / (double)q.rows);
+    // 32-bit byte offsets from the array bases for arrays of at most 2^30 floats
+    const char* o32s = std::getenv("FPDE_FUSED2D_OFF32");
+    const bool o32 = !(o32s && o32s[0] == '0') && (int64_t)q.n[0] * q.n[1] <= ((int64_t)1 << 30);
     const double h0 = q.h[0], h1 = q.h[1];
     switch (q.op) {
     case 1:
         p.f[0] = q.in[0]; p.src[0] = q.aux[0]; p.g[0] = q.out[0]; p.res[0] = res ? res[0] : nullptr;
         p.c[0] = sp(1.0 / (h0 * h0)); p.c[1] = sp(1.0 / (h1 * h1));
+        if (o32) return launch_kernel(fused2d_kernel<FusedPoisson, 4, true>, dim3(p.nitems), dim3(128), q.stream, p);
         return launch_kernel(fused2d_kernel<FusedPoisson, 4>, dim3(p.nitems), dim3(128), q.stream, p);
     case 2:
         for (int k = 0; k < 2; ++k) { p.f[k] = q.in[k]; p.g[k] = q.out[k]; p.res[k] = res ? res[k] : nullptr; }
         p.c[0] = sp(1.0 / (h0 * h0)); p.c[1] = sp(1.0 / (h1 * h1));
         p.c[2] = sp(q.coef[0]); p.c[3] = sp(q.coef[1]); p.c[4] = sp(q.coef[2]); p.c[5] = sp(q.coef[2] + q.coef[3]);
         if (fused2d_minb(2) == 3) return launch_kernel(fused2d_kernel<FusedGrayScott, 3>, dim3(p.nitems), dim3(128), q.stream, p);
+        if (o32) return launch_kernel(fused2d_kernel<FusedGrayScott, 4, true>, dim3(p.nitems), dim3(128), q.stream, p);
         return launch_kernel(fused2d_kernel<FusedGrayScott, 4>, dim3(p.nitems), dim3(128), q.stream, p);
     case 5:
         for (int k = 0; k < 3; ++k) { p.f[k] = q.in[k]; p.g[k] = q.out[k]; p.res[k] = res ? res[k] : nullptr; }
         p.c[0] = sp(0.5 / h0); p.c[1] = sp(0.5 / h1);
         p.c[2] = sp(-q.coef[0] / (h0 * h0)); p.c[3] = sp(-q.coef[0] / (h1 * h1));
-        if (fused2d_minb(5) == 3) return launch_kernel(fused2d_kernel<FusedNs2d, 3>, dim3(p.nitems), dim3(128), q.stream, p);
+        if (fused2d_minb(5) == 3) {
+            if (o32) return launch_kernel(fused2d_kernel<FusedNs2d, 3, true>, dim3(p.nitems), dim3(128), q.stream, p);
+            return launch_kernel(fused2d_kernel<FusedNs2d, 3>, dim3(p.nitems), dim3(128), q.stream, p);
+        }
         return launch_kernel(fused2d_kernel<FusedNs2d, 2>, dim3(p.nitems), dim3(128), q.stream, p);
     }
     return cudaErrorInvalidValue;

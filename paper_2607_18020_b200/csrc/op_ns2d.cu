@@ -38,7 +38,7 @@ struct Ns2dParams {
     int prefetch;           // rows ahead of the window to pull into L2 (0 = off)
 };
 
-template <bool BWD>
+template <bool BWD, bool O32 = false>
 __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
     constexpr int NA = BWD ? 5 : 3;
     pdl_wait_then_trigger();
@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
     // read as zero outside the rows of the operator.
     auto load = [&](int k, int r) -> V4 {
         const int rr = max(0, min(n0 - 1, r));
-        V4 v = ldv4(p.in[k] + rr * n1 + col);
+        V4 v = ldv4(at_off<O32>(p.in[k], rr * n1 + col));
         if (BWD && k >= 2) {
             v = v4mul(v, p.gs[k - 2]);
             if (r < 1 || r > n0 - 2) v = v4zero();
@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
     auto prefetch_row = [&](int r) {                 // one lane per 128-byte line
         if ((threadIdx.x & 7) == 0 && cvalid && r < n0) {
 #pragma unroll
-            for (int k = 0; k < NA; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.in[k] + r * n1 + col));
+            for (int k = 0; k < NA; ++k) asm volatile("prefetch.global.L2 [%0];" ::"l"(at_off<O32>(p.in[k], r * n1 + col)));
         }
     };
     if (p.prefetch > 0)
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
         for (int k = 0; k < NA; ++k) {
             nxt[k] = load(k, row + 1);
             E[k] = 0.f;
-            if (efetch) E[k] = __ldg(p.in[k] + row * n1 + eoff);
+            if (efetch) E[k] = __ldg(at_off<O32>(p.in[k], row * n1 + eoff));
         }
 #pragma unroll
         for (int k = 0; k < NA; ++k) {
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(128) ns2d_kernel(const Ns2dParams p) {
         if (cvalid) {
 #pragma unroll
             for (int e = 0; e < 3; ++e) {
-                stv4(p.out[e] + row * n1 + col, o[e][0], o[e][1]);
+                stv4(at_off<O32>(p.out[e], row * n1 + col), o[e][0], o[e][1]);
                 if (!BWD) acc[e] = fma2(o[e][0], o[e][0], fma2(o[e][1], o[e][1], acc[e]));
             }
         }
@@ -217,6 +217,12 @@ static void ns2d_geometry(const int* n, Ns2dParams& p, int& block) {
     if (p.prefetch < 0) p.prefetch = 0;
 }
 
+// 32-bit byte offsets are enough for arrays of at most 2^30 floats
+static bool ns2d_off32(const Problem& q) {
+    const char* s = std::getenv("FPDE_NS2D_OFF32");
+    return !(s && s[0] == '0') && (int64_t)q.n[0] * q.n[1] <= ((int64_t)1 << 30);
+}
+
 int ns2d_items(const int* n) {
     Ns2dParams p{}; int block;
     ns2d_geometry(n, p, block);
@@ -234,6 +240,7 @@ cudaError_t launch_ns2d_fwd(const Problem& q) {
     ns2d_consts(q, p);
     for (int k = 0; k < 3; ++k) { p.in[k] = q.in[k]; p.out[k] = q.out[k]; }
     p.partials = q.partials;
+    if (ns2d_off32(q)) return launch_kernel(ns2d_kernel<false, true>, dim3(p.nitems), dim3(block), q.stream, p);
     return launch_kernel(ns2d_kernel<false>, dim3(p.nitems), dim3(block), q.stream, p);
 }
 
@@ -244,6 +251,7 @@ cudaError_t launch_ns2d_bwd(const Problem& q) {
     p.in[0] = q.in[0]; p.in[1] = q.in[1];
     for (int k = 0; k < 3; ++k) { p.in[2 + k] = q.aux[k]; p.out[k] = q.out[k]; p.gs[k] = sp(q.gscale[k]); }
     p.partials = nullptr;
+    if (ns2d_off32(q)) return launch_kernel(ns2d_kernel<true, true>, dim3(p.nitems), dim3(block), q.stream, p);
     return launch_kernel(ns2d_kernel<true>, dim3(p.nitems), dim3(block), q.stream, p);
 }
 
