@@ -92,7 +92,7 @@ struct GrayScottBwd {
 
 // PX / PY: the row axis (x) / the column axis (y) is periodic.  Poisson: neither; Gray-Scott:
 // both; the slab form of Gray-Scott (x not periodic: rows at x-index 1..n0-2): PY only.
-template <class F, bool PX, bool PY, int U>
+template <class F, bool PX, bool PY, int U, bool O32 = false>
 __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
     constexpr int NH = F::NH, NC = F::NC, NO = F::NO;
     constexpr int NCA = NC > 0 ? NC : 1;
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
     auto load_h = [&](int k, int r) -> V4 {
         const int rr = in_row(r);
         if (ROWS_MASK_IN && rr < 0) return v4zero();
-        V4 v = ldv4(p.hin[k] + rr * n1 + col);
+        V4 v = BWD ? ldv4(p.hin[k] + rr * n1 + col) : ldv4(at_off<O32>(p.hin[k], rr * n1 + col));
         if (BWD) v = v4mul(v, p.hscale[k]);
         if (COLS_MASK_IN) {
             if (first_col) v.lo.x = 0.f;
@@ -159,13 +159,18 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
                 const int rr = in_row(row);
                 le[u][k] = 0.f; re[u][k] = 0.f;
                 if (!(ROWS_MASK_IN && rr < 0)) {
-                    const float* rp = p.hin[k] + rr * n1;
-                    if (lfetch) le[u][k] = __ldg(rp + lcol);
-                    if (rfetch) re[u][k] = __ldg(rp + rcol);
+                    if (BWD) {                    // (two forms of the same address: each direction keeps the one its build is faster with)
+                        const float* rp = p.hin[k] + rr * n1;
+                        if (lfetch) le[u][k] = __ldg(rp + lcol);
+                        if (rfetch) re[u][k] = __ldg(rp + rcol);
+                    } else {
+                        if (lfetch) le[u][k] = __ldg(at_off<O32>(p.hin[k], rr * n1 + lcol));
+                        if (rfetch) re[u][k] = __ldg(at_off<O32>(p.hin[k], rr * n1 + rcol));
+                    }
                 }
             }
 #pragma unroll
-            for (int k = 0; k < NC; ++k) cen[u][k] = ldv4(p.cin[k] + row * n1 + col);
+            for (int k = 0; k < NC; ++k) cen[u][k] = BWD ? ldv4(p.cin[k] + row * n1 + col) : ldv4(at_off<O32>(p.cin[k], row * n1 + col));
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -207,7 +212,8 @@ __global__ void __launch_bounds__(128) lap2d_kernel(const Lap2dParams p) {
                 if (cvalid) {
 #pragma unroll
                     for (int e = 0; e < NO; ++e) {
-                        stv4(p.out[e] + row * n1 + col, o_lo[e], o_hi[e]);
+                        if (BWD) stv4(p.out[e] + row * n1 + col, o_lo[e], o_hi[e]);
+                        else stv4(at_off<O32>(p.out[e], row * n1 + col), o_lo[e], o_hi[e]);
                         if (!BWD) acc[e] = fma2(o_lo[e], o_lo[e], fma2(o_hi[e], o_hi[e], acc[e]));
                     }
                 }
@@ -252,6 +258,10 @@ int lap2d_items(const int* n) {
 
 template <class F, bool PX, bool PY>
 static cudaError_t launch(const Lap2dParams& p, int block, cudaStream_t s) {
+    // 32-bit byte offsets from the array bases for arrays of at most 2^30 floats
+    const char* o = std::getenv("FPDE_LAP2D_OFF32");
+    if (!(o && o[0] == '0') && (int64_t)p.n0 * p.n1 <= ((int64_t)1 << 30))
+        return launch_kernel(lap2d_kernel<F, PX, PY, 4, true>, dim3(p.nitems), dim3(block), s, p);
     return launch_kernel(lap2d_kernel<F, PX, PY, 4>, dim3(p.nitems), dim3(block), s, p);
 }
 
