@@ -60,18 +60,18 @@ KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
 # summarised under profiles/; None where no capture has been taken yet.
 NCU_TRAFFIC_BYTES = {
     # half-size capture (64 planes) x 2: traffic is proportional to the number of planes
-    ("ns_tgv_128x16", "ns_fwd_kernel"): 2 * 518857216,
-    ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 762315264,
-    ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 223546880,
-    ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 366772224,
+    ("ns_tgv_128x16", "ns_fwd_kernel"): 2 * 518306560,
+    ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 761274112,
+    ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 222671616,
+    ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 366043648,
     ("helmholtz_256", "star3d_kernel<fwd>"): 185158400,
     ("helmholtz_256", "star3d_kernel<bwd>"): 101107200,
-    ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 360634368,
-    ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 508413184,
-    ("ns3d_steady_256", "ns3d_kernel<fwd>"): 515948032,
-    ("ns3d_steady_256", "ns3d_kernel<bwd>"): 734166272,
-    ("grayscott_4096", "fused2d_kernel<grayscott_2d>"): 234967552,
-    ("ns2d_steady_4096", "fused2d_kernel<ns_2d_steady>"): 373059840,
+    ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 362135040,
+    ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 511582720,
+    ("ns3d_steady_256", "ns3d_kernel<fwd>"): 516580096,
+    ("ns3d_steady_256", "ns3d_kernel<bwd>"): 734623232,
+    ("grayscott_4096", "fused2d_kernel<grayscott_2d>"): 235297280,
+    ("ns2d_steady_4096", "fused2d_kernel<ns_2d_steady>"): 372255488,
 }
 FALLBACK_HBM_GBS = 6650.0
 LAUNCHES_PER_STEP = 3               # forward kernel, loss finalise, adjoint kernel
