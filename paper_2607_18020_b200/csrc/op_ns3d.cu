@@ -145,7 +145,8 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
 }
 
 // O32: 32-bit byte offsets from the array bases (arrays of at most 2^30 floats); used where the
-// build comes out without spills (forward, and the adjoint without zero-extension)
+// build comes out without spills (forward, the adjoint without zero-extension, and the interior
+// steps of the masking adjoint: with its shell steps as well that kernel spills)
 template <bool BWD, int MINB, bool PRE = false, bool O32 = false>
 __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     constexpr int NA = BWD ? 7 : 4;
@@ -200,7 +201,7 @@ __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
 
     auto step = [&](int a, const V4 (&W0)[NA], const V4 (&W1)[NA], V4 (&W2)[NA]) {
-        if (!PRE && (y_edge_block || a <= 1 || a >= p.n0 - 2)) ns3d_step<BWD, true, NA, PRE, O32>(p, t, a, W0, W1, W2, acc);
+        if (!PRE && (y_edge_block || a <= 1 || a >= p.n0 - 2)) ns3d_step<BWD, true, NA, PRE, O32 && !BWD>(p, t, a, W0, W1, W2, acc);
         else ns3d_step<BWD, false, NA, PRE, O32>(p, t, a, W0, W1, W2, acc);
     };
     for (int a = a0; a < a1; a += 3) {
@@ -283,6 +284,7 @@ cudaError_t launch_ns3d_bwd(const Problem& q) {
         return launch_kernel(ns3d_kernel<true, 2, true>, dim3(p.nitems), block, q.stream, p);
     }
     if (env_int("FPDE_NS3D_MINB_B", 2) == 3) return launch_kernel(ns3d_kernel<true, 3>, dim3(p.nitems), block, q.stream, p);
+    if (ns3d_off32(q)) return launch_kernel(ns3d_kernel<true, 2, false, true>, dim3(p.nitems), block, q.stream, p);
     return launch_kernel(ns3d_kernel<true, 2>, dim3(p.nitems), block, q.stream, p);
 }
 
