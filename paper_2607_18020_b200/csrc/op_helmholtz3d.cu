@@ -19,6 +19,7 @@
 
 #include <algorithm>
 #include <cstdlib>
+#include <type_traits>
 
 namespace fpde {
 
@@ -35,7 +36,7 @@ struct Star3dParams {
     int prefetch;
 };
 
-__device__ __forceinline__ void prefetch_l2_line(const float* ptr) {
+__device__ __forceinline__ void prefetch_l2_line(const void* ptr) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
 }
 
@@ -46,9 +47,12 @@ __device__ __forceinline__ void prefetch_l2_line(const float* ptr) {
 // adjoint of an upstream array that is already zero off the rows (the residual array the forward
 // kernel of the same call wrote): the star itself, nothing to mask; clamped reads beyond the
 // array land in the zero band.
-template <int MODE, bool EDGE, int MINB>
+template <int MODE, bool EDGE, int MINB, bool O32>
 __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int mb, int ab) {
     constexpr bool FWD = MODE == 0;
+    // Byte offsets from the array base: 32-bit (the access is then base + zero-extended register,
+    // no 64-bit arithmetic per load) when every array is below 4 GiB, 64-bit otherwise.
+    using Off = typename std::conditional<O32, unsigned, size_t>::type;
     const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
     const int c4 = cb * blockDim.x + threadIdx.x;
     const int m = mb * blockDim.y + threadIdx.y;
@@ -59,63 +63,70 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     const bool first_col = c4 == 0, last_col = c4 == nc4 - 1;
     const int a0 = ab * p.planes_per_item;
     const int a1 = min(a0 + p.planes_per_item, n0);
-    const int PS = n1 * n2;
+    const Off PS4 = (Off)4 * (Off)n1 * (Off)n2;     // bytes per plane
     constexpr bool MASK_IN = MODE == 1;             // the adjoint zero-extends its input outside the rows
     constexpr bool ROWMASK = MASK_IN && EDGE;
-    const float* __restrict__ hin = p.hin;
+    const char* __restrict__ hin = reinterpret_cast<const char*>(p.hin);
+    const char* __restrict__ cin = reinterpret_cast<const char*>(p.cin);
+    char* __restrict__ out = reinterpret_cast<char*>(p.out);
 
-    // element offsets of the own row and of the four y neighbours (clamped into the grid: out of
-    // range rows only feed outputs that are masked, or are discarded by the selects below)
-    auto yoff = [&](int d) -> int { return max(0, min(n1 - 1, mc + d)) * n2 + col; };
-    auto yptr = [&](int d) -> const float* { return hin + yoff(d); };
+    // byte offsets of the own row and of the four y neighbours within a plane (clamped into the
+    // grid: out of range rows only feed outputs that are masked, or are discarded by the selects
+    // below); the neighbours as differences to the own row, constant over the march
+    auto yoff = [&](int d) -> int { return (EDGE ? max(0, min(n1 - 1, mc + d)) : mc + d) * n2 + col; };
     auto ydead = [&](int d) -> bool { const int r = mc + d; return ROWMASK && (r < 2 || r > n1 - 3); };
-    // one pointer per row: the plane offset of a step is then a single multiply-add per load
     const int o_c = yoff(0);
-    const float* __restrict__ p_c = yptr(0);
-    const float* __restrict__ p_m1 = yptr(-1);
-    const float* __restrict__ p_p1 = yptr(1);
-    const float* __restrict__ p_m2 = yptr(-2);
-    const float* __restrict__ p_p2 = yptr(2);
-    const bool d0 = ydead(0), dm1 = ydead(-1), dp1 = ydead(1), dm2 = ydead(-2), dp2 = ydead(2);
-    // Load from a row pointer at plane offset `pl` (already clamped); `dead` = reads as zero.
+    auto ydelta = [&](int d) -> Off { return (Off)(4 * (yoff(d) - o_c)); };   // wraps for d < 0: added modulo 2^32 / 2^64
+    const Off dm1 = ydelta(-1), dp1 = ydelta(1), dm2 = ydelta(-2), dp2 = ydelta(2);
+    const bool d0 = ydead(0), dm1d = ydead(-1), dp1d = ydead(1), dm2d = ydead(-2), dp2d = ydead(2);
+    auto ld_at = [&](const char* base, Off off) -> V4 {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(base + off));
+        V4 v; v.lo = make_float2(t.x, t.y); v.hi = make_float2(t.z, t.w);
+        return v;
+    };
+    // Load of the upstream / field array at a byte offset; `dead` = reads as zero.
     // OWN: the thread's own column (the x window).  Only that one is masked in the first / last
     // float4 of a row (the band in z); the y neighbours are not, their contribution to the two
     // band columns is removed after the sums instead (see the step).
-    auto load_h = [&](const float* rp, int pl, bool dead, bool own) -> V4 {
-        V4 v = ldv4(rp + pl);
+    auto load_h = [&](Off off, bool dead, bool own) -> V4 {
+        V4 v = ld_at(hin, off);
         if (MASK_IN) {
             if ((ROWMASK && dead) || (own && first_col)) v.lo = make_float2(0.f, 0.f);
             if ((ROWMASK && dead) || (own && last_col)) v.hi = make_float2(0.f, 0.f);
         }
         return v;
     };
-    auto pclamp = [&](int a) -> int { return EDGE ? max(0, min(n0 - 1, a)) * PS : a * PS; };
+    // own-column offset of plane a (clamped in the blocks that touch the ends of the x axis)
+    auto poff = [&](int a) -> Off { return (Off)(EDGE ? max(0, min(n0 - 1, a)) : a) * PS4 + (Off)(4 * o_c); };
     auto pdead = [&](int a) -> bool { return ROWMASK && (a < 2 || a > n0 - 3); };
     // The two floats beyond the float4 that the first / last lane of a warp cannot get by shuffle:
     // one predicated 8-byte load, issued with the other loads of the step (a load inside a
     // divergent branch would be waited for on its own).  At the ends of a z line it stays 0.
     const bool efetch = (lane == 0 && c4 > 0 && c4 < nc4) || (lane == 31 && c4 < nc4 - 1);
-    const int eoff = lane == 0 ? -2 : 4;
+    const Off eoff = lane == 0 ? (Off)(-8) : (Off)16;
+    const bool pf_lane = p.prefetch > 0 && (threadIdx.x & 7) == 0;
+    const int pf_last = min(a1 + 1, n0 - 1) - 2 - p.prefetch;      // last step that still prefetches
+    const Off pf_h = (Off)(2 + p.prefetch) * PS4, pf_c = (Off)p.prefetch * PS4;
 
-    V4 Q0 = load_h(p_c, pclamp(a0 - 2), d0 || pdead(a0 - 2), true), Q1 = load_h(p_c, pclamp(a0 - 1), d0 || pdead(a0 - 1), true);
-    V4 Q2 = load_h(p_c, pclamp(a0), d0 || pdead(a0), true), Q3 = load_h(p_c, pclamp(a0 + 1), d0 || pdead(a0 + 1), true), Q4;
+    V4 Q0 = load_h(poff(a0 - 2), d0 || pdead(a0 - 2), true), Q1 = load_h(poff(a0 - 1), d0 || pdead(a0 - 1), true);
+    V4 Q2 = load_h(poff(a0), d0 || pdead(a0), true), Q3 = load_h(poff(a0 + 1), d0 || pdead(a0 + 1), true), Q4;
+    Off off = poff(a0);                              // own float4 on the current plane
     float2 acc = make_float2(0.f, 0.f);
 
     // one x step: q0..q3 = planes a-2..a+1, q4 receives plane a+2
     auto step = [&](int a, const V4& q0, const V4& q1, const V4& q2, const V4& q3, V4& q4) {
-        const int pl = a * PS;
-        if (p.prefetch > 0 && (threadIdx.x & 7) == 0 && a + 2 + p.prefetch <= a1 + 1 && a + 2 + p.prefetch < n0) {
-            prefetch_l2_line(p_c + pl + (2 + p.prefetch) * PS);
-            if (FWD) prefetch_l2_line(p.cin + pl + p.prefetch * PS + o_c);
+        if (pf_lane && a <= pf_last) {
+            prefetch_l2_line(hin + (off + pf_h));
+            if (FWD) prefetch_l2_line(cin + (off + pf_c));
         }
         const bool pd = pdead(a);
-        q4 = load_h(p_c, pclamp(a + 2), d0 || pdead(a + 2), true);
-        const V4 a1v = load_h(p_m1, pl, dm1 || pd, false), b1v = load_h(p_p1, pl, dp1 || pd, false);
-        const V4 a2v = load_h(p_m2, pl, dm2 || pd, false), b2v = load_h(p_p2, pl, dp2 || pd, false);
+        q4 = load_h(EDGE ? poff(a + 2) : off + 2 * PS4, d0 || pdead(a + 2), true);
+        const V4 a1v = load_h(off + dm1, dm1d || pd, false), b1v = load_h(off + dp1, dp1d || pd, false);
+        const V4 a2v = load_h(off + dm2, dm2d || pd, false), b2v = load_h(off + dp2, dp2d || pd, false);
         V4 src = v4zero();
-        if (FWD) src = ldv4(p.cin + pl + o_c);
+        if (FWD) src = ld_at(cin, off);
         float2 E = make_float2(0.f, 0.f);
-        if (efetch) E = __ldg(reinterpret_cast<const float2*>(p_c + pl + eoff));
+        if (efetch) E = __ldg(reinterpret_cast<const float2*>(hin + (off + eoff)));
         if (ROWMASK && (d0 || pd)) E = make_float2(0.f, 0.f);
         // z neighbours from the adjacent lanes; the outer lanes of a warp take the fetched pair
         float l1 = __shfl_up_sync(FULL_MASK, q2.hi.y, 1), l2 = __shfl_up_sync(FULL_MASK, q2.hi.x, 1);
@@ -150,9 +161,10 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
             if (last_col) o.hi = make_float2(0.f, 0.f);
         }
         if (valid) {
-            stv4(p.out + pl + o_c, o.lo, o.hi);
+            *reinterpret_cast<float4*>(out + off) = make_float4(o.lo.x, o.lo.y, o.hi.x, o.hi.y);
             if (FWD) acc = fma2(o.lo, o.lo, fma2(o.hi, o.hi, acc));
         }
+        off += PS4;
     };
 
     for (int a = a0; a < a1; a += 5) {
@@ -168,7 +180,7 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     }
 }
 
-template <int MODE, int MINB>
+template <int MODE, int MINB, bool O32>
 __global__ void __launch_bounds__(256, MINB) star3d_kernel(const Star3dParams p) {
     pdl_wait_then_trigger();
     int item = blockIdx.x;
@@ -178,8 +190,8 @@ __global__ void __launch_bounds__(256, MINB) star3d_kernel(const Star3dParams p)
     const int m0 = mb * blockDim.y, a0 = ab * p.planes_per_item;
     // away from the band: every row m0-2 .. m0+TY+1 and plane a0-2 .. a1+1 is a row of the operator
     const bool interior = m0 >= 4 && m0 + (int)blockDim.y + 4 <= p.n1 && a0 >= 4 && a0 + p.planes_per_item + 4 <= p.n0;
-    if (interior) star3d_body<MODE, false, MINB>(p, cb, mb, ab);
-    else star3d_body<MODE, true, MINB>(p, cb, mb, ab);
+    if (interior) star3d_body<MODE, false, MINB, O32>(p, cb, mb, ab);
+    else star3d_body<MODE, true, MINB, O32>(p, cb, mb, ab);
 }
 
 static int env_int(const char* name, int dflt) {
@@ -224,13 +236,30 @@ int star3d_items(const int* n) {
     return p.nitems;
 }
 
+// 32-bit byte offsets when every array is below 4 GiB (FPDE_STAR3D_OFF32=0 forces the 64-bit form)
+static bool star3d_off32(const Problem& q) {
+    const char* e = std::getenv("FPDE_STAR3D_OFF32");
+    if (e && *e == '0') return false;
+    return (long long)q.n[0] * q.n[1] * q.n[2] <= (1ll << 30);
+}
+
+template <int MODE>
+static cudaError_t star3d_launch(const Problem& q, const Star3dParams& p, dim3 block) {
+    const bool m4 = env_int("FPDE_STAR3D_MINB", 4) >= 4;
+    if (star3d_off32(q)) {
+        if (m4) return launch_kernel(star3d_kernel<MODE, 4, true>, dim3(p.nitems), block, q.stream, p);
+        return launch_kernel(star3d_kernel<MODE, 3, true>, dim3(p.nitems), block, q.stream, p);
+    }
+    if (m4) return launch_kernel(star3d_kernel<MODE, 4, false>, dim3(p.nitems), block, q.stream, p);
+    return launch_kernel(star3d_kernel<MODE, 3, false>, dim3(p.nitems), block, q.stream, p);
+}
+
 cudaError_t launch_helmholtz_fwd(const Problem& q) {
     Star3dParams p{}; dim3 block;
     star3d_geometry(q, p, block, 1.0, true);
     p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0];
     p.partials = q.partials;
-    if (env_int("FPDE_STAR3D_MINB", 4) >= 4) return launch_kernel(star3d_kernel<0, 4>, dim3(p.nitems), block, q.stream, p);
-    return launch_kernel(star3d_kernel<0, 3>, dim3(p.nitems), block, q.stream, p);
+    return star3d_launch<0>(q, p, block);
 }
 
 cudaError_t launch_helmholtz_bwd(const Problem& q) {
@@ -238,13 +267,7 @@ cudaError_t launch_helmholtz_bwd(const Problem& q) {
     star3d_geometry(q, p, block, q.gscale[0], false);      // the operator is linear: the scale goes into the weights
     p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0];
     p.partials = nullptr;
-    const bool m4 = env_int("FPDE_STAR3D_MINB", 4) >= 4;
-    if (q.gres_zero_off_rows) {
-        if (m4) return launch_kernel(star3d_kernel<2, 4>, dim3(p.nitems), block, q.stream, p);
-        return launch_kernel(star3d_kernel<2, 3>, dim3(p.nitems), block, q.stream, p);
-    }
-    if (m4) return launch_kernel(star3d_kernel<1, 4>, dim3(p.nitems), block, q.stream, p);
-    return launch_kernel(star3d_kernel<1, 3>, dim3(p.nitems), block, q.stream, p);
+    return q.gres_zero_off_rows ? star3d_launch<2>(q, p, block) : star3d_launch<1>(q, p, block);
 }
 
 }  // namespace fpde
