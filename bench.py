@@ -395,6 +395,21 @@ def single_pass_figures(torch, prob, steps, warmup, flush, peak):
             "what": "fpde_fwd_bwd, residual arrays not stored; launches: 1 kernel + loss finalise"}
 
 
+class CleanFlush:
+    """An L2 flush that leaves the cache clean: the 256 MiB write, then a read of another 256 MiB.
+    After the write alone the whole L2 holds dirty lines, and the first kernel that follows pays
+    for writing them back (about 126 MB of DRAM traffic that is not its own)."""
+
+    def __init__(self, torch, write_buf):
+        self.w = write_buf
+        self.r = torch.zeros(64 << 20, dtype=torch.float32, device="cuda")
+        self.acc = torch.zeros((), dtype=torch.float32, device="cuda")
+
+    def fill_(self, k):
+        self.w.fill_(k)
+        self.acc += self.r.sum()
+
+
 def config_line(torch, B, name, steps, warmup, peak):
     """Secondary figures for one configuration: per-call medians with an L2 flush (a 256 MiB
     write) before every step, so small grids are measured cold like large ones."""
@@ -411,6 +426,14 @@ def config_line(torch, B, name, steps, warmup, peak):
            "gbs_pair": (fb + bb) * N / ((fm + bm) * 1e-3) / 1e9}
     out["frac_pair"] = out["gbs_pair"] / peak
     out["timing"] = "cold: 256 MiB L2 flush before every step, per-call medians"
+    # the same with the cache left clean (write, then read another buffer): what the kernels do when
+    # they do not also have to write back the flush's dirty lines
+    clean = CleanFlush(torch, flush)
+    _, f_ms, b_ms = timed_steps(torch, prob, steps, warmup, lambda: None, flush=clean, inner_events=True)
+    fc, bc = statistics.median(f_ms), statistics.median(b_ms)
+    out["clean_l2"] = {"ms_fwd": fc, "ms_bwd": bc, "frac_pair": (fb + bb) * N / ((fc + bc) * 1e-3) / 1e9 / peak,
+                       "what": "flush = 256 MiB write followed by a 256 MiB read (no dirty lines left in L2)"}
+    del clean
     # warm, back to back (working sets below L2 stay resident: say so), and the same pairs replayed
     # from one CUDA graph, which removes the host launch gaps of the latency-bound small grids
     total_ms, _, _ = timed_steps(torch, prob, steps, 3, lambda: None)

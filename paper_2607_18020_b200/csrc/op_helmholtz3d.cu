@@ -19,6 +19,7 @@
 
 #include <algorithm>
 #include <cstdlib>
+#include <cstddef>
 #include <type_traits>
 
 namespace fpde {
@@ -47,11 +48,15 @@ __device__ __forceinline__ void prefetch_l2_line(const void* ptr) {
 // adjoint of an upstream array that is already zero off the rows (the residual array the forward
 // kernel of the same call wrote): the star itself, nothing to mask; clamped reads beyond the
 // array land in the zero band.
+// Addressing: a position is a byte offset from the array bases (the three arrays are reached from
+// the same offset), 32-bit (O32) when every array is below 4 GiB; the y neighbours sit at
+// per-thread distances from it that are constant over the march.  (Builds with the y and z
+// extents fixed at compile time, where those distances become constants of the load
+// instructions, execute a tenth fewer instructions and run no faster: the kernels wait on
+// memory, not on issue slots.)
 template <int MODE, bool EDGE, int MINB, bool O32>
 __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int mb, int ab) {
     constexpr bool FWD = MODE == 0;
-    // Byte offsets from the array base: 32-bit (the access is then base + zero-extended register,
-    // no 64-bit arithmetic per load) when every array is below 4 GiB, 64-bit otherwise.
     using Off = typename std::conditional<O32, unsigned, size_t>::type;
     const int n0 = p.n0, n1 = p.n1, n2 = p.n2, nc4 = p.nc4;
     const int c4 = cb * blockDim.x + threadIdx.x;
@@ -69,35 +74,41 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     const char* __restrict__ hin = reinterpret_cast<const char*>(p.hin);
     const char* __restrict__ cin = reinterpret_cast<const char*>(p.cin);
     char* __restrict__ out = reinterpret_cast<char*>(p.out);
+    using Pos = Off;
+    auto h_at = [&](Pos pos, Off d) -> const char* { return hin + (Off)(pos + d); };
+    auto c_at = [&](Pos pos, Off d) -> const char* { return cin + (Off)(pos + d); };
+    auto o_at = [&](Pos pos) -> char* { return out + pos; };
 
-    // byte offsets of the own row and of the four y neighbours within a plane (clamped into the
+    // element offsets of the own row and of the four y neighbours within a plane (clamped into the
     // grid: out of range rows only feed outputs that are masked, or are discarded by the selects
-    // below); the neighbours as differences to the own row, constant over the march
+    // below); the neighbours as distances from the own row, constant over the march
     auto yoff = [&](int d) -> int { return (EDGE ? max(0, min(n1 - 1, mc + d)) : mc + d) * n2 + col; };
     auto ydead = [&](int d) -> bool { const int r = mc + d; return ROWMASK && (r < 2 || r > n1 - 3); };
     const int o_c = yoff(0);
-    auto ydelta = [&](int d) -> Off { return (Off)(4 * (yoff(d) - o_c)); };   // wraps for d < 0: added modulo 2^32 / 2^64
+    auto ydelta = [&](int d) -> Off { return (Off)(4 * (yoff(d) - o_c)); };   // d < 0: added modulo 2^32 / 2^64
     const Off dm1 = ydelta(-1), dp1 = ydelta(1), dm2 = ydelta(-2), dp2 = ydelta(2);
     const bool d0 = ydead(0), dm1d = ydead(-1), dp1d = ydead(1), dm2d = ydead(-2), dp2d = ydead(2);
-    auto ld_at = [&](const char* base, Off off) -> V4 {
-        const float4 t = __ldg(reinterpret_cast<const float4*>(base + off));
+    auto ld_at = [&](const char* ptr) -> V4 {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(ptr));
         V4 v; v.lo = make_float2(t.x, t.y); v.hi = make_float2(t.z, t.w);
         return v;
     };
-    // Load of the upstream / field array at a byte offset; `dead` = reads as zero.
+    // Load of the upstream / field array; `dead` = reads as zero.
     // OWN: the thread's own column (the x window).  Only that one is masked in the first / last
     // float4 of a row (the band in z); the y neighbours are not, their contribution to the two
     // band columns is removed after the sums instead (see the step).
-    auto load_h = [&](Off off, bool dead, bool own) -> V4 {
-        V4 v = ld_at(hin, off);
+    auto load_h = [&](const char* ptr, bool dead, bool own) -> V4 {
+        V4 v = ld_at(ptr);
         if (MASK_IN) {
             if ((ROWMASK && dead) || (own && first_col)) v.lo = make_float2(0.f, 0.f);
             if ((ROWMASK && dead) || (own && last_col)) v.hi = make_float2(0.f, 0.f);
         }
         return v;
     };
-    // own-column offset of plane a (clamped in the blocks that touch the ends of the x axis)
-    auto poff = [&](int a) -> Off { return (Off)(EDGE ? max(0, min(n0 - 1, a)) : a) * PS4 + (Off)(4 * o_c); };
+    // own column on plane a (clamped in the blocks that touch the ends of the x axis)
+    auto ppos = [&](int a) -> Pos {
+        return (Off)(EDGE ? max(0, min(n0 - 1, a)) : a) * PS4 + (Off)(4 * o_c);
+    };
     auto pdead = [&](int a) -> bool { return ROWMASK && (a < 2 || a > n0 - 3); };
     // The two floats beyond the float4 that the first / last lane of a warp cannot get by shuffle:
     // one predicated 8-byte load, issued with the other loads of the step (a load inside a
@@ -108,25 +119,25 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
     const int pf_last = min(a1 + 1, n0 - 1) - 2 - p.prefetch;      // last step that still prefetches
     const Off pf_h = (Off)(2 + p.prefetch) * PS4, pf_c = (Off)p.prefetch * PS4;
 
-    V4 Q0 = load_h(poff(a0 - 2), d0 || pdead(a0 - 2), true), Q1 = load_h(poff(a0 - 1), d0 || pdead(a0 - 1), true);
-    V4 Q2 = load_h(poff(a0), d0 || pdead(a0), true), Q3 = load_h(poff(a0 + 1), d0 || pdead(a0 + 1), true), Q4;
-    Off off = poff(a0);                              // own float4 on the current plane
+    V4 Q0 = load_h(h_at(ppos(a0 - 2), 0), d0 || pdead(a0 - 2), true), Q1 = load_h(h_at(ppos(a0 - 1), 0), d0 || pdead(a0 - 1), true);
+    V4 Q2 = load_h(h_at(ppos(a0), 0), d0 || pdead(a0), true), Q3 = load_h(h_at(ppos(a0 + 1), 0), d0 || pdead(a0 + 1), true), Q4;
+    Pos pos = ppos(a0);                              // own float4 on the current plane
     float2 acc = make_float2(0.f, 0.f);
 
     // one x step: q0..q3 = planes a-2..a+1, q4 receives plane a+2
     auto step = [&](int a, const V4& q0, const V4& q1, const V4& q2, const V4& q3, V4& q4) {
         if (pf_lane && a <= pf_last) {
-            prefetch_l2_line(hin + (off + pf_h));
-            if (FWD) prefetch_l2_line(cin + (off + pf_c));
+            prefetch_l2_line(h_at(pos, pf_h));
+            if (FWD) prefetch_l2_line(c_at(pos, pf_c));
         }
         const bool pd = pdead(a);
-        q4 = load_h(EDGE ? poff(a + 2) : off + 2 * PS4, d0 || pdead(a + 2), true);
-        const V4 a1v = load_h(off + dm1, dm1d || pd, false), b1v = load_h(off + dp1, dp1d || pd, false);
-        const V4 a2v = load_h(off + dm2, dm2d || pd, false), b2v = load_h(off + dp2, dp2d || pd, false);
+        q4 = load_h(EDGE ? h_at(ppos(a + 2), 0) : h_at(pos, 2 * PS4), d0 || pdead(a + 2), true);
+        const V4 a1v = load_h(h_at(pos, dm1), dm1d || pd, false), b1v = load_h(h_at(pos, dp1), dp1d || pd, false);
+        const V4 a2v = load_h(h_at(pos, dm2), dm2d || pd, false), b2v = load_h(h_at(pos, dp2), dp2d || pd, false);
         V4 src = v4zero();
-        if (FWD) src = ld_at(cin, off);
+        if (FWD) src = ld_at(c_at(pos, 0));
         float2 E = make_float2(0.f, 0.f);
-        if (efetch) E = __ldg(reinterpret_cast<const float2*>(hin + (off + eoff)));
+        if (efetch) E = __ldg(reinterpret_cast<const float2*>(h_at(pos, eoff)));
         if (ROWMASK && (d0 || pd)) E = make_float2(0.f, 0.f);
         // z neighbours from the adjacent lanes; the outer lanes of a warp take the fetched pair
         float l1 = __shfl_up_sync(FULL_MASK, q2.hi.y, 1), l2 = __shfl_up_sync(FULL_MASK, q2.hi.x, 1);
@@ -161,10 +172,10 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
             if (last_col) o.hi = make_float2(0.f, 0.f);
         }
         if (valid) {
-            *reinterpret_cast<float4*>(out + off) = make_float4(o.lo.x, o.lo.y, o.hi.x, o.hi.y);
+            *reinterpret_cast<float4*>(o_at(pos)) = make_float4(o.lo.x, o.lo.y, o.hi.x, o.hi.y);
             if (FWD) acc = fma2(o.lo, o.lo, fma2(o.hi, o.hi, acc));
         }
-        off += PS4;
+        pos += PS4;
     };
 
     for (int a = a0; a < a1; a += 5) {
@@ -208,7 +219,7 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     int tx = p.nc4 > 32 ? 64 : 32;
     tx = env_int("FPDE_STAR3D_TX", tx);
     tx = std::max(32, std::min(128, (tx / 32) * 32));
-    int ty = env_int("FPDE_STAR3D_TY", 2);
+    int ty = env_int("FPDE_STAR3D_TY", 4);
     ty = std::max(1, std::min(256 / tx, ty));
     block = dim3(tx, ty, 1);
     // the forward kernel (two input streams) runs best on long items, the adjoint on short ones
@@ -237,21 +248,12 @@ int star3d_items(const int* n) {
 }
 
 // 32-bit byte offsets when every array is below 4 GiB (FPDE_STAR3D_OFF32=0 forces the 64-bit form)
-static bool star3d_off32(const Problem& q) {
-    const char* e = std::getenv("FPDE_STAR3D_OFF32");
-    if (e && *e == '0') return false;
-    return (long long)q.n[0] * q.n[1] * q.n[2] <= (1ll << 30);
-}
-
 template <int MODE>
 static cudaError_t star3d_launch(const Problem& q, const Star3dParams& p, dim3 block) {
-    const bool m4 = env_int("FPDE_STAR3D_MINB", 4) >= 4;
-    if (star3d_off32(q)) {
-        if (m4) return launch_kernel(star3d_kernel<MODE, 4, true>, dim3(p.nitems), block, q.stream, p);
-        return launch_kernel(star3d_kernel<MODE, 3, true>, dim3(p.nitems), block, q.stream, p);
-    }
-    if (m4) return launch_kernel(star3d_kernel<MODE, 4, false>, dim3(p.nitems), block, q.stream, p);
-    return launch_kernel(star3d_kernel<MODE, 3, false>, dim3(p.nitems), block, q.stream, p);
+    const char* e = std::getenv("FPDE_STAR3D_OFF32");
+    const bool o32 = !(e && *e == '0') && (long long)p.n0 * p.n1 * p.n2 <= (1ll << 30);
+    if (o32) return launch_kernel(star3d_kernel<MODE, 4, true>, dim3(p.nitems), block, q.stream, p);
+    return launch_kernel(star3d_kernel<MODE, 4, false>, dim3(p.nitems), block, q.stream, p);
 }
 
 cudaError_t launch_helmholtz_fwd(const Problem& q) {

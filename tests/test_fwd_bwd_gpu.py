@@ -35,6 +35,7 @@ TWO_KERNEL = [
     ("helmholtz_256", (12, 20, 24)),
     ("helmholtz_256", (70, 45, 136)),              # ragged z line: the adjoint runs without zero-extension here
     ("helmholtz_256", (5, 5, 8)),
+    ("helmholtz_256", (41, 128, 128)),             # build with the y and z extents fixed
     ("ns_tgv_128x16", (8, 12, 16, 8)),
     ("ns3d_steady_256", (7, 5, 132)),
     ("ns3d_steady_256", (37, 22, 136)),

@@ -21,6 +21,9 @@ MEDIUM = [
     ("poisson_1024", (203, 300)),          # several row chunks and column blocks, ragged tails
     ("grayscott_4096", (1000, 1032)),
     ("helmholtz_256", (70, 45, 136)),
+    ("helmholtz_256", (45, 128, 128)),      # the builds with the y and z extents fixed at compile time:
+    ("helmholtz_256", (13, 256, 256)),      # interior and band blocks, several plane items in the adjoint
+    ("helmholtz_256", (9, 512, 512)),
     ("ns_tgv_128x16", (36, 21, 20, 16)),
     ("ns2d_steady_4096", (128, 128)),
     ("ns2d_steady_4096", (203, 300)),
