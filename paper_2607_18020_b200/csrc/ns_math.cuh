@@ -38,6 +38,8 @@ struct NsConsts {
     float2 a_t[3];        // [q]     gs_q / (2 dt)
     float2 l_g[3];        // [e]     gs_e
     float2 c_ih[3];       // [a]     gs_c / (2 h_a)
+    float2 nih[3];        // [a]     -1/(2 h_a)
+    float2 nv2c;          //         2 nu sum_a 1/h_a^2
 };
 
 // ---- one packed pair (two consecutive t of one z) of every array -----------------------------
@@ -76,11 +78,13 @@ __device__ __forceinline__ void ns_fwd_pair(const NsConsts& k, const float2 (&w0
 
 // Adjoint: arrays 0..2 = u,v,w ; 3..6 = upstream of mom_x, mom_y, mom_z, continuity;
 // dt[q] = G_q(t-1) - G_q(t+1) for the pair (end planes already counted as zero).  o[f]: g_u, g_v, g_w, g_p.
-// DIRECT: second difference of the upstream array as (gm + gp) - 2c (one instruction less per
-// axis; unlike the fields of the forward pass the upstream arrays are not smooth, nothing cancels)
-// instead of (gm - c) + (gp - c).  Same value up to rounding; each caller takes the form its
-// build is faster with.
-template <bool DIRECT = false>
+// MERGED: transposed advection and diffusion of component q share their neighbours,
+//   sum_a [ G_q(P-a) (c_a(P-a)/(2h_a) - nu/h_a^2) + G_q(P+a) (-c_a(P+a)/(2h_a) - nu/h_a^2) ] + 2 nu sum_a 1/h_a^2 G_q(P),
+// and the six coefficients are the same for the three components: two multiply-adds per
+// neighbour instead of six instructions.  The other form keeps (G(P-a) - G(P)) + (G(P+a) - G(P))
+// and separate products; same value up to rounding (the upstream arrays are not smooth, nothing
+// is gained by differencing first); each caller takes the form its build is faster with.
+template <bool MERGED = false>
 __device__ __forceinline__ void ns_bwd_pair(const NsConsts& k, const float2 (&w0)[7], const float2 (&w1)[7],
                                             const float2 (&w2)[7], const float2 (&ym)[7], const float2 (&yp)[7],
                                             const float2 (&zm)[7], const float2 (&zp)[7], const float2 (&dt)[3],
@@ -98,20 +102,35 @@ __device__ __forceinline__ void ns_bwd_pair(const NsConsts& k, const float2 (&w0
         const float2 cp = NP(a_, a_);
         ncp[a_] = make_float2(-cp.x, -cp.y);
     }
+    float2 am[3], apl[3];                       // MERGED: what G_q(P-a) and G_q(P+a) are multiplied by
+    if (MERGED) {
+#pragma unroll
+        for (int a_ = 0; a_ < 3; ++a_) {
+            am[a_] = fma2(cm[a_], k.ih[a_], k.nv[a_]);
+            apl[a_] = fma2(NP(a_, a_), k.nih[a_], k.nv[a_]);
+        }
+    }
     float2 gp = make_float2(0.f, 0.f);
 #pragma unroll
     for (int q = 0; q < 3; ++q) {
         const float2 c = w1[3 + q];
         float2 r = mul2(dt[q], k.a_t[q]);
+        if (MERGED) {
+            float2 T = mul2(c, k.nv2c);
 #pragma unroll
-        for (int a_ = 0; a_ < 3; ++a_) {
-            const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
-            const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
-            r = fma2(adv, k.a_ih[q][a_], r);
-            if (DIRECT) {
-                r = fma2(fma2(c, splat2(-2.f), add2(gm, gpl)), k.a_nv[q][a_], r);
+            for (int a_ = 0; a_ < 3; ++a_) {
+                const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
+                T = fma2(gm, am[a_], T);
+                T = fma2(gpl, apl[a_], T);
                 if (a_ == q) gp = fma2(sub2(gm, gpl), k.a_ih[q][q], gp);
-            } else {
+            }
+            r = fma2(T, k.l_g[q], r);
+        } else {
+#pragma unroll
+            for (int a_ = 0; a_ < 3; ++a_) {
+                const float2 gm = NM(3 + q, a_), gpl = NP(3 + q, a_);
+                const float2 adv = fma2(gpl, ncp[a_], mul2(gm, cm[a_]));
+                r = fma2(adv, k.a_ih[q][a_], r);
                 const float2 dm = sub2(gm, c), dp = sub2(gpl, c);
                 r = fma2(add2(dm, dp), k.a_nv[q][a_], r);
                 if (a_ == q) gp = fma2(sub2(dm, dp), k.a_ih[q][q], gp);
@@ -193,7 +212,9 @@ inline void ns_fill_consts(NsConsts& k, const double* h, double nu, const double
         k.ih[a] = sp(0.5 / h[a]);
         k.nv[a] = sp(-nu / (h[a] * h[a]));
         k.c_ih[a] = sp(gscale[3] * 0.5 / h[a]);
+        k.nih[a] = sp(-0.5 / h[a]);
     }
+    k.nv2c = sp(2.0 * nu * (1.0 / (h[0] * h[0]) + 1.0 / (h[1] * h[1]) + 1.0 / (h[2] * h[2])));
     k.iht = sp(0.5 / h[3]);
     for (int q = 0; q < 3; ++q) {
         k.a_t[q] = sp(gscale[q] * 0.5 / h[3]);

@@ -121,7 +121,7 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
         float2 w0[NA], w1[NA], w2[NA], ym[NA], yp[NA], zm[NA], zp[NA], oo[4];
         v4_half<NA>(W0, h, w0); v4_half<NA>(W1, h, w1); v4_half<NA>(W2, h, w2);
         v4_half<NA>(Ym, h, ym); v4_half<NA>(Yp, h, yp); v4_half<NA>(Zm, h, zm); v4_half<NA>(Zp, h, zp);
-        if constexpr (BWD) ns_bwd_pair(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
+        if constexpr (BWD) ns_bwd_pair<true>(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
         else ns_fwd_pair(p.k, w0, w1, w2, ym, yp, zm, zp, nodt, oo);
 #pragma unroll
         for (int e = 0; e < 4; ++e) o[e][h] = oo[e];
