@@ -479,11 +479,14 @@ int fpde_bwd_f64(int op, const double* const* fields, const double* const* gres,
 static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 
 // scratch the host-buffer call needs: the loss partial sums of whichever launch shape it uses
+// planes per work item of the pipelined host path's launches (the workspace is sized for it)
+static constexpr int HOST_PIPE_ITEM_PLANES = 4;
+
 static size_t host_workspace_bytes(int op, int ndim, const int64_t* shape) {
     size_t need = fpde_fwd_bwd_workspace_bytes(op, ndim, shape);
     int n[MAX_D] = {0, 0, 0, 0};
     if (op == FPDE_OP_NS_3D_T && check_shape(op, ndim, shape, n, nullptr, nullptr) == FPDE_OK)
-        need = std::max(need, round256((size_t)ns_items(n, false, 4) * REGISTRY[op].ne * sizeof(float)) + 4096);
+        need = std::max(need, round256((size_t)ns_items(n, false, HOST_PIPE_ITEM_PLANES) * REGISTRY[op].ne * sizeof(float)) + 4096);
     return need;
 }
 
@@ -501,22 +504,34 @@ size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape) {
 //
 // The plain form queues H2D(all fields) -> kernels -> D2H(all gradients) on one stream, so the two
 // copy directions never overlap and the step costs T_in + T_out.  Here the grid is cut into K
-// chunks of x-planes: the fields of a chunk go up on a copy stream, the forward kernel of chunk c
-// runs (on the caller's stream) as soon as chunks c-1, c, c+1 have arrived, the adjoint of chunk c
-// as soon as the residuals of c-1, c, c+1 exist, and its gradients go down on a second copy
-// stream while later chunks are still coming up.  Kernels are the ordinary ones launched over a
-// range of plane chunks (they read their x neighbours from the full arrays, periodic wrap
-// included, and write only their own planes), so nothing is copied or recomputed on the device.
-// Because of the periodic wrap the last chunk is sent first; the adjoint of the first and the
-// last two chunks has to wait for the last forward launch, so about 4/K of the D2H time stays
-// exposed.  The caller's stream waits for both copy streams at the end: synchronising it covers
-// everything, as in the plain form.
+// chunks of x-planes.  The fields go up on a copy stream in transfers that run one plane ahead of
+// the chunks (transfer c ends with the first plane of chunk c+1; the last plane of the grid, which
+// chunk 0 reads through the periodic wrap, goes first), so the forward kernel of chunk c can run
+// (on the caller's stream) as soon as transfer c has landed.  The adjoint of chunk c follows the
+// forward of chunk c+1, and its gradients go down on a second copy stream while later transfers
+// are still coming up.  Kernels are the ordinary ones launched over a range of work items (they
+// read their x neighbours from the full arrays, periodic wrap included, and write only their own
+// planes), so nothing is copied or recomputed on the device.
+// What stays exposed is the lead (three transfers before the first gradients exist) and the tail
+// (the gradients of the last two chunks and of chunk 0 wait for the last forward launch); the
+// two chunks at either end are therefore half as long as the others.  The caller's stream waits
+// for both copy streams at the end: synchronising it covers everything, as in the plain form.
 // ------------------------------------------------------------------------------------------
-static constexpr int HOST_PIPE_MIN_PLANES = 4;      // smallest chunk the pipeline may use (host_workspace_bytes sizes for it)
-static int host_pipe_planes() {                     // planes per work item and per chunk
+static int host_pipe_planes() {                     // planes per chunk away from the ends: a multiple of the item
     const char* s = std::getenv("FPDE_HOST_PIPE_PLANES");
     const int v = s && *s ? std::atoi(s) : 8;
-    return std::max(HOST_PIPE_MIN_PLANES, std::min(64, v));
+    return std::max(1, std::min(16, v / HOST_PIPE_ITEM_PLANES)) * HOST_PIPE_ITEM_PLANES;
+}
+// Item boundaries of the chunks: one-item chunks at the two ends (two each), host_pipe_planes()
+// in between.
+static std::vector<int> host_pipe_chunks(int n0) {
+    const int G = HOST_PIPE_ITEM_PLANES, items = (n0 + G - 1) / G, mid = host_pipe_planes() / G;
+    std::vector<int> ib{0};
+    const int ends = items >= 8 ? 2 : 0;
+    for (int i = 0; i < ends; ++i) ib.push_back(ib.back() + 1);
+    while (ib.back() + mid <= items - ends) ib.push_back(ib.back() + mid);
+    while (ib.back() < items) ib.push_back(ib.back() + 1);
+    return ib;
 }
 static std::mutex g_pipe_mutex;
 static cudaStream_t g_pipe_in[64], g_pipe_out[64];
@@ -524,8 +539,7 @@ static cudaStream_t g_pipe_in[64], g_pipe_out[64];
 static bool host_pipeline_wanted(int op, const int* n) {
     const char* s = std::getenv("FPDE_HOST_PIPELINE");
     if (s && s[0] == '0') return false;
-    const int P = host_pipe_planes();
-    return op == FPDE_OP_NS_3D_T && (n[0] + P - 1) / P >= 6;
+    return op == FPDE_OP_NS_3D_T && (int)host_pipe_chunks(n[0]).size() - 1 >= 6;
 }
 
 static cudaError_t host_pipeline_streams(cudaStream_t* in, cudaStream_t* out) {
@@ -552,43 +566,47 @@ static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, flo
                                     void* d_ws, int nf, int ne) {
     cudaStream_t cs = q.stream, s_in = nullptr, s_out = nullptr;
     if (host_pipeline_streams(&s_in, &s_out) != cudaSuccess) return FPDE_ERR_CUDA;
-    const int n0 = q.n[0];
+    const int n0 = q.n[0], G = HOST_PIPE_ITEM_PLANES;
     const int64_t plane = (int64_t)q.n[1] * q.n[2] * q.n[3];
-    const int HOST_PIPE_PLANES = host_pipe_planes();
-    const int K = (n0 + HOST_PIPE_PLANES - 1) / HOST_PIPE_PLANES;
+    const std::vector<int> ib = host_pipe_chunks(n0);
+    const int K = (int)ib.size() - 1;
     std::vector<cudaEvent_t> ev(2 * K + 2, nullptr);
     auto cleanup = [&]() { for (cudaEvent_t e : ev) if (e) cudaEventDestroy(e); };
     for (auto& e : ev)
         if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cleanup(); return FPDE_ERR_CUDA; }
-    cudaEvent_t* e_in = ev.data();           // chunk c has arrived
+    cudaEvent_t* e_in = ev.data();           // transfer c has landed
     cudaEvent_t* e_bwd = ev.data() + K;      // gradients of chunk c are complete
     cudaEvent_t e_start = ev[2 * K], e_done = ev[2 * K + 1];
     bool ok = true;
     auto chk = [&](cudaError_t ce) { ok = ok && ce == cudaSuccess; };
-    auto p0 = [&](int c) { return (int64_t)c * HOST_PIPE_PLANES; };
-    auto np = [&](int c) { return (int64_t)std::min(HOST_PIPE_PLANES, n0 - c * HOST_PIPE_PLANES); };
+    auto first = [&](int c) { return (int64_t)ib[c] * G; };                          // planes of chunk c: [first, end)
+    auto end = [&](int c) { return std::min<int64_t>((int64_t)ib[c + 1] * G, n0); };
 
     // the copy streams start after whatever the caller queued before this call
     chk(cudaEventRecord(e_start, cs));
     chk(cudaStreamWaitEvent(s_in, e_start, 0));
     chk(cudaStreamWaitEvent(s_out, e_start, 0));
-    // fields up: last chunk first (the first chunk's forward needs it through the periodic wrap)
-    for (int i = 0; i < K; ++i) {
-        const int c = i == 0 ? K - 1 : i - 1;
-        const size_t off = (size_t)(p0(c) * plane), bytes = (size_t)(np(c) * plane) * sizeof(float);
+    auto up = [&](int64_t lo, int64_t hi) {
+        if (hi <= lo) return;
+        const size_t off = (size_t)(lo * plane), bytes = (size_t)((hi - lo) * plane) * sizeof(float);
         for (int f = 0; f < nf; ++f)
             chk(cudaMemcpyAsync(d_f[f] + off, h_fields[f] + off, bytes, cudaMemcpyHostToDevice, s_in));
+    };
+    // fields up: the wrap plane, then transfer c = planes up to and including the first of chunk c+1
+    up(n0 - 1, n0);
+    for (int c = 0; c < K; ++c) {
+        up(c == 0 ? 0 : end(c - 1) + 1, c == K - 1 ? n0 - 1 : end(c) + 1);
         chk(cudaEventRecord(e_in[c], s_in));
     }
-    q.planes_per_item = HOST_PIPE_PLANES;
+    q.planes_per_item = G;
     q.partials = static_cast<float*>(d_ws);
     q.loss_out = d_loss;
     for (int f = 0; f < nf; ++f) q.in[f] = d_f[f];
     auto fwd = [&](int c) {
-        for (int d = -1; d <= 1; ++d) chk(cudaStreamWaitEvent(cs, e_in[(c + d + K) % K], 0));
+        chk(cudaStreamWaitEvent(cs, e_in[c], 0));
         Problem r = q;
         for (int e = 0; e < ne; ++e) r.out[e] = d_r[e];
-        r.chunk_lo = c; r.chunk_hi = c + 1;
+        r.chunk_lo = ib[c]; r.chunk_hi = ib[c + 1];
         chk(launch_ns_fwd(r));
     };
     auto bwd = [&](int c) {
@@ -596,24 +614,23 @@ static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, flo
         for (int e = 0; e < ne; ++e) { r.aux[e] = d_r[e]; r.gscale[e] = 2.0 / (double)q.rows; }
         for (int f = 0; f < nf; ++f) r.out[f] = d_g[f];
         r.partials = nullptr;
-        r.chunk_lo = c; r.chunk_hi = c + 1;
+        r.chunk_lo = ib[c]; r.chunk_hi = ib[c + 1];
         chk(launch_ns_bwd(r));
         chk(cudaEventRecord(e_bwd[c], cs));
         chk(cudaStreamWaitEvent(s_out, e_bwd[c], 0));
-        const size_t off = (size_t)(p0(c) * plane), bytes = (size_t)(np(c) * plane) * sizeof(float);
+        const size_t off = (size_t)(first(c) * plane), bytes = (size_t)((end(c) - first(c)) * plane) * sizeof(float);
         for (int f = 0; f < nf; ++f)
             chk(cudaMemcpyAsync(h_gfields[f] + off, d_g[f] + off, bytes, cudaMemcpyDeviceToHost, s_out));
     };
-    // forward of chunk c once c+1 is there; adjoint of chunk c once the forward of c+1 is queued
-    // (chunk 0's adjoint needs the last chunk's residuals and comes at the end)
+    // the adjoint of chunk c once the forward of c+1 is queued; the chunks next to the wrap
+    // (the last one and chunk 0) need the last forward launch and come at the end
     fwd(0);
-    for (int c = 1; c <= K - 2; ++c) {
+    fwd(1);
+    for (int c = 2; c <= K - 1; ++c) {
         fwd(c);
-        if (c >= 2) bwd(c - 1);
+        bwd(c - 1);
     }
-    fwd(K - 1);
-    chk(launch_loss_finalize(q.partials, ns_items(q.n, false, HOST_PIPE_PLANES), ne, q.rows, d_loss, cs));
-    bwd(K - 2);
+    chk(launch_loss_finalize(q.partials, ns_items(q.n, false, G), ne, q.rows, d_loss, cs));
     bwd(K - 1);
     bwd(0);
     chk(cudaMemcpyAsync(h_loss, d_loss, (ne + 1) * sizeof(double), cudaMemcpyDeviceToHost, cs));

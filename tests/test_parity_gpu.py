@@ -192,11 +192,12 @@ def test_loss_grad_from_host_buffers():
     assert st == 9
 
 
-@pytest.mark.parametrize("shape", [(48, 10, 8, 8), (53, 6, 8, 16), (128, 4, 8, 8)])
+@pytest.mark.parametrize("shape", [(48, 10, 8, 8), (53, 6, 8, 16), (128, 4, 8, 8), (29, 6, 8, 8), (33, 4, 8, 8)])
 def test_pipelined_host_entry_for_navier_stokes(shape, monkeypatch):
-    """Grids with six or more 8-plane chunks take the pipelined form of the host-buffer entry
-    (chunks of x-planes go up, through forward and adjoint launches over chunk ranges, and down
-    again on three streams).  It must match the oracle, give bit-identical gradients to the plain
+    """Grids of 29 or more x-planes (six or more chunks) take the pipelined form of the host-buffer
+    entry (transfers of x-planes go up, through forward and adjoint launches over item ranges, and
+    down again on three streams; 29 planes is the smallest such grid, with 33 the last chunk is a
+    single plane and the last transfer empty).  It must match the oracle, give bit-identical gradients to the plain
     form (the same arithmetic per node), leave the copy streams covered by the caller's stream,
     and be repeatable back to back."""
     w = W.make("ns_tgv_128x16", seed=47, shape=shape, kind="randn")
