@@ -60,16 +60,16 @@ KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
 # summarised under profiles/; None where no capture has been taken yet.
 NCU_TRAFFIC_BYTES = {
     # half-size capture (64 planes) x 2: traffic is proportional to the number of planes
-    ("ns_tgv_128x16", "ns_fwd_kernel"): 2 * 518306560,
-    ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 761274112,
+    ("ns_tgv_128x16", "ns_fwd_kernel"): 2 * 518003968,
+    ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 762521088,
     ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 222671616,
     ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 366043648,
-    ("helmholtz_256", "star3d_kernel<fwd>"): 185158400,
-    ("helmholtz_256", "star3d_kernel<bwd>"): 101107200,
+    ("helmholtz_256", "star3d_kernel<fwd>"): 179527424,
+    ("helmholtz_256", "star3d_kernel<bwd>"): 97955328,
     ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 362135040,
     ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 511582720,
-    ("ns3d_steady_256", "ns3d_kernel<fwd>"): 516580096,
-    ("ns3d_steady_256", "ns3d_kernel<bwd>"): 734623232,
+    ("ns3d_steady_256", "ns3d_kernel<fwd>"): 516224256,
+    ("ns3d_steady_256", "ns3d_kernel<bwd>"): 735408896,
     ("grayscott_4096", "fused2d_kernel<grayscott_2d>"): 235297280,
     ("ns2d_steady_4096", "fused2d_kernel<ns_2d_steady>"): 372255488,
 }
