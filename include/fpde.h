@@ -273,14 +273,28 @@ int fpde_bwd_f64(int op,
  *   d_arena    DEVICE scratch of at least fpde_host_arena_bytes() bytes, 256-byte aligned, owned
  *              by the caller (staging for fields, sources, residuals, gradients, loss, workspace)
  * Same status codes as fpde_fwd / fpde_bwd; FPDE_ERR_WORKSPACE if the arena is too small.
- * For FPDE_OP_NS_3D_T on grids of six or more 8-plane chunks the call is pipelined: chunks of
- * x-planes are copied up on one internal stream, run through forward and adjoint launches over
- * chunk ranges on `stream`, and copied down on a second internal stream, so the two copy
+ * For FPDE_OP_NS_3D_T on grids that split into six or more chunks of x-planes (29 planes and up)
+ * the call is pipelined: the fields are copied up on one internal stream in transfers that run one
+ * plane ahead of the chunks, run through forward and adjoint launches over the chunks' work items
+ * on `stream`, and the gradients are copied down on a second internal stream, so the two copy
  * directions overlap; `stream` waits for both internal streams before the call's work counts as
  * done on it, so synchronising `stream` is still all a caller has to do.  (FPDE_HOST_PIPELINE=0
  * in the environment selects the plain one-stream form.)
  */
 size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape);
+
+/*
+ * The plan the pipelined form of fpde_loss_grad_host follows for a grid of n0 x-planes (host-only
+ * query, no device needed).  Returns the number of chunks K, or 0 if such a grid takes the plain
+ * form.  If `planes` is not NULL it receives 3 ints per chunk c (cap = number of chunks it has room
+ * for; nothing is written and -K is returned if cap < K):
+ *   planes[3c]   first x-plane of chunk c (the chunk ends where the next one starts, the last at n0)
+ *   planes[3c+1] first x-plane of upload transfer c
+ *   planes[3c+2] one past the last x-plane of upload transfer c (an empty transfer has both equal)
+ * Plane n0-1 is uploaded before transfer 0.  The forward launch of chunk c follows transfer c; the
+ * adjoint launch of chunk c follows the forward launch of chunk c+1 (chunks K-1 and 0: the last one).
+ */
+int fpde_host_pipeline_plan(int n0, int* planes, int cap);
 int fpde_loss_grad_host(int op,
                         const float* const* h_fields,
                         const float* const* h_sources,

@@ -85,6 +85,8 @@ def lib():
                                    ctypes.c_void_p]
         L.fpde_host_arena_bytes.restype = ctypes.c_size_t
         L.fpde_host_arena_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_host_pipeline_plan.restype = ctypes.c_int
+        L.fpde_host_pipeline_plan.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.c_int]
         L.fpde_loss_grad_host.restype = ctypes.c_int
         L.fpde_loss_grad_host.argtypes = [ctypes.c_int, vpp, vpp, vpp, ctypes.c_void_p, ctypes.c_int,
                                           ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
@@ -290,6 +292,20 @@ def fpde_bwd(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, work
 
 def host_arena_bytes(op, shape) -> int:
     return int(lib().fpde_host_arena_bytes(_opid(op), len(shape), _i64(shape)))
+
+
+def host_pipeline_plan(n0: int):
+    """Chunks of the pipelined host path for n0 x-planes: list of (first plane of the chunk, first
+    plane of its upload transfer, one past the transfer's last plane); empty if the plain form runs."""
+    L = lib()
+    k = L.fpde_host_pipeline_plan(int(n0), None, 0)
+    if k <= 0:
+        return []
+    buf = (ctypes.c_int * (3 * k))()
+    got = L.fpde_host_pipeline_plan(int(n0), buf, k)
+    if got != k:
+        raise FpdeError("fpde_host_pipeline_plan", got)
+    return [(buf[3 * c], buf[3 * c + 1], buf[3 * c + 2]) for c in range(k)]
 
 
 def loss_grad_host_status(op, h_fields, h_sources, h_gfields, h_loss, shape, spacing, coeffs, bc, arena,

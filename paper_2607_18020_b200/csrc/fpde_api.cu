@@ -542,6 +542,35 @@ static bool host_pipeline_wanted(int op, const int* n) {
     return op == FPDE_OP_NS_3D_T && (int)host_pipe_chunks(n[0]).size() - 1 >= 6;
 }
 
+// Upload transfer c of a plan with item boundaries ib: planes [lo, hi).  Transfers run one plane
+// ahead of the chunks; plane n0-1 goes up separately, first.
+static void host_pipe_transfer(const std::vector<int>& ib, int n0, int c, int64_t* lo, int64_t* hi) {
+    const int G = HOST_PIPE_ITEM_PLANES, K = (int)ib.size() - 1;
+    auto end = [&](int k) { return std::min<int64_t>((int64_t)ib[k + 1] * G, n0); };
+    *lo = c == 0 ? 0 : end(c - 1) + 1;
+    *hi = c == K - 1 ? n0 - 1 : end(c) + 1;
+    if (*hi < *lo) *hi = *lo;
+}
+
+int fpde_host_pipeline_plan(int n0, int* planes, int cap) {
+    if (n0 < 1) return 0;
+    const std::vector<int> ib = host_pipe_chunks(n0);
+    const int K = (int)ib.size() - 1;
+    const char* s = std::getenv("FPDE_HOST_PIPELINE");
+    if ((s && s[0] == '0') || K < 6) return 0;
+    if (planes) {
+        if (cap < K) return -K;
+        for (int c = 0; c < K; ++c) {
+            int64_t lo, hi;
+            host_pipe_transfer(ib, n0, c, &lo, &hi);
+            planes[3 * c] = ib[c] * HOST_PIPE_ITEM_PLANES;
+            planes[3 * c + 1] = (int)lo;
+            planes[3 * c + 2] = (int)hi;
+        }
+    }
+    return K;
+}
+
 static cudaError_t host_pipeline_streams(cudaStream_t* in, cudaStream_t* out) {
     int dev = 0;
     cudaError_t ce = cudaGetDevice(&dev);
@@ -595,7 +624,9 @@ static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, flo
     // fields up: the wrap plane, then transfer c = planes up to and including the first of chunk c+1
     up(n0 - 1, n0);
     for (int c = 0; c < K; ++c) {
-        up(c == 0 ? 0 : end(c - 1) + 1, c == K - 1 ? n0 - 1 : end(c) + 1);
+        int64_t lo, hi;
+        host_pipe_transfer(ib, n0, c, &lo, &hi);
+        up(lo, hi);
         chk(cudaEventRecord(e_in[c], s_in));
     }
     q.planes_per_item = G;

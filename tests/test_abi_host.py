@@ -152,6 +152,41 @@ def test_fwd_bwd_and_f64_validation_without_a_gpu():
     assert st == 3
 
 
+def test_host_pipeline_plan_covers_every_plane_once_ahead_of_its_chunk(monkeypatch):
+    """The plan of the pipelined host path: chunks tile [0, n0) in whole 4-plane work items, the
+    upload transfers tile [0, n0-1) (plane n0-1 goes first, on its own), and transfer c ends one
+    plane past chunk c, which is what lets the forward launch of chunk c wait for transfer c alone."""
+    monkeypatch.delenv("FPDE_HOST_PIPELINE", raising=False)
+    monkeypatch.delenv("FPDE_HOST_PIPE_PLANES", raising=False)
+    assert B.host_pipeline_plan(28) == [] and B.host_pipeline_plan(1) == [] and B.host_pipeline_plan(0) == []
+    for n0 in (29, 30, 32, 33, 48, 53, 64, 127, 128, 129, 1000):
+        plan = B.host_pipeline_plan(n0)
+        K = len(plan)
+        assert K >= 6, n0
+        starts = [p[0] for p in plan] + [n0]
+        assert starts[0] == 0 and all(a < b for a, b in zip(starts, starts[1:])), (n0, starts)
+        assert all(s % 4 == 0 for s in starts[:-1])
+        sizes = [b - a for a, b in zip(starts, starts[1:])]
+        assert max(sizes) <= 8 and sizes[0] == sizes[1] == 4 and sizes[-2] <= 4 and sizes[-1] <= 4, (n0, sizes)
+        covered = []
+        for c, (first, lo, hi) in enumerate(plan):
+            assert 0 <= lo <= hi <= n0
+            covered += list(range(lo, hi))
+            end = starts[c + 1]
+            if c < K - 1:
+                assert hi == end + 1, (n0, c)            # one plane ahead of the chunk
+            # everything chunk c reads (its planes and one either side, periodic) is up by then
+            need = set(range(first, end)) | {(first - 1) % n0, end % n0}
+            assert need <= set(covered) | {n0 - 1}, (n0, c, sorted(need - set(covered)))
+        assert sorted(set(covered) | {n0 - 1}) == list(range(n0)), n0
+        assert len([p for p in covered if p != n0 - 1]) == len(set(covered) - {n0 - 1})   # nothing twice but the wrap plane
+    L = B.lib()
+    small = (ctypes.c_int * 6)()
+    assert L.fpde_host_pipeline_plan(128, small, 2) == -len(B.host_pipeline_plan(128))
+    monkeypatch.setenv("FPDE_HOST_PIPELINE", "0")
+    assert B.host_pipeline_plan(128) == []
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
     monkeypatch.setattr(B, "_lib", None)
