@@ -8,6 +8,7 @@ exception is raised.
 from __future__ import annotations
 
 import ctypes
+import functools
 import os
 from typing import List, Optional, Sequence
 
@@ -109,10 +110,8 @@ def _opid(op) -> int:
 
 
 def _ptr_array(ptrs: Sequence[Optional[int]]):
-    arr = (ctypes.c_void_p * max(1, len(ptrs)))()
-    for i, p in enumerate(ptrs):
-        arr[i] = p
-    return ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p))
+    # a ctypes array is accepted where the prototype says POINTER(c_void_p): no cast needed
+    return (ctypes.c_void_p * max(1, len(ptrs)))(*ptrs)
 
 
 def _dev_ptrs(tensors) -> List[int]:
@@ -125,16 +124,33 @@ def _dev_ptrs(tensors) -> List[int]:
     return out
 
 
+# The small host arrays of a call (shape, spacings, coefficients, boundary kinds) are read-only
+# for the library and repeat from call to call: built once per distinct value.
+@functools.lru_cache(maxsize=512)
+def _i64_of(t: tuple):
+    return (ctypes.c_int64 * max(1, len(t)))(*t)
+
+
+@functools.lru_cache(maxsize=512)
+def _f64_of(t: tuple):
+    return (ctypes.c_double * max(1, len(t)))(*t)
+
+
+@functools.lru_cache(maxsize=512)
+def _bcs_of(t: tuple):
+    return (ctypes.c_int * max(1, len(t)))(*[BC_IDS[b] if isinstance(b, str) else int(b) for b in t])
+
+
 def _i64(v):
-    return (ctypes.c_int64 * max(1, len(v)))(*[int(x) for x in v])
+    return _i64_of(tuple(int(x) for x in v))
 
 
 def _f64(v):
-    return (ctypes.c_double * max(1, len(v)))(*[float(x) for x in v])
+    return _f64_of(tuple(float(x) for x in v))
 
 
 def _bcs(bc):
-    return (ctypes.c_int * max(1, len(bc)))(*[BC_IDS[b] if isinstance(b, str) else int(b) for b in bc])
+    return _bcs_of(tuple(bc))
 
 
 def strerror(status: int) -> str:
