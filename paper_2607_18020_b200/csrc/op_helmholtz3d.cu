@@ -11,7 +11,7 @@
 //   five x-planes of its own column in registers (rotated by unrolling); the y+-1, y+-2
 //   neighbours of the current plane are read through L1 (other threads of the same block loaded
 //   those lines two steps earlier); z neighbours come from the adjacent lanes' registers.  The
-//   plane the window will need three steps later is prefetched into L2.  Arithmetic is packed
+//   plane the window loads in the next step is prefetched into L2.  Arithmetic is packed
 //   fp32x2; the star is evaluated as  sum_a w_a (16 (q[-1]+q[+1]) - (q[-2]+q[+2])) + K q  with
 //   K = k^2 - 30 sum_a w_a.
 #include "fpde_common.cuh"

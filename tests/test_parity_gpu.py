@@ -100,6 +100,30 @@ def test_config_fields(name, shape):
     _check_case(W.make(name, seed=42, shape=shape), "%s%s" % (name, shape or ""))
 
 
+WIDE_ADDRESS_SWITCHES = ("FPDE_LAP2D_OFF32", "FPDE_FUSED2D_OFF32", "FPDE_STAR3D_OFF32", "FPDE_NS2D_OFF32",
+                         "FPDE_NS3D_OFF32", "FPDE_NS_OFF32")
+
+
+@pytest.mark.parametrize("name,shape", [c for c in MEDIUM if c[1] is not None])
+def test_builds_with_64_bit_addressing(name, shape, monkeypatch):
+    """Arrays above 2^30 floats run kernel builds with 64-bit offsets; the switches select those
+    builds on grids small enough for the oracle (the 3-D+T, steady NS and single-pass kernels have
+    no other test at such sizes)."""
+    for k in WIDE_ADDRESS_SWITCHES:
+        monkeypatch.setenv(k, "0")
+    w = W.make(name, seed=48, shape=shape, kind="randn")
+    _check_case(w, "%s%s 64-bit offsets" % (name, shape))
+    if B.has_single_pass(w.op):
+        _, _, g_ref, _ = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+        grads = [torch.empty(w.shape, dtype=torch.float32, device="cuda") for _ in w.fields]
+        ws = torch.empty(B.fwd_bwd_workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+        B.fpde_fwd_bwd(w.op, to_dev(torch, w.fields), to_dev(torch, w.sources), None, grads, None, w.shape,
+                       w.spacing, w.coeffs, w.bc, ws)
+        torch.cuda.synchronize()
+        for f, (g, gr) in enumerate(zip(grads, g_ref)):
+            assert_close(g.cpu().numpy(), gr, "%s%s single pass, 64-bit offsets, gradient %d" % (name, shape, f))
+
+
 @pytest.mark.parametrize("name,shape", TINY)
 @pytest.mark.parametrize("seed", [42, 43, 44, 45, 46])
 def test_randn_fields_tiny(name, shape, seed):
