@@ -170,8 +170,9 @@ __global__ void __launch_bounds__(128, MINB) fused2d_kernel(const Fused2dParams 
     const int a0 = rc * p.rows_per_item;
     const int a1 = min(a0 + p.rows_per_item, n0);
 
+    // row read for index j in [-2, n0 + 1] (what the march asks for): wrapped once, no division
     auto row_of = [&](int j) -> int {
-        if (PER) { j %= n0; return j < 0 ? j + n0 : j; }
+        if (PER) return j < 0 ? j + n0 : (j >= n0 ? j - n0 : j);
         return max(0, min(n0 - 1, j));
     };
     auto load_row = [&](int j, V4 (&F)[NF], V4 (&S)[NSA]) {
