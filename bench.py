@@ -70,7 +70,7 @@ NCU_TRAFFIC_BYTES = {
     ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 511582720,
     ("ns3d_steady_256", "ns3d_kernel<fwd>"): 516224256,
     ("ns3d_steady_256", "ns3d_kernel<bwd>"): 735408896,
-    ("grayscott_4096", "fused2d_kernel<grayscott_2d>"): 235297280,
+    ("grayscott_4096", "fused2d_kernel<grayscott_2d>"): 235188736,
     ("ns2d_steady_4096", "fused2d_kernel<ns_2d_steady>"): 372255488,
 }
 FALLBACK_HBM_GBS = 6650.0
