@@ -144,9 +144,10 @@ __device__ __forceinline__ void ns3d_step(const Ns3dParams& p, const Ns3dThread&
     }
 }
 
-// O32: 32-bit byte offsets from the array bases (arrays of at most 2^30 floats); used where the
-// build comes out without spills (forward, the adjoint without zero-extension, and the interior
-// steps of the masking adjoint: with its shell steps as well that kernel spills)
+// O32: 32-bit byte offsets from the array bases (arrays of at most 2^30 floats): in the forward
+// kernel, the adjoint without zero-extension, and the interior steps of the masking adjoint (with
+// its shell steps as well that build spills 200 bytes; as it is, 16 bytes of stack at 255
+// registers, which the timed loop does not notice)
 template <bool BWD, int MINB, bool PRE = false, bool O32 = false>
 __global__ void __launch_bounds__(128, MINB) ns3d_kernel(const Ns3dParams p) {
     constexpr int NA = BWD ? 7 : 4;
