@@ -390,7 +390,13 @@ def single_pass_figures(torch, prob, steps, warmup, flush, peak):
     e1.record(); torch.cuda.synchronize()
     warm_ms = e0.elapsed_time(e1) / steps
     gbs = bpp * N / (ms * 1e-3) / 1e9
+
+    class OneCall:                      # the same step for the graph helper (one call instead of a pair)
+        fwd = staticmethod(prob.fwd_bwd)
+        bwd = staticmethod(lambda: None)
+
     return {"ms": ms, "points_per_s": N / (ms * 1e-3), "warm_points_per_s": N / (warm_ms * 1e-3),
+            "graph_points_per_s": graph_points_per_s(torch, OneCall, N, pairs=10, replays=max(3, steps // 10)),
             "algorithmic_bytes_per_point": bpp, "gbs": gbs, "frac": gbs / peak,
             "what": "fpde_fwd_bwd, residual arrays not stored; launches: 1 kernel + loss finalise"}
 
