@@ -27,7 +27,27 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("name,shape,world", CASES)
+def _random_cases():
+    """Randomly drawn (shape, number of slabs) per slab-capable operator, fixed seed."""
+    rng = np.random.RandomState(20260719)
+    out = []
+    for name in ("ns_tgv_128x16", "helmholtz_256", "poisson_1024", "ns2d_steady_4096", "ns3d_steady_256", "grayscott_4096"):
+        cfg = W.CONFIGS[name]
+        nd = len(cfg["shape"])
+        radius = S.RADIUS[cfg["op"]]
+        for _ in range(6):
+            world = int(rng.randint(1, 6))
+            shape = [int(rng.randint(max(2 * radius * world, 4 * radius + 1), 2 * radius * world + 30))]
+            for a in range(1, nd):
+                if a == nd - 1:
+                    shape.append(4 * int(rng.randint(2, 5 if nd == 4 else 30)))
+                else:
+                    shape.append(int(rng.randint(2 * radius + 1, 12)))
+            out.append((name, tuple(shape), world))
+    return out
+
+
+@pytest.mark.parametrize("name,shape,world", CASES + _random_cases())
 def test_slabs_reproduce_the_whole_grid(name, shape, world):
     w = W.make(name, seed=42, shape=shape, kind="randn")
     plan_list = S.plans(w.op, w.shape, world)
