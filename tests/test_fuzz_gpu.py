@@ -73,3 +73,29 @@ def test_random_shape(name, shape, seed):
         assert_close(g.cpu().numpy(), gr, "%s one-call gradient %d" % (tag, f))
     for e, (r, rr) in enumerate(zip(r1, R_ref)):
         assert_close(r.cpu().numpy(), rr, "%s one-call residual %d" % (tag, e))
+
+
+@pytest.mark.parametrize("name,shape,seed", CASES[::3], ids=["%s-%s" % (n, "x".join(map(str, s))) for n, s, _ in CASES[::3]])
+def test_random_shape_adjoint_of_arbitrary_upstream_arrays(name, shape, seed):
+    """fpde_bwd and its double-precision twin on upstream arrays that are not residuals (non-zero at
+    nodes without a row, where they must be ignored), unequal spacings and unequal scales."""
+    rng = np.random.RandomState(seed)
+    h = tuple(float(x) for x in rng.uniform(0.05, 0.4, size=len(shape)))
+    w = W.make(name, seed=seed, shape=shape, kind="randn", spacing=h)
+    G = W.random_sensitivities(w, seed=seed + 1)
+    gscale = [float(x) for x in rng.uniform(0.2, 2.0, size=len(G))]
+    ref = oracle.bwd(w.op, w.fields, [s * g.astype(np.float64) for s, g in zip(gscale, G)], w.shape, w.spacing, w.coeffs)
+    fields = to_dev(torch, w.fields)
+    grads = run_bwd(torch, w, fields, to_dev(torch, G), gscale)
+    for f, (g, gr) in enumerate(zip(grads, ref)):
+        assert_close(g.view.cpu().numpy(), gr, "%s%s adjoint %d" % (name, shape, f))
+    f64 = [torch.from_numpy(np.ascontiguousarray(a, dtype=np.float64)).cuda() for a in w.fields]
+    g64 = [torch.from_numpy(np.ascontiguousarray(a, dtype=np.float64)).cuda() for a in G]
+    out = [torch.empty(w.shape, dtype=torch.float64, device="cuda") for _ in w.fields]
+    B.fpde_bwd_f64(w.op, f64, g64, gscale, out, w.shape, w.spacing, w.coeffs, w.bc)
+    torch.cuda.synchronize()
+    ref64 = oracle.bwd(w.op, [a.astype(np.float64) for a in w.fields],
+                       [s * g.astype(np.float64) for s, g in zip(gscale, G)], w.shape, w.spacing, w.coeffs)
+    for f, (g, gr) in enumerate(zip(out, ref64)):
+        d = np.abs(g.cpu().numpy() - gr).max()
+        assert d <= 1e-11 * max(1.0, np.abs(gr).max()), "%s%s fp64 adjoint %d: %g" % (name, shape, f, d)
