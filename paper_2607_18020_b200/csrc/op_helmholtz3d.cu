@@ -135,7 +135,11 @@ __device__ __forceinline__ void star3d_body(const Star3dParams& p, int cb, int m
         const V4 a1v = load_h(h_at(pos, dm1), dm1d || pd, false), b1v = load_h(h_at(pos, dp1), dp1d || pd, false);
         const V4 a2v = load_h(h_at(pos, dm2), dm2d || pd, false), b2v = load_h(h_at(pos, dp2), dp2d || pd, false);
         V4 src = v4zero();
-        if (FWD) src = ld_at(c_at(pos, 0));
+        if (FWD) {
+            // read once and by nobody else: streamed past L1, which the y neighbours' lines need
+            const float4 t4 = __ldcs(reinterpret_cast<const float4*>(c_at(pos, 0)));
+            src.lo = make_float2(t4.x, t4.y); src.hi = make_float2(t4.z, t4.w);
+        }
         float2 E = make_float2(0.f, 0.f);
         if (efetch) E = __ldg(reinterpret_cast<const float2*>(h_at(pos, eoff)));
         if (ROWMASK && (d0 || pd)) E = make_float2(0.f, 0.f);
