@@ -64,8 +64,8 @@ NCU_TRAFFIC_BYTES = {
     ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 762521088,
     ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 222671616,
     ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 366043648,
-    ("helmholtz_256", "star3d_kernel<fwd>"): 179527424,
-    ("helmholtz_256", "star3d_kernel<bwd>"): 97955328,
+    ("helmholtz_256", "star3d_kernel<fwd>"): 169988352,
+    ("helmholtz_256", "star3d_kernel<bwd>"): 97383424,
     ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 362135040,
     ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 511582720,
     ("ns3d_steady_256", "ns3d_kernel<fwd>"): 516224256,
