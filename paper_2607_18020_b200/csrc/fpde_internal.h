@@ -81,6 +81,18 @@ inline cudaError_t launch_kernel_smem(void (*kernel)(KArgs...), dim3 grid, dim3 
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
 }
 
+// Planes per work item of the 2.5-D kernels: the length tuned on large grids, halved on grids that
+// items of that length would not spread over the GPU, never below 4.  On small grids a step is
+// latency-bound and what counts is how many items march concurrently: at least four per SM on
+// grids whose arrays fit L2 several times over (under 2^22 points), two per SM above that, where
+// longer items pay by re-reading fewer halo planes.
+inline int planes_for_grid(int n0, int tuned, long items_per_chunk, long long points) {
+    const long target = (points < (1ll << 22) ? 4 : 2) * 148;
+    int planes = tuned;
+    while (planes > 4 && items_per_chunk * ((n0 + planes - 1) / planes) < target) planes = planes / 2 < 4 ? 4 : planes / 2;
+    return planes;
+}
+
 // Launchers: return cudaGetLastError() after queuing the kernels.
 cudaError_t launch_burgers_fwd(const Problem& p);
 cudaError_t launch_burgers_bwd(const Problem& p);

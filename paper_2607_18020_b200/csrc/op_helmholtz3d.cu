@@ -227,9 +227,12 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     ty = std::max(1, std::min(256 / tx, ty));
     block = dim3(tx, ty, 1);
     // the forward kernel (two input streams) runs best on long items, the adjoint on short ones
-    p.planes_per_item = fwd ? env_int("FPDE_STAR3D_PLANES_F", 32) : env_int("FPDE_STAR3D_PLANES_B", 10);
     p.ncb = (p.nc4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
+    const long per_chunk = (long)p.ncb * p.nmb;
+    const long long points = (long long)p.n0 * p.n1 * p.n2;
+    p.planes_per_item = fwd ? env_int("FPDE_STAR3D_PLANES_F", planes_for_grid(p.n0, 32, per_chunk, points))
+                            : env_int("FPDE_STAR3D_PLANES_B", planes_for_grid(p.n0, 10, per_chunk, points));
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     double wsum = 0.0;
     for (int a = 0; a < 3; ++a) {

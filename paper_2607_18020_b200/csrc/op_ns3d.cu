@@ -232,9 +232,9 @@ static void ns3d_geometry(const int* n, Ns3dParams& p, dim3& block) {
     int ty = env_int("FPDE_NS3D_TY", 128 / tx);
     ty = std::max(1, std::min(128 / tx, ty));
     block = dim3(tx, ty, 1);
-    p.planes_per_item = env_int("FPDE_NS3D_PLANES", 24);
     p.ncb = (p.nc4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
+    p.planes_per_item = env_int("FPDE_NS3D_PLANES", planes_for_grid(p.n0, 24, (long)p.ncb * p.nmb, (long long)n[0] * n[1] * n[2]));
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     const char* pf = std::getenv("FPDE_NS3D_PREFETCH");
     p.prefetch = pf && *pf ? std::atoi(pf) : 2;

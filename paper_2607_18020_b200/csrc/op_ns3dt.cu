@@ -277,9 +277,10 @@ static void ns_geometry(const Problem& q, NsParams& p, dim3& block) {
     int ty = env_int("FPDE_NS_TY", 128 / tx);
     ty = std::max(1, std::min(128 / tx, ty));
     block = dim3(tx, ty, 1);
-    p.planes_per_item = q.planes_per_item > 0 ? q.planes_per_item : env_int("FPDE_NS_PLANES", 24);
     p.ncb = (p.C4 + tx - 1) / tx;
     p.nmb = (p.n1 + ty - 1) / ty;
+    p.planes_per_item = q.planes_per_item > 0 ? q.planes_per_item
+                                              : env_int("FPDE_NS_PLANES", planes_for_grid(p.n0, 24, (long)p.ncb * p.nmb, (long long)q.n[0] * q.n[1] * q.n[2] * q.n[3]));
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     const char* pf = std::getenv("FPDE_NS_PREFETCH");
     p.prefetch = pf && *pf ? std::atoi(pf) : 2;
