@@ -6,7 +6,7 @@
  * sensitivities dL/dres back to dL/dfield with a hand-derived discrete adjoint in gather form.
  * It is the method of the paper's Section 2 ("Kernel design and discrete analytic adjoints"):
  * fused forward stencil (Section 2.1), analytic discrete-adjoint backward (Section 2.2,
- * Eq. 1, Appendix A.2) and boundary-gradient correction (Section 2.3, Appendix A.4).
+ * Eq. 1, Appendix A.3) and boundary-gradient correction (Section 2.3, Appendix A.5).
  *
  * General rules (all entry points)
  *   - Plain C types only.  Nothing throws or aborts; every call returns an fpde_status.
@@ -14,9 +14,12 @@
  *     shape.  Space-time grids keep t as the last (contiguous) axis.
  *   - "device" pointers are CUDA device memory owned by the caller, 16-byte aligned, not
  *     overlapping; "host" pointers are ordinary host memory read during the call only.
- *   - The library allocates no device memory and keeps no state between calls.  Work is queued
- *     on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and the
- *     call returns without waiting for it.
+ *   - The library allocates no device memory.  The kernel entry points keep no state between
+ *     calls.  Two entry points keep a little per device, created on first use and held until the
+ *     process exits: fpde_loss_grad_host (two copy streams and a pool of events for its pipelined
+ *     form) and fpde_fwd_noalloc (the address of its fixed scratch array).  Work is queued on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and the call
+ *     returns without waiting for it.
  *   - On any status other than FPDE_OK nothing has been launched.  FPDE_ERR_CUDA reports a
  *     launch the CUDA runtime rejected.
  *   - With no CUDA device the entry points still load and validate, and a launch attempt
@@ -105,7 +108,7 @@ typedef enum {
     FPDE_OP_COUNT = 9
 } fpde_op;
 
-/* Boundary kind of one array axis (Appendix A.4 names the three causes of boundary terms:
+/* Boundary kind of one array axis (Appendix A.5 names the three causes of boundary terms:
  * prescribed values, one-sided formulas, omitted neighbours). */
 typedef enum {
     FPDE_BC_PERIODIC = 0,   /* rows at every node, wrap-around neighbours                       */
@@ -131,7 +134,10 @@ const char* fpde_strerror(int status);
 int64_t fpde_row_count(int op, int ndim, const int64_t* shape);
 
 /* Bytes of device scratch fpde_fwd needs for this operator and grid (loss partial sums); 0 if
- * the operator / shape is invalid.  fpde_bwd needs none.  Host only. */
+ * the operator / shape is invalid.  fpde_bwd needs none.  Host only.
+ * The figure follows the launch shape, which the FPDE_* tuning variables of the environment can
+ * change (they are read on every call): size the workspace after setting them, not before.  A call
+ * whose workspace has become too small is refused with FPDE_ERR_WORKSPACE, never run short. */
 size_t fpde_workspace_bytes(int op, int ndim, const int64_t* shape);
 
 /*
@@ -322,7 +328,9 @@ int fpde_loss_grad_host(int op,
  * cudaMalloc / cudaFree and calls no allocating routine.
  *
  *   - Grids whose forward pass needs more scratch than that (fpde_workspace_bytes() >
- *     FPDE_NOALLOC_SCRATCH_BYTES) are refused with FPDE_ERR_WORKSPACE; nothing is launched.
+ *     FPDE_NOALLOC_SCRATCH_BYTES) are refused with FPDE_ERR_WORKSPACE; nothing is launched.  The
+ *     need follows the launch shape, so a tuning variable that shortens the work items can turn
+ *     an accepted grid into a refused one.
  *   - The first call on each device looks up the array's device address (with that device
  *     current).  Make that first call outside any stream capture.
  *   - Every call on a device shares the one array.  The kernels overwrite every slot they later
@@ -350,6 +358,16 @@ int fpde_fwd_noalloc(int op,
  * Returns UINT_MAX if the counter cannot be read.
  */
 unsigned int fpde_diag_tma_timeouts(void);
+
+/*
+ * Diagnostic, host only.  1 if the shared-memory-staged Navier-Stokes kernels (an opt-in variant,
+ * FPDE_NS_TMA=1) can take an (x,y,z,t) grid of this shape with tiles of `tile_rows` rows (4 or 8)
+ * and `narrays` arrays per pipeline stage (4 forward, 7 adjoint) inside `smem_limit` bytes of
+ * dynamic shared memory; 0 otherwise, in which case fpde_fwd / fpde_bwd run the default kernels.
+ * The rule includes the copy engine's requirement that every destination in shared memory starts
+ * on a 128-byte boundary.
+ */
+int fpde_diag_ns_tma_geometry(const int64_t* shape, int tile_rows, int narrays, size_t smem_limit);
 
 #ifdef __cplusplus
 }

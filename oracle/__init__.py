@@ -7,7 +7,7 @@ double here; nothing is regenerated.
 
 ``fwd`` evaluates every residual row from its definition and the mean-square loss
 (Section 2.1 of the paper for the residual structure, with the per-operator readings listed in
-the design notes); ``bwd`` forms ``J^T G`` by scatter over rows (Section 2.2 / Appendix A.2).
+the design notes); ``bwd`` forms ``J^T G`` by scatter over rows (Section 2.2 / Appendix A.3).
 """
 from __future__ import annotations
 

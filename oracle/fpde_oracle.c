@@ -9,9 +9,9 @@
  * CPU-baseline leg may call it.
  *
  * What is computed follows the paper's Section 2.1 (residuals assembled from centred finite
- * differences of grid-aligned fields), Section 2.2 and Appendix A.2 (the gradient is the action
+ * differences of grid-aligned fields), Section 2.2 and Appendix A.3 (the gradient is the action
  * of the transposed discrete Jacobian on the upstream sensitivities G = dL/dres), and Appendix
- * A.4 (near-boundary rows differ because of prescribed values, one-sided formulas or omitted
+ * A.5 (near-boundary rows differ because of prescribed values, one-sided formulas or omitted
  * neighbours).  The paper spells out only the steady 2-D Navier-Stokes operator; the other row
  * definitions used here are the readings listed in this repository's design notes.
  *
@@ -43,7 +43,7 @@ typedef struct { int n; i64 idx[6]; double w[6]; } stencil;
 
 static i64 wrap(i64 i, i64 n) { return ((i % n) + n) % n; }
 
-/* First derivative, second order (Appendix A.2 centred formula q_x = (q[i+1]-q[i-1])/(2h);
+/* First derivative, second order (Appendix A.3 centred formula q_x = (q[i+1]-q[i-1])/(2h);
  * one-sided rows: (-3,4,-1)/(2h) and (3,-4,1)/(2h)).  Returns 0 where the axis carries no row. */
 static int d1(int bc, i64 i, i64 n, double h, stencil* s) {
     double c = 1.0 / (2.0 * h);
@@ -65,7 +65,7 @@ static int d1(int bc, i64 i, i64 n, double h, stencil* s) {
     return 1;
 }
 
-/* Second derivative, second order (Appendix A.2: q_xx = (q[i+1]-2q[i]+q[i-1])/h^2; one-sided
+/* Second derivative, second order (Appendix A.3: q_xx = (q[i+1]-2q[i]+q[i-1])/h^2; one-sided
  * rows use the four-point second-order formula (2,-5,4,-1)/h^2). */
 static int d2(int bc, i64 i, i64 n, double h, stencil* s) {
     double c = 1.0 / (h * h);
@@ -323,7 +323,7 @@ static i64 ns3dt(int mode, const double* const* fld, double* const* res, const d
 /* Steady incompressible Navier-Stokes on an (x,y) array, exactly the paper's Section 2.1 system:
  *   res_u = u u_x + v u_y + p_x - nu (u_xx + u_yy),  res_v = u v_x + v v_y + p_y - nu (v_xx + v_yy),
  *   res_div = u_x + v_y,
- * centred differences (Appendix A.2), rows at the nodes where they fit (interior points); the
+ * centred differences (Appendix A.3), rows at the nodes where they fit (interior points); the
  * outer ring is data.  fld = {u,v,p}; res / G / grd index: 0 res_u, 1 res_v, 2 res_div. */
 static i64 ns2d(int mode, const double* const* fld, double* const* res, const double* const* G,
                 double* const* grd, const i64* n, const double* h, const double* c) {

@@ -101,6 +101,9 @@ def lib():
                                        ctypes.c_void_p]
         L.fpde_diag_tma_timeouts.restype = ctypes.c_uint
         L.fpde_diag_tma_timeouts.argtypes = []
+        L.fpde_diag_ns_tma_geometry.restype = ctypes.c_int
+        L.fpde_diag_ns_tma_geometry.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_size_t]
         _lib = L
     return _lib
 
@@ -243,6 +246,42 @@ def _stream_handle(stream) -> Optional[int]:
     return int(stream)
 
 
+class _on_device_of:
+    """Context for one call: every tensor argument must live on one CUDA device, and that device
+    is made current for the call (the library launches on the current device, so a tensor of
+    another GPU would be dereferenced there as a foreign address)."""
+
+    def __init__(self, *groups):
+        dev = None
+        for g in groups:
+            if g is None:
+                continue
+            for t in (g if isinstance(g, (list, tuple)) else [g]):
+                d = getattr(t, "device", None)
+                if d is None or not hasattr(t, "data_ptr"):
+                    continue
+                if d.type != "cuda":
+                    raise ValueError("fpde: tensor on %s, expected a CUDA tensor" % (d,))
+                if dev is None:
+                    dev = d
+                elif d != dev:
+                    raise ValueError("fpde: tensors of one call live on different devices (%s and %s)" % (dev, d))
+        self._ctx = None
+        if dev is not None:
+            import torch
+            self._ctx = torch.cuda.device(dev)
+
+    def __enter__(self):
+        if self._ctx is not None:
+            self._ctx.__enter__()
+        return self
+
+    def __exit__(self, *exc):
+        if self._ctx is not None:
+            return self._ctx.__exit__(*exc)
+        return False
+
+
 def fpde_fwd(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, stream=None):
     """Queue the fused forward residual + loss on `stream` (default: torch's current stream).
 
@@ -250,8 +289,9 @@ def fpde_fwd(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, b
     loss_out: fp64 CUDA tensor with nresiduals+1 entries, or None; workspace: a CUDA tensor of at
     least workspace_bytes(op, shape) bytes (uint8 or any dtype)."""
     wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
-    st = fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, wsb,
-                    _stream_handle(stream))
+    with _on_device_of(fields, sources, residuals, loss_out, workspace):
+        st = fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, wsb,
+                        _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd")
 
@@ -264,8 +304,9 @@ def fpde_fwd_bwd(op, fields, sources, residuals, gfields, loss_out, shape, spaci
     (only where has_single_pass(op); the other operators need all of them).  workspace: a CUDA
     tensor of at least fwd_bwd_workspace_bytes(op, shape) bytes."""
     wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
-    st = fwd_bwd_status(op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc, workspace,
-                        wsb, _stream_handle(stream))
+    with _on_device_of(fields, sources, residuals, gfields, loss_out, workspace):
+        st = fwd_bwd_status(op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc, workspace,
+                            wsb, _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd_bwd")
 
@@ -277,22 +318,24 @@ def workspace_bytes_f64(op, shape) -> int:
 def fpde_fwd_f64(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, stream=None):
     """fpde_fwd on fp64 CUDA tensors (verification path)."""
     wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
-    st = lib().fpde_fwd_f64(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(sources)),
-                            _ptr_array(_dev_ptrs(residuals)),
-                            _dev_ptrs([loss_out])[0] if loss_out is not None else None, len(shape), _i64(shape),
-                            _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
-                            _dev_ptrs([workspace])[0] if workspace is not None else None, int(wsb),
-                            _stream_handle(stream))
+    with _on_device_of(fields, sources, residuals, loss_out, workspace):
+        st = lib().fpde_fwd_f64(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(sources)),
+                                _ptr_array(_dev_ptrs(residuals)),
+                                _dev_ptrs([loss_out])[0] if loss_out is not None else None, len(shape), _i64(shape),
+                                _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                                _dev_ptrs([workspace])[0] if workspace is not None else None, int(wsb),
+                                _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd_f64")
 
 
 def fpde_bwd_f64(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, stream=None):
     """fpde_bwd on fp64 CUDA tensors (verification path)."""
-    st = lib().fpde_bwd_f64(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(gres)),
-                            _f64(gscale) if gscale is not None else None, _ptr_array(_dev_ptrs(gfields)),
-                            len(shape), _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
-                            _stream_handle(stream))
+    with _on_device_of(fields, gres, gfields):
+        st = lib().fpde_bwd_f64(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(gres)),
+                                _f64(gscale) if gscale is not None else None, _ptr_array(_dev_ptrs(gfields)),
+                                len(shape), _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                                _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_bwd_f64")
 
@@ -300,8 +343,9 @@ def fpde_bwd_f64(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, 
 def fpde_bwd(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace=None, stream=None):
     """Queue the gather-form adjoint (with its boundary correction) on `stream`."""
     wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
-    st = bwd_status(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace, wsb,
-                    _stream_handle(stream))
+    with _on_device_of(fields, gres, gfields, workspace):
+        st = bwd_status(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace, wsb,
+                        _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_bwd")
 
@@ -340,8 +384,9 @@ def fpde_loss_grad_host(op, h_fields, h_sources, h_gfields, h_loss, shape, spaci
     adjoint and D2H copies are queued on `stream`; synchronise it before reading the results.
     `arena` is a CUDA tensor of at least host_arena_bytes(op, shape) bytes."""
     ab = arena.numel() * arena.element_size()
-    st = loss_grad_host_status(op, h_fields, h_sources, h_gfields, h_loss, shape, spacing, coeffs, bc, arena, ab,
-                               _stream_handle(stream))
+    with _on_device_of(arena):
+        st = loss_grad_host_status(op, h_fields, h_sources, h_gfields, h_loss, shape, spacing, coeffs, bc, arena, ab,
+                                   _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_loss_grad_host")
 
@@ -363,10 +408,16 @@ def fpde_fwd_noalloc(op, fields, sources, residuals, loss_out, shape, spacing, c
     library.  Grids needing more than NOALLOC_SCRATCH_BYTES of scratch raise FpdeError (status 9).
     Calls on one device share that array, so keep them ordered on the GPU; make the first call on
     a device outside stream capture."""
-    st = fwd_noalloc_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc,
-                            _stream_handle(stream))
+    with _on_device_of(fields, sources, residuals, loss_out):
+        st = fwd_noalloc_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc,
+                                _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd_noalloc")
+
+
+def diag_ns_tma_geometry(shape, tile_rows: int, narrays: int, smem_limit: int) -> bool:
+    """Host-only: would the shared-memory-staged NS kernels take this (x,y,z,t) grid?"""
+    return bool(lib().fpde_diag_ns_tma_geometry(_i64(shape), int(tile_rows), int(narrays), int(smem_limit)))
 
 
 def diag_tma_timeouts() -> int:

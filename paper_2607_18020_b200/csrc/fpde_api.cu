@@ -533,8 +533,17 @@ static std::vector<int> host_pipe_chunks(int n0) {
     while (ib.back() < items) ib.push_back(ib.back() + 1);
     return ib;
 }
+// Per-device state of the pipelined host path, created on first use and kept until the process
+// exits: the two copy streams and a pool of timing-free events (a call needs 2K+2 of them; making
+// and destroying them on every call cost more than the launches they order).  Calls are queued
+// under the mutex, one at a time; an event recorded again by a later call does not disturb the
+// waits an earlier call queued on it (a stream wait captures the record that precedes it).
 static std::mutex g_pipe_mutex;
-static cudaStream_t g_pipe_in[64], g_pipe_out[64];
+struct HostPipeState {
+    cudaStream_t in = nullptr, out = nullptr;
+    std::vector<cudaEvent_t> events;
+};
+static HostPipeState g_pipe[64];
 
 static bool host_pipeline_wanted(int op, const int* n) {
     const char* s = std::getenv("FPDE_HOST_PIPELINE");
@@ -571,21 +580,28 @@ int fpde_host_pipeline_plan(int n0, int* planes, int cap) {
     return K;
 }
 
-static cudaError_t host_pipeline_streams(cudaStream_t* in, cudaStream_t* out) {
+// (g_pipe_mutex held)  The current device's state with at least `nevents` events in its pool.
+static cudaError_t host_pipeline_state(int nevents, HostPipeState** out) {
     int dev = 0;
     cudaError_t ce = cudaGetDevice(&dev);
     if (ce != cudaSuccess) return ce;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> lock(g_pipe_mutex);
-    if (g_pipe_in[dev] == nullptr) {
+    HostPipeState& st = g_pipe[dev];
+    if (st.in == nullptr) {
         cudaStream_t a = nullptr, b = nullptr;
         ce = cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking);
         if (ce != cudaSuccess) return ce;
         ce = cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking);
         if (ce != cudaSuccess) { cudaStreamDestroy(a); return ce; }
-        g_pipe_in[dev] = a; g_pipe_out[dev] = b;
+        st.in = a; st.out = b;
     }
-    *in = g_pipe_in[dev]; *out = g_pipe_out[dev];
+    while ((int)st.events.size() < nevents) {
+        cudaEvent_t e = nullptr;
+        ce = cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
+        if (ce != cudaSuccess) return ce;
+        st.events.push_back(e);
+    }
+    *out = &st;
     return cudaSuccess;
 }
 
@@ -593,18 +609,17 @@ static cudaError_t host_pipeline_streams(cudaStream_t* in, cudaStream_t* out) {
 static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, float* const* h_gfields, double* h_loss,
                                     float* const* d_f, float* const* d_r, float* const* d_g, double* d_loss,
                                     void* d_ws, int nf, int ne) {
-    cudaStream_t cs = q.stream, s_in = nullptr, s_out = nullptr;
-    if (host_pipeline_streams(&s_in, &s_out) != cudaSuccess) return FPDE_ERR_CUDA;
     const int n0 = q.n[0], G = HOST_PIPE_ITEM_PLANES;
     const int64_t plane = (int64_t)q.n[1] * q.n[2] * q.n[3];
     const std::vector<int> ib = host_pipe_chunks(n0);
     const int K = (int)ib.size() - 1;
-    std::vector<cudaEvent_t> ev(2 * K + 2, nullptr);
-    auto cleanup = [&]() { for (cudaEvent_t e : ev) if (e) cudaEventDestroy(e); };
-    for (auto& e : ev)
-        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cleanup(); return FPDE_ERR_CUDA; }
-    cudaEvent_t* e_in = ev.data();           // transfer c has landed
-    cudaEvent_t* e_bwd = ev.data() + K;      // gradients of chunk c are complete
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipeState* hp = nullptr;
+    if (host_pipeline_state(2 * K + 2, &hp) != cudaSuccess) { (void)cudaGetLastError(); return FPDE_ERR_CUDA; }
+    cudaStream_t cs = q.stream, s_in = hp->in, s_out = hp->out;
+    cudaEvent_t* ev = hp->events.data();
+    cudaEvent_t* e_in = ev;                  // transfer c has landed
+    cudaEvent_t* e_bwd = ev + K;             // gradients of chunk c are complete
     cudaEvent_t e_start = ev[2 * K], e_done = ev[2 * K + 1];
     bool ok = true;
     auto chk = [&](cudaError_t ce) { ok = ok && ce == cudaSuccess; };
@@ -668,7 +683,6 @@ static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, flo
     // the caller's stream covers the copy streams
     chk(cudaEventRecord(e_done, s_out));
     chk(cudaStreamWaitEvent(cs, e_done, 0));
-    cleanup();
     return ok ? FPDE_OK : FPDE_ERR_CUDA;
 }
 
@@ -779,5 +793,15 @@ int fpde_fwd_noalloc(int op, const float* const* fields, const float* const* sou
 }
 
 unsigned int fpde_diag_tma_timeouts(void) { return ns_tma_timeouts(); }
+
+int fpde_diag_ns_tma_geometry(const int64_t* shape, int tile_rows, int narrays, size_t smem_limit) {
+    if (!shape) return 0;
+    int n[MAX_D];
+    for (int a = 0; a < 4; ++a) {
+        if (shape[a] < 1 || shape[a] > (int64_t)1 << 30) return 0;
+        n[a] = (int)shape[a];
+    }
+    return ns_tma_geometry_ok(n, tile_rows, narrays, smem_limit) ? 1 : 0;
+}
 
 }  // extern "C"

@@ -107,6 +107,7 @@ cudaError_t launch_ns3d_bwd(const Problem& p);
 cudaError_t launch_ns_fwd(const Problem& p);
 // TMA-staged variants (op_ns3dt_tma.cu); `launched` false = this grid is not eligible
 bool ns_tma_wanted(const int* n);
+bool ns_tma_geometry_ok(const int* n, int ty, int na, size_t smem_limit);
 int ns_tma_items(const int* n);
 cudaError_t launch_ns_fwd_tma(const Problem& p, bool& launched);
 cudaError_t launch_ns_bwd_tma(const Problem& p, bool& launched);

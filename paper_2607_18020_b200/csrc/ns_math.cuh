@@ -5,7 +5,7 @@
 // Forward (Section 2.1 extended by d_t, w, d_z), per momentum component q along axis a_q:
 //   mom_q = d_t q + u d_x q + v d_y q + w d_z q + d_{a_q} p - nu (d_xx + d_yy + d_zz) q
 //   cont  = d_x u + d_y v + d_z w
-// Adjoint (Eq. 1 / Appendix A.2 extended the same way), G = upstream arrays (zero at the first
+// Adjoint (Eq. 1 / Appendix A.3 extended the same way), G = upstream arrays (zero at the first
 // and last t), c = (u,v,w):
 //   g_q(P) = sum_e G_e(P) (d_{a_q} e)(P)                                   local terms
 //          + sum_a [ (G_q c_a)(P-a) - (G_q c_a)(P+a) ] / (2 h_a)           transposed advection

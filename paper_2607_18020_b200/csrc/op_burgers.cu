@@ -2,7 +2,7 @@
 // centred second-order differences inside and second-order one-sided differences on the first
 // and last node of each axis (per axis).  Forward (Section 2.1) and gather-form adjoint with
 // its boundary-gradient correction (Sections 2.2, 2.3): this is the operator whose correction
-// terms come from one-sided formulas (Appendix A.4), not merely from omitted neighbours.
+// terms come from one-sided formulas (Appendix A.5), not merely from omitted neighbours.
 //
 // Adjoint:  g = D_t^T G + (D_x u) . G + D_x^T (u . G) - nu D_xx^T G.
 // A transposed difference matrix acts on w as

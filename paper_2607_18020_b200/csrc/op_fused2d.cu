@@ -15,7 +15,7 @@
 // A chunk of rows recomputes r on one row above and below itself.
 //
 // Boundary handling is the zero extension of r outside the rows of the operator (omitted
-// neighbours, Appendix A.4): on interior axes r is forced to 0 on the outer ring and outside
+// neighbours, Appendix A.5): on interior axes r is forced to 0 on the outer ring and outside
 // the array, on periodic axes row and column indices wrap.
 //
 // Field rows are requested one step before they are first used (five-slot rotation, unrolled).

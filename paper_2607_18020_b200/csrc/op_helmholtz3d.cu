@@ -3,7 +3,7 @@
 // 2.1) and the gather-form adjoint with its two-cell boundary band (Sections 2.2, 2.3).
 //
 // The Jacobian is constant and the star is symmetric, so the adjoint is the same star applied
-// to the upstream array treated as zero outside the rows (omitted neighbours, Appendix A.4);
+// to the upstream array treated as zero outside the rows (omitted neighbours, Appendix A.5);
 // that one rule produces the gradient of the two outer layers and the truncated sums of layers
 // 2 and 3.  Forward and adjoint are therefore two instances of one 2.5-D engine:
 //

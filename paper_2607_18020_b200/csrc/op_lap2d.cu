@@ -15,7 +15,7 @@
 //
 // The five-point sum is formed as ih0*((up+dn) - 2c) + ih1*((l+r) - 2c).
 //
-// Boundary handling (Section 2.3 / Appendix A.4) is part of the same launch:
+// Boundary handling (Section 2.3 / Appendix A.5) is part of the same launch:
 //   periodic axes   - row and column indices wrap;
 //   interior axes   - forward: nodes of the outer ring carry no row and get 0;
 //                     adjoint: the upstream array is treated as 0 outside the rows (omitted

@@ -1,5 +1,5 @@
 // Steady incompressible Navier-Stokes on an (x,y) array: the operator the paper works through
-// (Section 2.1 residuals, Eq. 1 / Appendix A.2 adjoint, Appendix A.3 pseudocode).
+// (Section 2.1 residuals, Eq. 1 / Appendix A.3 adjoint, Appendix A.4 pseudocode).
 //   res_u = u u_x + v u_y + p_x - nu (u_xx + u_yy)
 //   res_v = u v_x + v v_y + p_y - nu (v_xx + v_yy)
 //   res_div = u_x + v_y

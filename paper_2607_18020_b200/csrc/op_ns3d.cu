@@ -6,7 +6,7 @@
 //   mom_q = u d_x q + v d_y q + w d_z q + d_{a_q} p - nu (d_xx + d_yy + d_zz) q     q in (u,v,w)
 //   cont  = d_x u + d_y v + d_z w
 //
-// The adjoint is Eq. (1) / Appendix A.2 extended the same way (ns_math.cuh writes it out); the
+// The adjoint is Eq. (1) / Appendix A.3 extended the same way (ns_math.cuh writes it out); the
 // boundary-gradient correction of Section 2.3 is the zero extension of the upstream arrays
 // outside the rows: a shell node receives only the terms of the interior rows that read it, an
 // interior node next to the shell loses the terms of the rows that do not exist.

@@ -1,7 +1,7 @@
 // Unsteady incompressible Navier-Stokes on an (x,y,z,t) array (t contiguous), space periodic,
 // rows at interior t: four residuals (momentum x,y,z and continuity) from four fields
 // (u,v,w,p).  This is Section 2.1's steady 2-D system extended by d_t, w and d_z; the adjoint
-// below is Eq. (1) / Appendix A.2 extended the same way (drop w, z and t and it is the printed
+// below is Eq. (1) / Appendix A.3 extended the same way (drop w, z and t and it is the printed
 // u-gradient term by term).
 //
 // Memory view: (x, y, row) with row = (z,t) flattened, n2*n3 contiguous floats.  Along a row,
@@ -17,7 +17,7 @@
 // the large centre value.
 //
 // Nodes at the first / last t carry no row: the forward pass writes 0 there; in the adjoint the
-// upstream arrays count as 0 there (omitted neighbours, Appendix A.4).  Every spatial read of an
+// upstream arrays count as 0 there (omitted neighbours, Appendix A.5).  Every spatial read of an
 // output node happens at the node's own t, so that rule only changes (i) the t-neighbour of the
 // nodes next to the two end planes and (ii) the end planes themselves, where only the
 // transposed d_t term survives: that is the boundary-gradient correction of this operator, and

@@ -291,22 +291,51 @@ static int env_int(const char* name, int dflt) {
     return v >= 0 ? v : dflt;
 }
 
-// Can the TMA-staged kernels take this grid?  (exact tiling, t groups aligned to lanes, 128-byte
-// aligned halo regions; anything else runs on the L1-staged kernels)
 // rows per tile: 8 when the grid allows it (fewer, larger boxes and less halo per byte), else 4
 static int ns_tma_ty(const int* n) {
     const int want = env_int("FPDE_NS_TMA_TY", 4);
     return (want >= 8 && n[1] % 8 == 0) ? 8 : 4;
 }
 
+// Dynamic shared memory of a launch with `na` arrays per stage.
+static size_t ns_tma_smem_bytes(const int* n, int ty, int na) {
+    const size_t slot = (size_t)(4 * NS_TMA_TX + 2 * n[3]) * (ty + 2);
+    return (size_t)NS_TMA_STAGES * na * slot * 4 + 128;
+}
+
+// Pure geometry: can a kernel with tiles of `ty` rows and `na` arrays per stage take this grid
+// within `smem_limit` bytes of dynamic shared memory?  Exact tiling; t groups aligned to lanes;
+// every bulk-copy destination (array slot, stage) on a 128-byte boundary, which the copy engine
+// requires -- the slot is (128 + 2 n_t)(ty + 2) floats, a multiple of 32 floats only when n_t is
+// a multiple of 8 for the even tile heights used here; the stage ring within the limit.
+bool ns_tma_geometry_ok(const int* n, int ty, int na, size_t smem_limit) {
+    const int n3 = n[3], C = n[2] * n[3], nt4 = n3 / 4;
+    if (n3 % 4 != 0 || nt4 < 1 || 32 % nt4 != 0) return false;
+    if (ty < 1 || n[1] % ty != 0 || C % (4 * NS_TMA_TX) != 0) return false;
+    if ((ty * n3) % 32 != 0 || n3 > 64) return false;      // n3 <= 64: the one-box tile fits 256 elements
+    const size_t slot_bytes = (size_t)(4 * NS_TMA_TX + 2 * n3) * (ty + 2) * 4;
+    if (slot_bytes % 128 != 0 || (na * slot_bytes) % 128 != 0) return false;
+    return ns_tma_smem_bytes(n, ty, na) <= smem_limit;
+}
+
+static size_t smem_optin_limit() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return (size_t)v;
+}
+
+// Can the TMA-staged kernels take this grid?  Both directions must fit (forward: 4 arrays per
+// stage, adjoint: 7), because the loss workspace is sized for one launch shape per grid; anything
+// else runs on the L1-staged kernels.
 static bool ns_tma_applicable(const int* n) {
     if (env_int("FPDE_NS_TMA", 0) == 0 || encode_fn() == nullptr) return false;
-    const int n3 = n[3], C = n[2] * n[3], nt4 = n3 / 4;
-    if (nt4 < 1 || 32 % nt4 != 0) return false;
     const int ty = ns_tma_ty(n);
-    if (n[1] % ty != 0 || C % (4 * NS_TMA_TX) != 0) return false;
-    if ((ty * n3) % 32 != 0 || n3 > 64) return false;      // n3 <= 64: the one-box tile fits 256 elements
-    return true;
+    const size_t limit = smem_optin_limit();
+    return ns_tma_geometry_ok(n, ty, 4, limit) && ns_tma_geometry_ok(n, ty, 7, limit);
 }
 
 template <int NA, bool FWD, int TY, int MINB>
@@ -334,8 +363,7 @@ static cudaError_t launch_tma(const Problem& q, const float* const* arrays, cons
     p.nmb = p.n1 / TY;
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     p.partials = FWD ? q.partials : nullptr;
-    const int slot = (TXF + 2 * p.n3) * (TY + 2);
-    const size_t smem = (size_t)NS_TMA_STAGES * NA * slot * 4 + 128;
+    const size_t smem = ns_tma_smem_bytes(q.n, TY, NA);
     auto kern = ns_tma_kernel<NA, FWD, TY, MINB>;
     cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ce != cudaSuccess) return ce;

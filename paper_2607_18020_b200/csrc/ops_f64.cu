@@ -6,7 +6,7 @@
 //
 // Conventions.  A node carries a residual row iff on every INTERIOR axis its index lies in
 // [radius, n-1-radius].  The adjoint reads the upstream arrays through G(), which returns 0 at
-// nodes without a row and outside the array (omitted neighbours, Appendix A.4); with that rule
+// nodes without a row and outside the array (omitted neighbours, Appendix A.5); with that rule
 // the gather formulas below hold at every node, boundary layers included (Section 2.3).
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
@@ -267,7 +267,7 @@ __device__ void adjoint_at(const F64Params& p, const Node& q, double* g) {
         g[0] = G_d2o4(p, 0, q, 0) + G_d2o4(p, 0, q, 1) + G_d2o4(p, 0, q, 2) + p.coef[0] * p.coef[0] * G(p, 0, q, 0, 0);
         break;
     default: {
-        // Eq. (1) / Appendix A.2 and their extension by w, d_z and d_t:
+        // Eq. (1) / Appendix A.3 and their extension by w, d_z and d_t:
         //   g_c = sum_e G_e d_c(e)  +  sum_a D_a^T (u_a G_c)  -  nu sum_a D_aa G_c  +  D_t^T G_c  +  D_c^T G_div
         //   g_p = sum_c D_c^T G_c
         double gp = 0.0;

@@ -192,3 +192,28 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     with pytest.raises(RuntimeError, match="no fallback"):
         B.lib()
+
+
+def test_ns_tma_geometry_predicate_requires_aligned_slots_and_a_ring_that_fits():
+    """The shared-memory-staged NS kernels copy each array's tile to `slot`-sized regions of a stage;
+    the copy engine needs every region on a 128-byte boundary.  slot = (128 + 2 n_t)(rows + 2)
+    floats, so the rule is checked here from that formula, independently of the library."""
+    limit = 227 * 1024
+    for ty in (4, 8):
+        for nt in (4, 8, 16, 32, 64):
+            for na in (4, 7):
+                shape = (16, 32, 64, nt)
+                slot_bytes = (128 + 2 * nt) * (ty + 2) * 4
+                ring = 4 * na * slot_bytes + 128
+                lanes_ok = (ty * nt) % 32 == 0 and 32 % (nt // 4) == 0
+                want = lanes_ok and slot_bytes % 128 == 0 and (na * slot_bytes) % 128 == 0 and ring <= limit
+                got = B.diag_ns_tma_geometry(shape, ty, na, limit)
+                assert got == want, (ty, nt, na, slot_bytes, ring)
+    # the case that used to pass the gate with 64-byte-aligned slots
+    assert not B.diag_ns_tma_geometry((16, 32, 64, 4), 8, 4, limit)
+    # the adjoint ring of the widest t extent does not fit, the forward ring does
+    assert B.diag_ns_tma_geometry((16, 32, 64, 64), 8, 4, limit)
+    assert not B.diag_ns_tma_geometry((16, 32, 64, 64), 8, 7, limit)
+    # rows that do not tile, t extent beyond the one-box limit
+    assert not B.diag_ns_tma_geometry((16, 30, 64, 16), 4, 4, limit)
+    assert not B.diag_ns_tma_geometry((16, 32, 64, 128), 4, 4, limit)

@@ -7,12 +7,14 @@
   * convergence order on manufactured smooth fields (2nd order, 4th for Helmholtz);
   * the adjoint identity <J du, w> = <du, J^T w>, with J du obtained from the forward only;
   * brute-force central finite differences of the loss on tiny grids;
-  * the paper's printed u-adjoint of steady 2-D Navier-Stokes (Eq. 1 / Appendix A.2), to which
+  * the paper's printed u-adjoint of steady 2-D Navier-Stokes (Eq. 1 / Appendix A.3), to which
     the 3-D unsteady operator must reduce for fields constant in z and t;
   * special cases and symmetries; two hand-worked fixtures under tests/golden/.
 """
 import math
 import os
+
+import zlib
 
 import numpy as np
 import pytest
@@ -306,7 +308,7 @@ CASES = [
 
 def _rand_problem(op, shape):
     nf = len(W.OP_META[op]["fields"]); ns = len(W.OP_META[op]["sources"]); ne = len(W.OP_META[op]["residuals"])
-    r = np.random.default_rng(hash(op) % 1000 + 5)
+    r = np.random.default_rng(zlib.crc32(op.encode()) % 1000 + 5)   # fixed per operator: the cases repeat run to run
     F = [r.standard_normal(shape) for _ in range(nf)]
     S = [r.standard_normal(shape) for _ in range(ns)]
     dF = [r.standard_normal(shape) for _ in range(nf)]

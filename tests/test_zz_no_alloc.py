@@ -40,7 +40,27 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
         ref, got, lr, lg = _both(w)
         for e, (a, b) in enumerate(zip(got, ref)):
             assert_close(a.cpu().numpy(), b.cpu().numpy().astype(np.float64), "%s residual %d" % (name, e))
+            # same kernels, same slots of partial sums, only the scratch differs: every bit agrees
+            assert torch.equal(a, b), "%s residual %d differs from fpde_fwd" % (name, e)
         assert np.all(np.abs(lg - lr) <= LOSS_TOL * np.abs(lr)), (lg, lr)
+        assert np.array_equal(lg, lr), (lg, lr)
+
+
+def test_noalloc_against_the_oracle_and_without_a_loss():
+    import oracle
+    w = W.make("ns_tgv_128x16", seed=45, shape=(12, 8, 8, 8))
+    _, got, _, lg = _both(w)
+    res, loss, _ = oracle.fwd(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    for e, a in enumerate(got):
+        assert_close(a.cpu().numpy(), res[e], "residual %d vs oracle" % e)
+    assert np.all(np.abs(lg - loss) <= LOSS_TOL * np.abs(loss)), (lg, loss)
+    # no loss asked for: no scratch is touched, the residuals are the same
+    fields = [torch.from_numpy(f).cuda() for f in w.fields]
+    again = [torch.full(w.shape, 5.0, dtype=torch.float32, device="cuda") for _ in got]
+    B.fpde_fwd_noalloc(w.op, fields, [], again, None, w.shape, w.spacing, w.coeffs, w.bc)
+    torch.cuda.synchronize()
+    for a, b in zip(again, got):
+        assert torch.equal(a, b)
 
 
 def test_noalloc_refuses_grids_beyond_its_scratch():
