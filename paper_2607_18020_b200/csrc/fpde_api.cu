@@ -248,7 +248,7 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     case FPDE_OP_POISSON_2D:
     case FPDE_OP_GRAYSCOTT_2D:
     case FPDE_OP_GRAYSCOTT_2D_XSLAB: ce = launch_lap2d_fwd(q); items = lap2d_items(q.n); break;
-    case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q); items = star3d_items(q.n); break;
+    case FPDE_OP_HELMHOLTZ_3D_O4: ce = launch_helmholtz_fwd(q, &items); break;
     case FPDE_OP_NS_3D_T: ce = launch_ns_fwd(q); items = ns_items(q.n, false); break;
     case FPDE_OP_NS_3D_T_XSLAB: ce = launch_ns_fwd(q); items = ns_items(q.n, true); break;
     case FPDE_OP_NS_2D_STEADY: ce = launch_ns2d_fwd(q); items = ns2d_items(q.n); break;
@@ -792,7 +792,10 @@ int fpde_fwd_noalloc(int op, const float* const* fields, const float* const* sou
                     scratch, scratch ? (size_t)FPDE_NOALLOC_SCRATCH_BYTES : 0, stream);
 }
 
-unsigned int fpde_diag_tma_timeouts(void) { return ns_tma_timeouts(); }
+unsigned int fpde_diag_tma_timeouts(void) {
+    const unsigned int a = ns_tma_timeouts(), b = star3d_tma_timeouts();
+    return (a == ~0u || b == ~0u) ? ~0u : a + b;
+}
 
 int fpde_diag_ns_tma_geometry(const int64_t* shape, int tile_rows, int narrays, size_t smem_limit) {
     if (!shape) return 0;

@@ -98,13 +98,19 @@ cudaError_t launch_burgers_fwd(const Problem& p);
 cudaError_t launch_burgers_bwd(const Problem& p);
 cudaError_t launch_lap2d_fwd(const Problem& p);     // Poisson 2-D and Gray-Scott
 cudaError_t launch_lap2d_bwd(const Problem& p);
-cudaError_t launch_helmholtz_fwd(const Problem& p);
+cudaError_t launch_helmholtz_fwd(const Problem& p, int* items);   // *items: loss partial sums written
 cudaError_t launch_helmholtz_bwd(const Problem& p);
 cudaError_t launch_ns2d_fwd(const Problem& p);    // steady 2-D Navier-Stokes
 cudaError_t launch_ns2d_bwd(const Problem& p);
 cudaError_t launch_ns3d_fwd(const Problem& p);    // steady 3-D Navier-Stokes
 cudaError_t launch_ns3d_bwd(const Problem& p);
 cudaError_t launch_ns_fwd(const Problem& p);
+// Helmholtz engine staged through shared memory by the copy engine (op_helmholtz3d_tma.cu);
+// `launched` false = this grid runs on the L1-staged engine
+bool star3d_tma_wanted(const int* n);
+int star3d_tma_items(const int* n);
+cudaError_t launch_star3d_tma(const Problem& p, int mode, int* items, bool& launched);
+unsigned int star3d_tma_timeouts();
 // TMA-staged variants (op_ns3dt_tma.cu); `launched` false = this grid is not eligible
 bool ns_tma_wanted(const int* n);
 bool ns_tma_geometry_ok(const int* n, int ty, int na, size_t smem_limit);

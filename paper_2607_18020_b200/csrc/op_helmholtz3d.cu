@@ -247,11 +247,18 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     if (p.prefetch < 0) p.prefetch = 0;
 }
 
-int star3d_items(const int* n) {
+static int star3d_l1_items(const int* n) {
     Problem q{}; q.n[0] = n[0]; q.n[1] = n[1]; q.n[2] = n[2]; q.h[0] = q.h[1] = q.h[2] = 1.0;
     Star3dParams p{}; dim3 block;
     star3d_geometry(q, p, block, 1.0, true);
     return p.nitems;
+}
+
+// Loss partial sums a forward launch may write: the larger of the two engines' item counts (which
+// engine runs is decided per launch; the launcher reports the count it used).
+int star3d_items(const int* n) {
+    const int l1 = star3d_l1_items(n);
+    return star3d_tma_wanted(n) ? std::max(l1, star3d_tma_items(n)) : l1;
 }
 
 // 32-bit byte offsets when every array is below 4 GiB (FPDE_STAR3D_OFF32=0 forces the 64-bit form)
@@ -263,15 +270,22 @@ static cudaError_t star3d_launch(const Problem& q, const Star3dParams& p, dim3 b
     return launch_kernel(star3d_kernel<MODE, 4, false>, dim3(p.nitems), block, q.stream, p);
 }
 
-cudaError_t launch_helmholtz_fwd(const Problem& q) {
+cudaError_t launch_helmholtz_fwd(const Problem& q, int* items) {
+    bool launched = false;
+    cudaError_t ce = launch_star3d_tma(q, 0, items, launched);
+    if (launched || ce != cudaSuccess) return ce;
     Star3dParams p{}; dim3 block;
     star3d_geometry(q, p, block, 1.0, true);
     p.hin = q.in[0]; p.cin = q.aux[0]; p.out = q.out[0];
     p.partials = q.partials;
+    if (items) *items = p.nitems;
     return star3d_launch<0>(q, p, block);
 }
 
 cudaError_t launch_helmholtz_bwd(const Problem& q) {
+    bool launched = false;
+    cudaError_t ce = launch_star3d_tma(q, q.gres_zero_off_rows ? 2 : 1, nullptr, launched);
+    if (launched || ce != cudaSuccess) return ce;
     Star3dParams p{}; dim3 block;
     star3d_geometry(q, p, block, q.gscale[0], false);      // the operator is linear: the scale goes into the weights
     p.hin = q.aux[0]; p.cin = nullptr; p.out = q.out[0];

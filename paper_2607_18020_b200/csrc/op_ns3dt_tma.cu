@@ -27,11 +27,10 @@
 //
 // Every wait on an mbarrier is bounded: after the limit the kernel counts a timeout in a global
 // word and carries on with whatever is in shared memory, so it always terminates.
-#include <cuda.h>
-
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
 #include "ns_math.cuh"
+#include "tma_common.cuh"
 
 #include <algorithm>
 #include <cstdlib>
@@ -58,46 +57,6 @@ struct NsTmaParams {
 
 __device__ unsigned int g_ns_tma_timeouts = 0;   // number of bounded waits that gave up (0 in a healthy run)
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the phase with the given parity to complete.  A thread that has given up once
-// (`gave_up`) does not wait again, so a broken pipeline costs one bounded wait per thread, not one
-// per step.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, bool& gave_up) {
-    if (gave_up) return;
-    for (int it = 0; it < (1 << 16); ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return;
-    }
-    gave_up = true;
-    atomicAdd(&g_ns_tma_timeouts, 1u);
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
-}
-__device__ __forceinline__ V4 ldsv4(uint32_t addr) {
-    float4 t;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "r"(addr));
-    V4 v; v.lo = make_float2(t.x, t.y); v.hi = make_float2(t.z, t.w);
-    return v;
-}
 __device__ __forceinline__ int wrapn(int i, int n) { return i < 0 ? i + n : (i >= n ? i - n : i); }
 
 template <int NA, bool FWD, int TY, int MINB>
@@ -135,8 +94,7 @@ ns_tma_kernel(const __grid_constant__ NsTmaParams<NA> p) {
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < ST; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, TY); }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_fence_init();
     }
     __syncthreads();
     pdl_wait_then_trigger();          // nothing of the previous kernel's output is read before this
@@ -148,7 +106,7 @@ ns_tma_kernel(const __grid_constant__ NsTmaParams<NA> p) {
     auto issue = [&](int seq) {
         const int stage = seq & (ST - 1);
         const uint32_t fb = full0 + 8u * stage;
-        if (seq >= ST) mbar_wait(empty0 + 8u * stage, (uint32_t)(((seq / ST) - 1) & 1), gave_up);
+        if (seq >= ST) mbar_wait(empty0 + 8u * stage, (uint32_t)(((seq / ST) - 1) & 1), gave_up, &g_ns_tma_timeouts);
         const int pl = wrapn(a0 + seq, n0);
         const uint32_t sb = base + (uint32_t)stage * stage_bytes;
         if (tx == 0) mbar_expect_tx(fb, fill_bytes);
@@ -194,7 +152,7 @@ ns_tma_kernel(const __grid_constant__ NsTmaParams<NA> p) {
 #pragma unroll
         for (int k = 0; k < NA; ++k) A[k] = ldv4(p.arr[k] + om);
     }
-    mbar_wait(full0, 0, gave_up);
+    mbar_wait(full0, 0, gave_up, &g_ns_tma_timeouts);
 #pragma unroll
     for (int k = 0; k < NA; ++k) B[k] = ldsv4(base + (uint32_t)(k * SLOT) * 4u + o_own);
 
@@ -205,7 +163,7 @@ ns_tma_kernel(const __grid_constant__ NsTmaParams<NA> p) {
     // step s: plane a0+s from stage S0 (neighbours), plane a0+s+1 from stage S1 (own column -> W2)
     auto step = [&](int s, const V4 (&W0)[NA], const V4 (&W1)[NA], V4 (&W2)[NA]) {
         const int S0 = s & (ST - 1), S1 = (s + 1) & (ST - 1);
-        mbar_wait(full0 + 8u * S1, (uint32_t)(((s + 1) / ST) & 1), gave_up);
+        mbar_wait(full0 + 8u * S1, (uint32_t)(((s + 1) / ST) & 1), gave_up, &g_ns_tma_timeouts);
         const uint32_t b0 = base + (uint32_t)S0 * stage_bytes, b1 = base + (uint32_t)S1 * stage_bytes;
         V4 Ym[NA], Yp[NA], Zm[NA], Zp[NA];
 #pragma unroll
@@ -255,33 +213,8 @@ ns_tma_kernel(const __grid_constant__ NsTmaParams<NA> p) {
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static std::once_flag once;
-    static EncodeTiledFn fn = nullptr;
-    std::call_once(once, [] {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(f);
-        else
-            (void)cudaGetLastError();
-    });
-    return fn;
-}
-
 static bool encode_box(CUtensorMap* m, const float* ptr, int C, int n1, int n0, int bx, int by) {
-    const cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)n1, (cuuint64_t)n0};
-    const cuuint64_t strides[2] = {(cuuint64_t)C * 4u, (cuuint64_t)C * (cuuint64_t)n1 * 4u};
-    const cuuint32_t box[3] = {(cuuint32_t)bx, (cuuint32_t)by, 1u};
-    const cuuint32_t estr[3] = {1u, 1u, 1u};
-    return encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(ptr), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tma_encode_3d(m, ptr, C, n1, n0, C, (long long)C * n1, bx, by);
 }
 
 static int env_int(const char* name, int dflt) {
@@ -332,7 +265,7 @@ static size_t smem_optin_limit() {
 // stage, adjoint: 7), because the loss workspace is sized for one launch shape per grid; anything
 // else runs on the L1-staged kernels.
 static bool ns_tma_applicable(const int* n) {
-    if (env_int("FPDE_NS_TMA", 0) == 0 || encode_fn() == nullptr) return false;
+    if (env_int("FPDE_NS_TMA", 0) == 0 || tma_encode_fn() == nullptr) return false;
     const int ty = ns_tma_ty(n);
     const size_t limit = smem_optin_limit();
     return ns_tma_geometry_ok(n, ty, 4, limit) && ns_tma_geometry_ok(n, ty, 7, limit);

@@ -1,0 +1,109 @@
+// Helpers of the kernels that stage their tiles through shared memory with the copy engine
+// (cp.async.bulk.tensor, no multicast): mbarrier primitives with bounded waits, the tiled bulk
+// load, 64- and 128-bit shared-memory loads, and the host-side tensor-map encoder.
+//
+// Every wait on an mbarrier is bounded: after the limit the waiting thread counts a timeout in a
+// global word of its translation unit and carries on with whatever is in shared memory, so a
+// kernel always terminates and the host can see that its results are not to be trusted.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "fpde_common.cuh"
+
+namespace fpde {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// Bounded wait for the phase with the given parity to complete.  A thread that has given up once
+// (`gave_up`) does not wait again, so a broken pipeline costs one bounded wait per thread, not one
+// per step.  `timeouts` is the translation unit's counter.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, bool& gave_up, unsigned int* timeouts) {
+    if (gave_up) return;
+    for (int it = 0; it < (1 << 16); ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return;
+    }
+    gave_up = true;
+    atomicAdd(timeouts, 1u);
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+__device__ __forceinline__ V4 ldsv4(uint32_t addr) {
+    float4 t;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "r"(addr));
+    V4 v; v.lo = make_float2(t.x, t.y); v.hi = make_float2(t.z, t.w);
+    return v;
+}
+__device__ __forceinline__ float2 ldsv2(uint32_t addr) {
+    float2 t;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(t.x), "=f"(t.y) : "r"(addr));
+    return t;
+}
+__device__ __forceinline__ void stsv4(uint32_t addr, const V4& v) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.lo.x), "f"(v.lo.y), "f"(v.hi.x), "f"(v.hi.y) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// host side: cuTensorMapEncodeTiled through the runtime's driver entry point (no -lcuda)
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn tma_encode_fn() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+        else
+            (void)cudaGetLastError();
+    });
+    return fn;
+}
+
+// fp32 array of extents (d0 contiguous, d1, d2) with the strides of a dense (.., s1, s0) array:
+// boxes of bx x by x 1 elements; reads outside the extents give 0.
+inline bool tma_encode_3d(CUtensorMap* m, const float* ptr, long long d0, long long d1, long long d2,
+                          long long stride1_elems, long long stride2_elems, int bx, int by) {
+    EncodeTiledFn fn = tma_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)d0, (cuuint64_t)d1, (cuuint64_t)d2};
+    const cuuint64_t strides[2] = {(cuuint64_t)stride1_elems * 4u, (cuuint64_t)stride2_elems * 4u};
+    const cuuint32_t box[3] = {(cuuint32_t)bx, (cuuint32_t)by, 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace fpde

@@ -282,3 +282,36 @@ def test_ns_adjoint_on_smooth_fields_at_fine_spacing(name, shape, cells):
     grads = run_bwd(torch, w, fields, [r.view for r in res], [2.0 / rows] * len(res))
     for k, g in enumerate(grads):
         assert_close(g.view.cpu().numpy(), g_ref[k], "%s smooth gradient %d (2 pi / %d)" % (name, k, cells))
+
+
+@pytest.mark.parametrize("shape", [(20, 40, 136), (9, 45, 260), (37, 72, 256), (12, 130, 392)])
+@pytest.mark.parametrize("engine", ["l1", "tma", "tma_fwd"])
+def test_helmholtz_engines_agree_with_oracle(shape, engine, monkeypatch):
+    """The Helmholtz operator has two engines: plane tiles staged through L1 and registers, and plane
+    tiles staged through shared memory by the copy engine (default for the adjoint; the forward pass
+    with FPDE_STAR3D_TMA_FWD=1).  Shapes with ragged tiles in y and z, grids of fewer tile-planes than
+    CTAs would take and grids where one CTA's share spans two tiles; forward, the adjoint of the
+    residuals (through both entry points) and the adjoint of an arbitrary upstream array."""
+    monkeypatch.setenv("FPDE_STAR3D_TMA", "0" if engine == "l1" else "1")
+    monkeypatch.setenv("FPDE_STAR3D_TMA_FWD", "1" if engine == "tma_fwd" else "0")
+    w = W.make("helmholtz_256", seed=47, shape=shape, kind="randn")
+    _check_case(w, "helmholtz %s engine %s" % (shape, engine))
+    # arbitrary upstream array with entries off the rows, and the one-call entry point
+    rng = np.random.default_rng(5)
+    G = rng.standard_normal(shape).astype(np.float32)
+    Gz = G.astype(np.float64).copy()
+    Gz[:2] = 0; Gz[-2:] = 0; Gz[:, :2] = 0; Gz[:, -2:] = 0; Gz[:, :, :2] = 0; Gz[:, :, -2:] = 0
+    g_ref = oracle.bwd(w.op, w.fields, [0.37 * Gz], w.shape, w.spacing, w.coeffs)
+    fields = to_dev(torch, w.fields)
+    grads = run_bwd(torch, w, fields, to_dev(torch, [G]), [0.37])
+    assert_close(grads[0].view.cpu().numpy(), g_ref[0], "helmholtz %s engine %s arbitrary upstream" % (shape, engine))
+    _, loss_ref, g2_ref, _ = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    res = [torch.empty(shape, dtype=torch.float32, device="cuda")]
+    gr = [torch.empty(shape, dtype=torch.float32, device="cuda")]
+    loss = torch.zeros(2, dtype=torch.float64, device="cuda")
+    ws = torch.empty(B.fwd_bwd_workspace_bytes(w.op, shape), dtype=torch.uint8, device="cuda")
+    B.fpde_fwd_bwd(w.op, fields, to_dev(torch, w.sources), res, gr, loss, shape, w.spacing, w.coeffs, w.bc, ws)
+    torch.cuda.synchronize()
+    assert_close(gr[0].cpu().numpy(), g2_ref[0], "helmholtz %s engine %s one call" % (shape, engine))
+    assert abs(loss[-1].item() - loss_ref[-1]) <= 1e-5 * abs(loss_ref[-1])
+    assert B.diag_tma_timeouts() == 0
