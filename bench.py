@@ -74,6 +74,7 @@ NCU_TRAFFIC_BYTES = {
     ("ns2d_steady_4096", "fused2d_kernel<ns_2d_steady>"): 372255488,
 }
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0            # the vendor figure the workload text quotes; fractions of it go beside the measured ones
 LAUNCHES_PER_STEP = 3               # forward kernel, loss finalise, adjoint kernel
 
 
@@ -98,7 +99,7 @@ class ClockSampler:
     test by ~7 %."""
 
     def __init__(self, torch, device_index: int, period_s: float = 0.025):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.stamps, self.reasons, self.max_mhz = [], [], set(), None
         self.period = period_s
         self._stop = threading.Event()
         self._thread = None
@@ -119,6 +120,7 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.stamps.append(time.perf_counter())
                 try:
                     mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
                 except Exception:
@@ -139,6 +141,16 @@ class ClockSampler:
         if self._thread is not None:
             self._stop.set()
             self._thread.join()
+
+    def mhz_between(self, t0: float, t1: float):
+        """Median SM clock of the samples taken in [t0, t1] (host clock), else the sample nearest to it."""
+        inside = [m for m, t in zip(self.samples, self.stamps) if t0 <= t <= t1]
+        if inside:
+            return statistics.median(inside)
+        if not self.samples:
+            return None
+        mid = 0.5 * (t0 + t1)
+        return min(zip(self.samples, self.stamps), key=lambda p: abs(p[1] - mid))[0]
 
     def summary(self):
         if self._h is None:
@@ -178,17 +190,63 @@ def time_oracle(w, reps: int):
     return best
 
 
+def _oracle_worker(args):
+    """One worker of the all-cores leg: the oracle, as it stands, on this worker's own sample (the
+    first `planes` slices of the workload's recipe under the worker's own seed)."""
+    name, planes, seed, reps, t_go = args
+    w = oracle_sample(name, planes, seed=seed)
+    import oracle
+    oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)      # warm-up: page-in, library load
+    while time.time() < t_go:                       # all workers start their timed passes together
+        time.sleep(0.001)
+    t0 = time.time()
+    for _ in range(reps):
+        oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    return t0, time.time(), w.npoints * reps
+
+
+def cpu_baseline_all_cores(name: str, planes_per_worker: int, reps: int = 2):
+    """P = os.cpu_count() processes, each running the single-thread oracle on its own sample at the
+    same time; aggregate points per second over the window from the first start to the last end."""
+    import multiprocessing as mp
+    P = os.cpu_count() or 1
+    n0 = W.CONFIGS[name]["shape"][0]
+    planes = max(5, min(planes_per_worker, n0))
+    ctx = mp.get_context("spawn")
+    t_go = time.time() + 8.0                        # imports, sample generation and the warm-up pass come first
+    with ctx.Pool(P) as pool:
+        out = pool.map(_oracle_worker, [(name, planes, 1042 + i, reps, t_go) for i in range(P)], chunksize=1)
+    t_first, t_last = min(o[0] for o in out), max(o[1] for o in out)
+    pts = sum(o[2] for o in out)
+    late = sum(1 for o in out if o[0] > t_go + 0.5)
+    return {"value": pts / (t_last - t_first), "cores": P, "planes_per_worker": planes, "reps": reps,
+            "seconds": t_last - t_first, "late_starters": late}
+
+
 def cpu_baseline(name: str):
-    """The oracle as it stands (single thread), fwd + bwd, on a sample of about 10-30 s of work."""
+    """The oracle as it stands, fwd + bwd, on a bounded sample: one thread, and one process per host
+    core running at the same time (the oracle itself is single-threaded and stays so)."""
     cfg_shape = W.CONFIGS[name]["shape"]
     per_plane = int(np.prod(cfg_shape[1:]))
     planes = max(5, min(cfg_shape[0], int(8.0e6 // per_plane) or 1))
     w = oracle_sample(name, planes)
     t = time_oracle(w, 3)
-    return {"value": w.npoints / t, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "first %d of %d slices along axis 0 of %s (%d points), fp64 fwd+bwd incl. loss, best of 3"
-                      % (w.shape[0], cfg_shape[0], name, w.npoints),
-            "seconds": t}
+    single = w.npoints / t
+    out = {"value": single, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": "first %d of %d slices along axis 0 of %s (%d points), fp64 fwd+bwd incl. loss, best of 3"
+                     % (w.shape[0], cfg_shape[0], name, w.npoints),
+           "seconds": t, "host_cores": os.cpu_count()}
+    try:
+        allc = cpu_baseline_all_cores(name, max(5, int(2.0e6 // per_plane) or 1))
+        out.update({"single_thread": single, "value": allc["value"], "cores": allc["cores"],
+                    "sample": "%d processes at once, each the single-thread oracle on its own seeded sample of %d "
+                              "slices along axis 0 of %s, %d passes each (fp64 fwd+bwd incl. loss); single_thread = "
+                              "one process on %d slices, best of 3"
+                              % (allc["cores"], allc["planes_per_worker"], name, allc["reps"], w.shape[0]),
+                    "seconds_all_cores": allc["seconds"], "late_starters": allc["late_starters"]})
+    except Exception as exc:             # no multiprocessing here: the one-thread figure stands
+        out["all_cores_error"] = repr(exc)
+    return out
 
 
 def run_reference(args, rank):
@@ -426,12 +484,13 @@ def config_line(torch, B, name, steps, warmup, peak):
     fm, bm = statistics.median(f_ms), statistics.median(b_ms)
     fb, bb = ALGO_BYTES[w.op]
     N = w.npoints
-    out = {"shape": list(w.shape), "points": N, "ms_fwd": fm, "ms_bwd": bm,
+    out = {"shape": list(w.shape), "points": N, "ms_fwd": fm, "ms_bwd": bm, "ms_fwd_min": min(f_ms), "ms_bwd_min": min(b_ms),
            "points_per_s": N / ((fm + bm) * 1e-3),
            "gbs_fwd": fb * N / (fm * 1e-3) / 1e9, "gbs_bwd": bb * N / (bm * 1e-3) / 1e9,
            "gbs_pair": (fb + bb) * N / ((fm + bm) * 1e-3) / 1e9}
     out["frac_pair"] = out["gbs_pair"] / peak
-    out["timing"] = "cold: 256 MiB L2 flush before every step, per-call medians"
+    out["frac_pair_min"] = (fb + bb) * N / ((min(f_ms) + min(b_ms)) * 1e-3) / 1e9 / peak
+    out["timing"] = "cold: 256 MiB L2 flush before every step, per-call medians (and minima) of %d steps after %d" % (steps, warmup)
     # the same with the cache left clean (write, then read another buffer): what the kernels do when
     # they do not also have to write back the flush's dirty lines
     clean = CleanFlush(torch, flush)
@@ -444,6 +503,7 @@ def config_line(torch, B, name, steps, warmup, peak):
     # from one CUDA graph, which removes the host launch gaps of the latency-bound small grids
     total_ms, _, _ = timed_steps(torch, prob, steps, 3, lambda: None)
     out["warm_points_per_s"] = N * steps / (total_ms * 1e-3)
+    out["frac_warm"] = (fb + bb) * N * steps / (total_ms * 1e-3) / 1e9 / peak
     out["l2_resident"] = bool((fb + bb) * N < (100 << 20))
     out["graph_points_per_s"] = graph_points_per_s(torch, prob, N, pairs=10, replays=max(3, steps // 10))
     if B.has_single_pass(w.op):
@@ -539,6 +599,17 @@ def main():
     total_ms, _, _ = timed_steps(torch, prob, args.steps, args.warmup, barrier)
     # same K steps again with an event pair around every call: per-kernel durations for the roofline
     _, fwd_ms, bwd_ms = timed_steps(torch, prob, args.steps, 0, barrier, inner_events=True)
+    # The K-step block repeated (every block timed like the first, a host sync and a time stamp
+    # between blocks) until about 0.3 s have passed, with the clock sampler running across all of
+    # them: median and fastest block, and per block ms x SM MHz, so that a reader can tell a faster
+    # kernel from a faster clock.  `value` stays the first block's (the K steps the contract names).
+    blocks = []
+    if world == 1 and not args.slabs:
+        n_blocks = max(10, min(200, int(300.0 / max(total_ms, 1e-3)) + 1))
+        for _ in range(n_blocks):
+            t0 = time.perf_counter()
+            ms, _, _ = timed_steps(torch, prob, args.steps, 0, barrier)
+            blocks.append((ms, t0, time.perf_counter()))
     sampler.stop()
     total_ms = max_over_ranks(total_ms, dist, "cuda")
     value = job_value(1 if args.slabs else world, N, args.steps, total_ms)
@@ -576,11 +647,25 @@ def main():
                                  "achieved": (fb, bb)[1 - dom] * Nk / ((f_avg, b_avg)[1 - dom] * 1e-3) / 1e9},
                 "pair_achieved": (fb + bb) * Nk * args.steps / (total_ms * 1e-3) / 1e9,
                 "pair_frac": (fb + bb) * Nk * args.steps / (total_ms * 1e-3) / 1e9 / peak}
+    roofline["frac_of_nominal_8000"] = achieved / NOMINAL_HBM_GBS
+    roofline["pair_frac_of_nominal_8000"] = roofline["pair_achieved"] / NOMINAL_HBM_GBS
+    if blocks:
+        b_ms = [b[0] / args.steps for b in blocks]
+        b_mhz = [sampler.mhz_between(b[1], b[2]) for b in blocks]
+        pair_bytes = (fb + bb) * Nk
+        roofline["blocks"] = {
+            "n": len(blocks), "steps_per_block": args.steps,
+            "ms_per_step_median": statistics.median(b_ms), "ms_per_step_min": min(b_ms),
+            "pair_frac_median": pair_bytes / (statistics.median(b_ms) * 1e-3) / 1e9 / peak,
+            "pair_frac_best": pair_bytes / (min(b_ms) * 1e-3) / 1e9 / peak,
+            "ms_x_mhz": [None if m is None else round(t * m, 1) for t, m in zip(b_ms, b_mhz)],
+            "sm_mhz": b_mhz,
+            "what": "the K-step block repeated back to back; ms_x_mhz = ms per step x median SM MHz sampled during the block"}
     if args.slabs:
         roofline["note"] = "per-call times include the halo exchange of the step (and the loss all-reduce)"
     elif not args.single_pass:
         # the dominant kernel launched K times back to back between ONE pair of events: its
-        # sustained per-launch time, with the ramp and tail of consecutive launches overlapping
+        # per-launch time with the ramp and tail of consecutive launches overlapping
         # (programmatic dependent launch) as they do inside a step
         call = prob.bwd if dom == 1 else prob.fwd
         for _ in range(3):
@@ -592,9 +677,9 @@ def main():
             call()
         s1.record(); torch.cuda.synchronize()
         sus_ms = s0.elapsed_time(s1) / args.steps
-        roofline["sustained"] = {"avg_ms": sus_ms, "achieved": dom_bytes / (sus_ms * 1e-3) / 1e9,
-                                 "frac": dom_bytes / (sus_ms * 1e-3) / 1e9 / peak,
-                                 "what": "%d consecutive launches of the dominant kernel between one event pair" % args.steps}
+        roofline["back_to_back"] = {"avg_ms": sus_ms, "achieved": dom_bytes / (sus_ms * 1e-3) / 1e9,
+                                    "frac": dom_bytes / (sus_ms * 1e-3) / 1e9 / peak,
+                                    "what": "%d consecutive launches of the dominant kernel between one event pair" % args.steps}
 
     # The same step over about two seconds: on these parts the SM clock comes down from its boost
     # value a few tenths of a second into a sustained load (power management), and these kernels
@@ -615,9 +700,15 @@ def main():
         ec.record(); torch.cuda.synchronize()
         s_sampler.stop()
         sus_ms = eb.elapsed_time(ec) / (n_sus - half)
+        s_clk = s_sampler.summary()
         sustained = {"steps": n_sus, "seconds": ea.elapsed_time(ec) * 1e-3, "ms_per_step": sus_ms,
                      "value": N / (sus_ms * 1e-3), "pair_frac": (fb + bb) * Nk / (sus_ms * 1e-3) / 1e9 / peak,
-                     "clocks": s_sampler.summary(), "what": "second half of a ~2 s back-to-back run of the same step"}
+                     "pair_frac_of_nominal_8000": (fb + bb) * Nk / (sus_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                     "ms_x_mhz": None if s_clk.get("sm_mhz") is None else sus_ms * s_clk["sm_mhz"],
+                     "clocks": s_clk, "what": "second half of a ~2 s back-to-back run of the same step"}
+        roofline["sustained"] = {k: sustained[k] for k in ("ms_per_step", "pair_frac", "pair_frac_of_nominal_8000", "ms_x_mhz")}
+        roofline["sustained"].update({"sm_mhz_median": s_clk.get("sm_mhz"), "reasons": s_clk.get("reasons"),
+                                      "what": sustained["what"]})
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -641,8 +732,26 @@ def main():
     if world == 1 and not args.no_extras:
         del prob
         torch.cuda.empty_cache()
-        line["per_config"] = {name: config_line(torch, B, name, 30, 5, peak) for name in W.CONFIG_ORDER + W.EXTRA_CONFIGS}
+        line["per_config"] = {name: config_line(torch, B, name, 100, 50, peak) for name in W.CONFIG_ORDER + W.EXTRA_CONFIGS}
+        # the same figures in short, inside a key every reader of the line keeps: per workload the
+        # pair's fraction of the measured peak cold (L2 flushed by a write), cold with a clean L2,
+        # back to back, the CUDA-graph figure, and the single-pass / one-call entry point
+        short = {}
+        for name, c in line["per_config"].items():
+            sp, fc = c.get("single_pass"), c.get("fwd_bwd_call")
+            short[name] = {"frac_cold": round(c["frac_pair"], 4), "frac_cold_best": round(c["frac_pair_min"], 4),
+                           "frac_clean": round(c["clean_l2"]["frac_pair"], 4), "frac_warm": round(c["frac_warm"], 4),
+                           "frac_cold_of_nominal_8000": round(c["gbs_pair"] / NOMINAL_HBM_GBS, 4),
+                           "points_per_s_cold": c["points_per_s"], "graph_points_per_s": c["graph_points_per_s"],
+                           "l2_resident": c["l2_resident"]}
+            if sp:
+                short[name]["single_pass"] = {"frac": round(sp["frac"], 4), "points_per_s": sp["points_per_s"],
+                                              "graph_points_per_s": sp["graph_points_per_s"]}
+            if fc:
+                short[name]["fwd_bwd_call_frac"] = round(fc["frac_pair"], 4)
+        line["roofline"]["per_workload"] = short
         line["cpu_baseline"] = cpu_baseline(args.workload)
+        line["config"]["cpu_sample"] = line["cpu_baseline"]["sample"]
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
