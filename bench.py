@@ -554,6 +554,9 @@ def main():
     ap.add_argument("--single-pass", action="store_true",
                     help="time fpde_fwd_bwd (one kernel: loss + gradient, residual arrays not stored) as the step; "
                          "only for operators that have a single-pass kernel")
+    ap.add_argument("--one-call", action="store_true",
+                    help="time fpde_fwd_bwd as the step for any operator (forward, loss and adjoint queued by one call; "
+                         "operators without a single-pass kernel pass their residual arrays as the intermediate)")
     ap.add_argument("--slabs", action="store_true",
                     help="strong scaling: ONE grid split into x-slabs, one per rank, with halo exchange "
                          "(default: independent replicas, weak scaling)")
@@ -591,6 +594,8 @@ def main():
     if args.single_pass:
         if not B.has_single_pass(w.op):
             raise SystemExit("--single-pass: operator %s has no single-pass kernel" % w.op)
+        prob.fwd, prob.bwd = prob.fwd_bwd, (lambda: None)
+    if args.one_call:
         prob.fwd, prob.bwd = prob.fwd_bwd, (lambda: None)
     N = w.npoints
 
@@ -631,6 +636,10 @@ def main():
         fb, bb = 4 * (2 * len(w.fields) + len(w.sources)), 0
         knames = ("fused2d_kernel<%s>" % w.op, "-")
         b_avg = 0.0
+    elif args.one_call:         # the pair's bytes against the time of the one call
+        fb, bb = fb + bb, 0
+        knames = ("fpde_fwd_bwd(%s)" % w.op, "-")
+        b_avg = 0.0
     dom = 1 if b_avg >= f_avg else 0
     Nk = N // world if args.slabs else N       # grid points one rank's kernels process (own planes)
     dom_bytes = (fb, bb)[dom] * Nk
@@ -641,7 +650,7 @@ def main():
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom_name)),
                 "algorithmic_bytes": dom_bytes, "avg_ms": dom_ms,
-                "other_kernel": None if args.single_pass else
+                "other_kernel": None if (args.single_pass or args.one_call) else
                                 {"kernel": knames[1 - dom], "avg_ms": (f_avg, b_avg)[1 - dom],
                                  "note": "forward figure includes the one-block loss finalise launch",
                                  "achieved": (fb, bb)[1 - dom] * Nk / ((f_avg, b_avg)[1 - dom] * 1e-3) / 1e9},
@@ -663,7 +672,7 @@ def main():
             "what": "the K-step block repeated back to back; ms_x_mhz = ms per step x median SM MHz sampled during the block"}
     if args.slabs:
         roofline["note"] = "per-call times include the halo exchange of the step (and the loss all-reduce)"
-    elif not args.single_pass:
+    elif not (args.single_pass or args.one_call):
         # the dominant kernel launched K times back to back between ONE pair of events: its
         # per-launch time with the ramp and tail of consecutive launches overlapping
         # (programmatic dependent launch) as they do inside a step
@@ -715,7 +724,8 @@ def main():
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "strong" if args.slabs else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "operator": w.op, "shape": list(w.shape), "points": N,
-                   "fields": len(w.fields), "step": "fpde_fwd_bwd (single pass)" if args.single_pass else "fpde_fwd + fpde_bwd",
+                   "fields": len(w.fields), "step": "fpde_fwd_bwd (single pass)" if args.single_pass else
+                           ("fpde_fwd_bwd (one call)" if args.one_call else "fpde_fwd + fpde_bwd"),
                    "parallelism": ("x-slabs x%d of one grid, halo exchange per step" if args.slabs
                                    else "replicas x%d (no exchange step)") % world,
                    "l2": "per-step traffic %.0f MB >> L2, no flush needed" % ((fb + bb) * N / 1e6)

@@ -312,6 +312,13 @@ static int bwd_impl(int op, const float* const* fields, const float* const* gres
     return ce == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
 }
 
+// The Helmholtz single-pass kernel is a measured prototype: slower than forward + adjoint on the
+// grids tried (see the design notes), so it only runs when asked for (FPDE_STAR3D_SINGLE_PASS=1).
+static bool helmholtz_single_pass_wanted(const int* n) {
+    const char* s = std::getenv("FPDE_STAR3D_SINGLE_PASS");
+    return s && s[0] == '1' && star3d_fused_supported(n);
+}
+
 int fpde_has_single_pass(int op) {
     return (op >= 0 && op < FPDE_OP_COUNT && fused2d_supported(op)) ? 1 : 0;
 }
@@ -334,6 +341,28 @@ int fpde_fwd_bwd(int op, const float* const* fields, const float* const* sources
     if (st != FPDE_OK) return st;
     const OpEntry& e = REGISTRY[op];
     if (!gfields) return FPDE_ERR_NULL;
+    if (op == FPDE_OP_HELMHOLTZ_3D_O4 && helmholtz_single_pass_wanted(q.n)) {
+        // one kernel: the planes of r go from the forward star to the adjoint star through shared memory
+        if (!sources || !sources[0] || !gfields[0]) return FPDE_ERR_NULL;
+        if (!aligned16(sources[0]) || !aligned16(gfields[0])) return FPDE_ERR_ALIGN;
+        float* res = residuals ? residuals[0] : nullptr;
+        if (res && !aligned16(res)) return FPDE_ERR_ALIGN;
+        q.aux[0] = sources[0]; q.out[0] = gfields[0];
+        if (loss_out) {
+            if (!aligned16(loss_out)) return FPDE_ERR_ALIGN;
+            if (!workspace || !aligned16(workspace) || workspace_bytes < (size_t)star3d_fused_items(q.n) * sizeof(float))
+                return FPDE_ERR_WORKSPACE;
+            q.partials = static_cast<float*>(workspace);
+            q.loss_out = loss_out;
+        }
+        q.stream = static_cast<cudaStream_t>(stream);
+        int items = 0;
+        cudaError_t ce = launch_star3d_fused(q, res, &items);
+        if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+        if (loss_out && launch_loss_finalize(q.partials, items, e.ne, q.rows, loss_out, q.stream) != cudaSuccess)
+            return FPDE_ERR_CUDA;
+        return FPDE_OK;
+    }
     if (!fused2d_supported(op)) {
         // two kernels with the residual arrays as the intermediate
         if (!residuals) return FPDE_ERR_NULL;
@@ -793,8 +822,8 @@ int fpde_fwd_noalloc(int op, const float* const* fields, const float* const* sou
 }
 
 unsigned int fpde_diag_tma_timeouts(void) {
-    const unsigned int a = ns_tma_timeouts(), b = star3d_tma_timeouts();
-    return (a == ~0u || b == ~0u) ? ~0u : a + b;
+    const unsigned int a = ns_tma_timeouts(), b = star3d_tma_timeouts(), c = star3d_fused_timeouts();
+    return (a == ~0u || b == ~0u || c == ~0u) ? ~0u : a + b + c;
 }
 
 int fpde_diag_ns_tma_geometry(const int64_t* shape, int tile_rows, int narrays, size_t smem_limit) {

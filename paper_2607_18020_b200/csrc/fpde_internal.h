@@ -111,6 +111,12 @@ bool star3d_tma_wanted(const int* n);
 int star3d_tma_items(const int* n);
 cudaError_t launch_star3d_tma(const Problem& p, int mode, int* items, bool& launched);
 unsigned int star3d_tma_timeouts();
+// Helmholtz single pass (op_helmholtz3d_fused.cu): residual, loss partial sums and gradient in one
+// kernel; `res` may be NULL (residuals not stored)
+bool star3d_fused_supported(const int* n);
+int star3d_fused_items(const int* n);
+cudaError_t launch_star3d_fused(const Problem& p, float* res, int* items);
+unsigned int star3d_fused_timeouts();
 // TMA-staged variants (op_ns3dt_tma.cu); `launched` false = this grid is not eligible
 bool ns_tma_wanted(const int* n);
 bool ns_tma_geometry_ok(const int* n, int ty, int na, size_t smem_limit);

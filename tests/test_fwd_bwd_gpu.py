@@ -132,3 +132,30 @@ def test_two_kernel_operators(name, shape):
     st = B.fwd_bwd_status(w.op, fields, to_dev(torch, w.sources), None, grads, None, w.shape, w.spacing, w.coeffs,
                           w.bc, None, 0, None)
     assert st == 2
+
+
+@pytest.mark.parametrize("shape", [(9, 16, 128), (21, 45, 128), (12, 24, 256), (37, 50, 256)])
+@pytest.mark.parametrize("store_res", [False, True])
+def test_helmholtz_single_pass_prototype(shape, store_res, monkeypatch):
+    """FPDE_STAR3D_SINGLE_PASS=1: residual, loss and gradient of the Helmholtz operator from one kernel
+    (planes of r handed from the forward star to the adjoint star through shared memory) on grids
+    whose z lines are 128 or 256 floats; ragged row tiles, CTAs whose share spans several tiles."""
+    monkeypatch.setenv("FPDE_STAR3D_SINGLE_PASS", "1")
+    w = W.make("helmholtz_256", seed=49, shape=shape, kind="randn")
+    R_ref, loss_ref, g_ref, _ = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    fields, sources = to_dev(torch, w.fields), to_dev(torch, w.sources)
+    res = Guarded(torch, shape, fill=7.0) if store_res else None
+    grad = Guarded(torch, shape, fill=9.0)
+    loss = torch.full((2,), -1.0, dtype=torch.float64, device="cuda")
+    ws = torch.empty(B.fwd_bwd_workspace_bytes(w.op, shape), dtype=torch.uint8, device="cuda")
+    B.fpde_fwd_bwd(w.op, fields, sources, [res.view] if store_res else None, [grad.view], loss, shape, w.spacing,
+                   w.coeffs, w.bc, ws)
+    torch.cuda.synchronize()
+    grad.check()
+    assert_close(grad.view.cpu().numpy(), g_ref[0], "helmholtz single pass %s gradient" % (shape,))
+    L = loss.cpu().numpy()
+    assert np.all(np.abs(L - loss_ref) <= LOSS_TOL * np.abs(loss_ref)), (L, loss_ref)
+    if store_res:
+        res.check()
+        assert_close(res.view.cpu().numpy(), R_ref[0], "helmholtz single pass %s residual" % (shape,))
+    assert B.diag_tma_timeouts() == 0
