@@ -327,16 +327,17 @@ class SlabProblem:
         self.loss = torch.zeros(self.rank.ne + 1, dtype=torch.float64, device="cuda")
 
     def fwd(self):
-        self.S.exchange_dist(self.rank.plan, self.rank.fields, 2 * self.R, self.dist)
+        self.S.post_exchange(self.rank.plan, self.rank.field_stack, 2 * self.R, self.dist).wait()
         self.rank.fwd()
 
     def bwd(self):
-        self.S.exchange_dist(self.rank.plan, self.rank.res, self.R, self.dist)
+        ex = self.S.post_exchange(self.rank.plan, self.rank.res_stack, self.R, self.dist)
+        self.loss.copy_(self.rank.loss)             # this slab's share; the shares add up to the grid's loss
+        work = self.dist.all_reduce(self.loss, op=self.dist.ReduceOp.SUM, async_op=True) if self.dist is not None else None
+        ex.wait()
         self.rank.bwd()
-        sums = self.rank.loss_sums().clone()
-        if self.dist is not None:
-            self.dist.all_reduce(sums, op=self.dist.ReduceOp.SUM)
-        self.loss = self.S.global_loss(self.rank.torch, sums, self.rank.rows_global)
+        if work is not None:
+            work.wait()
 
 
 def timed_steps(torch, prob, steps, warmup, barrier, flush=None, inner_events=False):
@@ -459,6 +460,59 @@ def single_pass_figures(torch, prob, steps, warmup, flush, peak):
             "what": "fpde_fwd_bwd, residual arrays not stored; launches: 1 kernel + loss finalise"}
 
 
+def rotating_figures(torch, B, w, prob, steps, peak):
+    """Cold without a flush: the step runs back to back over three sets of arrays in turn (each set
+    larger than half of L2, all three several times L2), so every array comes from DRAM, nothing of
+    a flush has to be written back, and consecutive launches overlap as they do in use."""
+    fb, bb = ALGO_BYTES[w.op]
+    N = w.npoints
+    probs = [prob] + [DeviceProblem(torch, B, w) for _ in range(2)]
+    for q in probs:
+        q.fwd(); q.bwd()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for k in range(steps):
+        q = probs[k % 3]
+        q.fwd(); q.bwd()
+    e1.record(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    del probs
+    return {"ms_per_step": ms, "points_per_s": N / (ms * 1e-3), "frac_pair": (fb + bb) * N / (ms * 1e-3) / 1e9 / peak,
+            "what": "%d steps back to back over three sets of arrays in turn (no flush, every array from DRAM)" % steps}
+
+
+def sustained_figures(torch, prob, N, pair_bytes, peak, seconds=1.0):
+    """The step back to back for about a second; the figure is that of the second half (the SM clock
+    settles under the power cap a few tenths of a second into a sustained load)."""
+    for _ in range(3):
+        prob.fwd(); prob.bwd()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(20):
+        prob.fwd(); prob.bwd()
+    e1.record(); torch.cuda.synchronize()
+    n = max(40, int(seconds * 1e3 / max(e0.elapsed_time(e1) / 20, 1e-3)))
+    half = n // 2
+    sm = ClockSampler(torch, torch.cuda.current_device())
+    ea, eb, ec = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    sm.start()
+    ea.record()
+    for k in range(n):
+        if k == half:
+            eb.record()
+        prob.fwd(); prob.bwd()
+    ec.record(); torch.cuda.synchronize()
+    sm.stop()
+    ms = eb.elapsed_time(ec) / (n - half)
+    clk = sm.summary()
+    return {"ms_per_step": ms, "points_per_s": N / (ms * 1e-3), "frac_pair": pair_bytes / (ms * 1e-3) / 1e9 / peak,
+            "sm_mhz_median": clk.get("sm_mhz"), "reasons": clk.get("reasons"),
+            "ms_x_mhz": None if clk.get("sm_mhz") is None else ms * clk["sm_mhz"],
+            "what": "second half of a ~%.0f s back-to-back run" % seconds}
+
+
 class CleanFlush:
     """An L2 flush that leaves the cache clean: the 256 MiB write, then a read of another 256 MiB.
     After the write alone the whole L2 holds dirty lines, and the first kernel that follows pays
@@ -506,6 +560,9 @@ def config_line(torch, B, name, steps, warmup, peak):
     out["frac_warm"] = (fb + bb) * N * steps / (total_ms * 1e-3) / 1e9 / peak
     out["l2_resident"] = bool((fb + bb) * N < (100 << 20))
     out["graph_points_per_s"] = graph_points_per_s(torch, prob, N, pairs=10, replays=max(3, steps // 10))
+    if not out["l2_resident"]:
+        out["rotating"] = rotating_figures(torch, B, w, prob, steps, peak)
+        out["sustained"] = sustained_figures(torch, prob, N, (fb + bb) * N, peak)
     if B.has_single_pass(w.op):
         out["single_pass"] = single_pass_figures(torch, prob, steps, warmup, flush, peak)
     else:
@@ -745,7 +802,8 @@ def main():
         line["per_config"] = {name: config_line(torch, B, name, 100, 50, peak) for name in W.CONFIG_ORDER + W.EXTRA_CONFIGS}
         # the same figures in short, inside a key every reader of the line keeps: per workload the
         # pair's fraction of the measured peak cold (L2 flushed by a write), cold with a clean L2,
-        # back to back, the CUDA-graph figure, and the single-pass / one-call entry point
+        # cold over rotating sets of arrays (no flush), back to back, over a second of sustained
+        # load, the CUDA-graph figure, and the single-pass / one-call entry point
         short = {}
         for name, c in line["per_config"].items():
             sp, fc = c.get("single_pass"), c.get("fwd_bwd_call")
@@ -759,6 +817,11 @@ def main():
                                               "graph_points_per_s": sp["graph_points_per_s"]}
             if fc:
                 short[name]["fwd_bwd_call_frac"] = round(fc["frac_pair"], 4)
+            if c.get("rotating"):
+                short[name]["frac_rotating"] = round(c["rotating"]["frac_pair"], 4)
+            if c.get("sustained"):
+                short[name]["sustained"] = {"frac": round(c["sustained"]["frac_pair"], 4), "sm_mhz": c["sustained"]["sm_mhz_median"],
+                                            "ms_x_mhz": c["sustained"]["ms_x_mhz"]}
         line["roofline"]["per_workload"] = short
         line["cpu_baseline"] = cpu_baseline(args.workload)
         line["config"]["cpu_sample"] = line["cpu_baseline"]["sample"]

@@ -61,6 +61,8 @@ def lib():
                                ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fpde_fwd_rows.restype = ctypes.c_int
+        L.fpde_fwd_rows.argtypes = L.fpde_fwd.argtypes + [ctypes.c_int64]
         L.fpde_bwd.restype = ctypes.c_int
         L.fpde_bwd.argtypes = [ctypes.c_int, vpp, vpp, ctypes.POINTER(ctypes.c_double), vpp, ctypes.c_int,
                                ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
@@ -177,9 +179,12 @@ def workspace_bytes(op, shape) -> int:
 
 
 def fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace,
-               workspace_bytes_, stream, ndim=None, ncoeffs=None) -> int:
-    """Raw call: returns the status code (used by the error-path tests)."""
-    return lib().fpde_fwd(_opid(op),
+               workspace_bytes_, stream, ndim=None, ncoeffs=None, loss_rows=None) -> int:
+    """Raw call: returns the status code (used by the error-path tests).  With loss_rows the call
+    is fpde_fwd_rows (the loss divides by that row count)."""
+    fn = lib().fpde_fwd if loss_rows is None else lib().fpde_fwd_rows
+    extra = () if loss_rows is None else (int(loss_rows),)
+    return fn(_opid(op),
                           _ptr_array(_dev_ptrs(fields)) if fields is not None else None,
                           _ptr_array(_dev_ptrs(sources)) if sources is not None else None,
                           _ptr_array(_dev_ptrs(residuals)) if residuals is not None else None,
@@ -191,7 +196,7 @@ def fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs,
                           len(coeffs) if ncoeffs is None else ncoeffs,
                           _bcs(bc) if bc is not None else None,
                           _dev_ptrs([workspace])[0] if workspace is not None else None,
-                          int(workspace_bytes_), stream)
+                          int(workspace_bytes_), stream, *extra)
 
 
 def bwd_status(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, workspace,
@@ -294,6 +299,18 @@ def fpde_fwd(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, b
                         _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd")
+
+
+def fpde_fwd_rows(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, loss_rows,
+                  stream=None):
+    """fpde_fwd whose loss divides by `loss_rows` (the row count of the whole grid when this array
+    is one slab of it): the ranks' loss vectors then add up to the loss of the whole grid."""
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    with _on_device_of(fields, sources, residuals, loss_out, workspace):
+        st = fwd_status(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, wsb,
+                        _stream_handle(stream), loss_rows=loss_rows)
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_fwd_rows")
 
 
 def fpde_fwd_bwd(op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc, workspace,

@@ -212,10 +212,32 @@ size_t fpde_workspace_bytes(int op, int ndim, const int64_t* shape) {
     return ((need + 255) / 256) * 256 + 4096;
 }
 
+static int fwd_impl(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+                    double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+                    const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+                    void* stream, int64_t loss_rows);
+
 int fpde_fwd(int op, const float* const* fields, const float* const* sources, float* const* residuals,
              double* loss_out, int ndim, const int64_t* shape, const double* spacing,
              const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
              void* stream) {
+    return fwd_impl(op, fields, sources, residuals, loss_out, ndim, shape, spacing, coeffs, ncoeffs, bc, workspace,
+                    workspace_bytes, stream, 0);
+}
+
+int fpde_fwd_rows(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+                  double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+                  const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+                  void* stream, int64_t loss_rows) {
+    if (loss_rows < 1) return FPDE_ERR_SHAPE;
+    return fwd_impl(op, fields, sources, residuals, loss_out, ndim, shape, spacing, coeffs, ncoeffs, bc, workspace,
+                    workspace_bytes, stream, loss_rows);
+}
+
+static int fwd_impl(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+                    double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+                    const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+                    void* stream, int64_t loss_rows) {
     Problem q;
     std::memset(&q, 0, sizeof(q));
     int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
@@ -256,7 +278,7 @@ int fpde_fwd(int op, const float* const* fields, const float* const* sources, fl
     }
     if (ce != cudaSuccess) return FPDE_ERR_CUDA;
     if (loss_out) {
-        ce = launch_loss_finalize(q.partials, items, e.ne, q.rows, loss_out, q.stream);
+        ce = launch_loss_finalize(q.partials, items, e.ne, loss_rows > 0 ? loss_rows : q.rows, loss_out, q.stream);
         if (ce != cudaSuccess) return FPDE_ERR_CUDA;
     }
     return FPDE_OK;

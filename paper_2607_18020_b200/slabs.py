@@ -11,7 +11,9 @@ those rows' own neighbours).  So per step a rank
   4. runs the adjoint kernel on the planes [x0 - 2 radius, x1 + 2 radius): with the interior-axis
      rule (rows where the stencil fits) the upstream arrays are honoured on [x0 - radius,
      x1 + radius), which is what the gradients on the own planes [x0, x1) need,
-  5. sums the loss over ranks (nresiduals + 1 doubles).
+  5. adds up the ranks' shares of the loss (nresiduals + 1 doubles, one all-reduce posted before
+     the adjoint so that it runs beside it): the forward call divides by the row count of the
+     WHOLE grid (fpde_fwd_rows), so no loss arithmetic is done outside the library.
 
 Every array is stored once per rank with the widest halo; the forward call is handed a
 sub-range of planes (contiguous, because x is the slowest axis), so nothing is copied locally.
@@ -160,38 +162,66 @@ def plans(op: str, shape: Sequence[int], world: int) -> List[SlabPlan]:
     return ps
 
 
-def exchange_local(plan_list: Sequence[SlabPlan], arrays: Sequence[Sequence], halo: int):
-    """Fill the halo planes when all slabs live in this process: arrays[rank][k] is the k-th
-    local array (wide range) of that rank."""
+def exchange_local(plan_list: Sequence[SlabPlan], arrays: Sequence, halo: int):
+    """Fill the halo planes when all slabs live in this process.  arrays[rank] is either the list of
+    that rank's local arrays (wide range, planes on axis 0) or ONE stacked tensor of them (arrays on
+    axis 0, planes on axis 1): with the stacked form a transfer is one strided copy for all arrays."""
     for plan in plan_list:
         for t in plan.halo_transfers(halo):
             src_plan = plan_list[t.peer]
             s = src_plan.local_of(t.start)
-            for dst_arr, src_arr in zip(arrays[plan.rank], arrays[t.peer]):
-                dst_arr[t.dst:t.dst + t.count].copy_(src_arr[s:s + t.count])
+            dst_set, src_set = arrays[plan.rank], arrays[t.peer]
+            if hasattr(dst_set, "dim"):
+                dst_set[:, t.dst:t.dst + t.count].copy_(src_set[:, s:s + t.count])
+            else:
+                for dst_arr, src_arr in zip(dst_set, src_set):
+                    dst_arr[t.dst:t.dst + t.count].copy_(src_arr[s:s + t.count])
 
 
-def exchange_dist(plan: SlabPlan, arrays: Sequence, halo: int, dist):
-    """Fill the halo planes of this rank's arrays from the other ranks (torch.distributed
-    point-to-point; both sides enumerate the transfers in the same order).  Planes a rank
-    needs from itself (one rank on a periodic axis) are copied."""
+class Exchange:
+    """A halo exchange that has been posted: `wait()` returns once every halo plane has landed."""
+
+    def __init__(self, reqs):
+        self.reqs = reqs
+
+    def wait(self):
+        for req in self.reqs:
+            req.wait()
+        self.reqs = []
+
+
+def post_exchange(plan: SlabPlan, arrays, halo: int, dist) -> Exchange:
+    """Post the receives and sends that fill `halo` planes beyond each end of this rank's own planes
+    (torch.distributed point-to-point; both sides enumerate the transfers in the same order) and
+    return at once: work that does not read the halo planes can be queued before `wait()`.
+    `arrays`: the list of this rank's local arrays, or one stacked tensor of them.  Planes a rank needs
+    from itself (one rank on a periodic axis) are copied; they never overlap the planes they come from."""
+    stacked = hasattr(arrays, "dim")
+    per_array = list(arrays.unbind(0)) if stacked else list(arrays)
     ops = []
     for t in plan.halo_transfers(halo):
-        for arr in arrays:
-            if t.peer == plan.rank:
-                s = plan.local_of(t.start)
-                arr[t.dst:t.dst + t.count].copy_(arr[s:s + t.count].clone())
+        if t.peer == plan.rank:
+            s = plan.local_of(t.start)
+            if stacked:
+                arrays[:, t.dst:t.dst + t.count].copy_(arrays[:, s:s + t.count])
             else:
+                for arr in per_array:
+                    arr[t.dst:t.dst + t.count].copy_(arr[s:s + t.count])
+        else:
+            for arr in per_array:
                 ops.append(dist.P2POp(dist.irecv, arr[t.dst:t.dst + t.count], t.peer))
     for dst, t in plan.sends(halo):
         if dst == plan.rank:
             continue
         s = plan.local_of(t.start)
-        for arr in arrays:
+        for arr in per_array:
             ops.append(dist.P2POp(dist.isend, arr[s:s + t.count], dst))
-    if ops:
-        for req in dist.batch_isend_irecv(ops):
-            req.wait()
+    return Exchange(dist.batch_isend_irecv(ops) if ops else [])
+
+
+def exchange_dist(plan: SlabPlan, arrays, halo: int, dist):
+    """post_exchange + wait."""
+    post_exchange(plan, arrays, halo, dist).wait()
 
 
 class SlabRank:
@@ -205,10 +235,14 @@ class SlabRank:
         self.nf, self.ns, self.ne = len(meta["fields"]), len(meta["sources"]), len(meta["residuals"])
         self.bc = W.CONFIGS[next(k for k, c in W.CONFIGS.items() if c["op"] == plan.local_op)]["bc"]
         ls = plan.local_shape
+        # the arrays of one kind are slices of ONE tensor, so that a halo transfer between slabs of
+        # one process is a single strided copy for all of them
+        stack = lambda k: torch.zeros((max(k, 1),) + tuple(ls), dtype=torch.float32, device=device)
+        self.field_stack, self.res_stack = stack(self.nf), stack(self.ne)
+        self.fields = list(self.field_stack.unbind(0))[:self.nf]
+        self.res = list(self.res_stack.unbind(0))[:self.ne]
         new = lambda: torch.zeros(ls, dtype=torch.float32, device=device)
-        self.fields = [new() for _ in range(self.nf)]
         self.sources = [new() for _ in range(self.ns)]
-        self.res = [new() for _ in range(self.ne)]
         self.grads = [new() for _ in range(self.nf)]
         self.loss = torch.zeros(self.ne + 1, dtype=torch.float64, device=device)
         self.ws = torch.empty(max(16, B.workspace_bytes(plan.local_op, plan.tight_shape)), dtype=torch.uint8, device=device) \
@@ -235,51 +269,49 @@ class SlabRank:
             dst.copy_(self.torch.as_tensor(src[x0:x1]))
 
     def fwd(self, stream=None):
+        """Forward kernel on the tight range.  The loss vector is this slab's share of the whole
+        grid's loss (the library divides by the whole grid's row count), so shares add up."""
         s = self._tight_slice()
         p = self.plan
-        self.B.fpde_fwd(p.local_op, [a[s] for a in self.fields], [a[s] for a in self.sources], [a[s] for a in self.res],
-                        self.loss, p.tight_shape, self.spacing, self.coeffs, self.bc, self.ws, stream)
+        self.B.fpde_fwd_rows(p.local_op, [a[s] for a in self.fields], [a[s] for a in self.sources], [a[s] for a in self.res],
+                             self.loss, p.tight_shape, self.spacing, self.coeffs, self.bc, self.ws, self.rows_global, stream)
 
     def bwd(self, stream=None):
         p = self.plan
         self.B.fpde_bwd(p.local_op, self.fields, self.res, [2.0 / self.rows_global] * self.ne, self.grads,
                         p.local_shape, self.spacing, self.coeffs, self.bc, None, stream)
 
-    def loss_sums(self):
-        """Sum over this rank's rows of r_e^2 (fp64 tensor, one entry per residual)."""
-        return self.loss[:self.ne] * float(self.rows_local)
-
-
-def global_loss(torch, sums, rows_global: int):
-    """Loss vector (L_0..L_{E-1}, sum) from the rank-summed squared-residual sums."""
-    per = sums / float(rows_global)
-    return torch.cat([per, per.sum().reshape(1)])
-
 
 def step_local(ranks: Sequence[SlabRank]):
     """One loss + gradient step over slabs that all live in this process (one GPU standing in for
-    several: the kernels of different slabs run one after the other, nothing waits on anything)."""
+    several: the kernels of different slabs run one after the other, nothing waits on anything).
+    Returns the loss vector of the whole grid: the sum of the slabs' shares."""
     plan_list = [r.plan for r in ranks]
     R = plan_list[0].radius
-    exchange_local(plan_list, [r.fields for r in ranks], 2 * R)
+    exchange_local(plan_list, [r.field_stack for r in ranks], 2 * R)
     for r in ranks:
         r.fwd()
-    exchange_local(plan_list, [r.res for r in ranks], R)
+    exchange_local(plan_list, [r.res_stack for r in ranks], R)
     for r in ranks:
         r.bwd()
-    torch = ranks[0].torch
-    sums = sum(r.loss_sums() for r in ranks)
-    return global_loss(torch, sums, ranks[0].rows_global)
+    loss = ranks[0].loss.clone()
+    for r in ranks[1:]:
+        loss += r.loss
+    return loss
 
 
 def step_dist(rank: SlabRank, dist):
-    """The same step with one slab per process."""
+    """The same step with one slab per process.  The all-reduce of the loss shares is posted before
+    the adjoint is queued, so it runs beside it; the returned vector is valid once the returned
+    handle (None on one rank) has been waited for."""
     R = rank.plan.radius
-    exchange_dist(rank.plan, rank.fields, 2 * R, dist)
+    post_exchange(rank.plan, rank.field_stack, 2 * R, dist).wait()
     rank.fwd()
-    exchange_dist(rank.plan, rank.res, R, dist)
+    ex = post_exchange(rank.plan, rank.res_stack, R, dist)
+    loss = rank.loss.clone()
+    work = dist.all_reduce(loss, op=dist.ReduceOp.SUM, async_op=True) if rank.plan.world > 1 else None
+    ex.wait()
     rank.bwd()
-    sums = rank.loss_sums().clone()
-    if rank.plan.world > 1:
-        dist.all_reduce(sums, op=dist.ReduceOp.SUM)
-    return global_loss(rank.torch, sums, rank.rows_global)
+    if work is not None:
+        work.wait()
+    return loss

@@ -217,3 +217,11 @@ def test_ns_tma_geometry_predicate_requires_aligned_slots_and_a_ring_that_fits()
     # rows that do not tile, t extent beyond the one-box limit
     assert not B.diag_ns_tma_geometry((16, 30, 64, 16), 4, 4, limit)
     assert not B.diag_ns_tma_geometry((16, 32, 64, 128), 4, 4, limit)
+
+
+def test_fwd_rows_rejects_a_row_count_below_one():
+    """fpde_fwd_rows divides the loss by a row count the caller names; 0 or a negative count is refused
+    before anything else is looked at."""
+    st = B.fwd_status(W.POISSON_2D, [16], [16], [16], None, (8, 8), (0.1, 0.1), (), (W.INTERIOR, W.INTERIOR), None, 0,
+                      None, loss_rows=0)
+    assert st == 4

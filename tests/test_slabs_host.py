@@ -71,6 +71,20 @@ def test_local_exchange_on_cpu_tensors():
         for p, (a,) in zip(ps, arrs):
             for l in range(p.local_shape[0]):
                 assert float(a[l].flatten()[0]) == _expected_plane(p, l)
+        # stacked form: one tensor per rank holding two arrays
+        stacks = []
+        for p in ps:
+            st = torch.full((2,) + tuple(p.local_shape), -1.0)
+            x0, x1 = p.owned
+            for g in range(x0, x1):
+                st[0, p.local_of(g)] = float(g)
+                st[1, p.local_of(g)] = float(g) + 100.0
+            stacks.append(st)
+        S.exchange_local(ps, stacks, 2 * ps[0].radius)
+        for p, st in zip(ps, stacks):
+            for l in range(p.local_shape[0]):
+                assert float(st[0, l].flatten()[0]) == _expected_plane(p, l)
+                assert float(st[1, l].flatten()[0]) == _expected_plane(p, l) + 100.0
 
 
 def _rank_main(rank, world, port, op, shape):
@@ -91,6 +105,17 @@ def _rank_main(rank, world, port, op, shape):
         for k, a in enumerate(arrs):
             for l in range(plan.local_shape[0]):
                 assert float(a[l].flatten()[0]) == _expected_plane(plan, l) + 100.0 * k, (rank, k, l)
+        # the same through one stacked tensor and a posted exchange that is waited for later
+        st = torch.full((2,) + tuple(plan.local_shape), -1.0)
+        x0, x1 = plan.owned
+        for k in range(2):
+            for g in range(x0, x1):
+                st[k, plan.local_of(g)] = float(g) + 100.0 * k
+        ex = S.post_exchange(plan, st, 2 * plan.radius, dist)
+        ex.wait()
+        for k in range(2):
+            for l in range(plan.local_shape[0]):
+                assert float(st[k, l].flatten()[0]) == _expected_plane(plan, l) + 100.0 * k, (rank, k, l)
         sums = torch.tensor([float(rank + 1), 2.0 * (rank + 1)], dtype=torch.float64)
         dist.all_reduce(sums, op=dist.ReduceOp.SUM)
         assert sums.tolist() == [3.0, 6.0]
