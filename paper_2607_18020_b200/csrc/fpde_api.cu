@@ -5,6 +5,7 @@
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
@@ -111,16 +112,17 @@ static int validate(int op, const float* const* fields, int ndim, const int64_t*
     return FPDE_OK;
 }
 
-// Fixed-order final sum.  Thread t adds partials t, t+1024, ... (four independent loads in
-// flight, combined in a fixed order) in fp64; then a shuffle tree inside each warp and one over
-// the 32 warp sums.  One block, so no inter-block ordering exists to vary: the result depends
-// on the data only.
+// Fixed-order final sum.  Thread t adds partials t, t+T, ... (T = threads of the block, four
+// independent loads in flight, combined in a fixed order) in fp64; then a shuffle tree inside each
+// warp and one over the warp sums.  One block, so no inter-block ordering exists to vary: the
+// result depends on the data and on T only, and T is a function of the number of partials.
 __global__ void __launch_bounds__(1024) loss_finalize_kernel(const float* __restrict__ partials, int nitems,
                                                              int nres, double inv_rows,
                                                              double* __restrict__ loss_out) {
     __shared__ double sm[MAX_F][32];
     pdl_wait_then_trigger();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int T = blockDim.x, nwarps = T >> 5;
     double s[MAX_F];
 #pragma unroll
     for (int e = 0; e < MAX_F; ++e) {
@@ -128,11 +130,11 @@ __global__ void __launch_bounds__(1024) loss_finalize_kernel(const float* __rest
         if (e < nres) {
             const float* p = partials + (size_t)e * nitems;
             int i = tid;
-            for (; i + 3072 < nitems; i += 4096) {
-                const float a = p[i], b = p[i + 1024], c = p[i + 2048], d = p[i + 3072];
+            for (; i + 3 * T < nitems; i += 4 * T) {
+                const float a = p[i], b = p[i + T], c = p[i + 2 * T], d = p[i + 3 * T];
                 s[e] += ((double)a + (double)b) + ((double)c + (double)d);
             }
-            for (; i < nitems; i += 1024) s[e] += (double)p[i];
+            for (; i < nitems; i += T) s[e] += (double)p[i];
         }
     }
 #pragma unroll
@@ -146,7 +148,7 @@ __global__ void __launch_bounds__(1024) loss_finalize_kernel(const float* __rest
         double total = 0.0;
 #pragma unroll
         for (int e = 0; e < MAX_F; ++e) {
-            double v = sm[e][lane];
+            double v = lane < nwarps ? sm[e][lane] : 0.0;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(FULL_MASK, v, o);
             if (e < nres) {
@@ -161,7 +163,12 @@ __global__ void __launch_bounds__(1024) loss_finalize_kernel(const float* __rest
 
 cudaError_t launch_loss_finalize(const float* partials, int nitems, int nres, int64_t rows,
                                  double* loss_out, cudaStream_t stream) {
-    return launch_kernel(loss_finalize_kernel, dim3(1), dim3(1024), stream, partials, nitems, nres,
+    // a small block for few partial sums (it starts sooner and its tree is shorter), the full one
+    // for many
+    const char* e = std::getenv("FPDE_FINALIZE_THREADS");
+    int threads = e && *e ? std::atoi(e) : (nitems <= 1024 ? 128 : (nitems <= 8192 ? 256 : 1024));
+    threads = std::max(32, std::min(1024, (threads / 32) * 32));
+    return launch_kernel(loss_finalize_kernel, dim3(1), dim3(threads), stream, partials, nitems, nres,
                          1.0 / (double)rows, loss_out);
 }
 
