@@ -1,6 +1,6 @@
 // Fourth-order Helmholtz star, r = Lap4 u + k^2 u - f (Section 2.1), and its gather-form adjoint
 // with the two-cell boundary band (Sections 2.2, 2.3): the engine that stages plane tiles through
-// shared memory with the copy engine (cp.async.bulk.tensor, no multicast).
+// shared memory with the copy engine (cp.async.bulk.tensor, each copy to the issuing CTA only).
 //
 // How it differs from the L1-staged engine (op_helmholtz3d.cu), which holds every load of a step in
 // registers while it is in flight and issues five 128-bit loads per output float4:

@@ -1,5 +1,5 @@
 // Navier-Stokes forward / adjoint kernels whose plane tiles are staged through shared memory by
-// TMA (cp.async.bulk.tensor, no multicast) in a four-stage ring, instead of through L1.
+// TMA (cp.async.bulk.tensor, each copy to the issuing CTA only) in a four-stage ring, instead of through L1.
 //
 // Why: the L1 variants keep every load of a step in registers while it is in flight, and at
 // 160-240 registers per thread only 2-3 small blocks fit on an SM, so DRAM / L2 latency is

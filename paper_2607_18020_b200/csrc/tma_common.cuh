@@ -1,5 +1,5 @@
 // Helpers of the kernels that stage their tiles through shared memory with the copy engine
-// (cp.async.bulk.tensor, no multicast): mbarrier primitives with bounded waits, the tiled bulk
+// (cp.async.bulk.tensor, each copy to the issuing CTA only): mbarrier primitives with bounded waits, the tiled bulk
 // load, 64- and 128-bit shared-memory loads, and the host-side tensor-map encoder.
 //
 // Every wait on an mbarrier is bounded: after the limit the waiting thread counts a timeout in a
