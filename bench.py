@@ -325,17 +325,30 @@ class SlabProblem:
         self.rank.load_owned(w.fields, w.sources)
         self.R = self.rank.plan.radius
         self.loss = torch.zeros(self.rank.ne + 1, dtype=torch.float64, device="cuda")
+        # launches over plane ranges (inner planes while the halos are in flight) only pay with real transfers
+        self.chunks = self.rank.chunk_plan() if world > 1 else None
 
     def fwd(self):
-        self.S.post_exchange(self.rank.plan, self.rank.field_stack, 2 * self.R, self.dist).wait()
-        self.rank.fwd()
+        ex = self.S.post_exchange(self.rank.plan, self.rank.field_stack, 2 * self.R, self.dist)
+        if self.chunks is not None:             # planes away from the halos while the halos are in flight
+            self.rank.fwd_inner(self.chunks[0])
+            ex.wait()
+            self.rank.fwd_edges(self.chunks[0])
+        else:
+            ex.wait()
+            self.rank.fwd()
 
     def bwd(self):
         ex = self.S.post_exchange(self.rank.plan, self.rank.res_stack, self.R, self.dist)
         self.loss.copy_(self.rank.loss)             # this slab's share; the shares add up to the grid's loss
         work = self.dist.all_reduce(self.loss, op=self.dist.ReduceOp.SUM, async_op=True) if self.dist is not None else None
-        ex.wait()
-        self.rank.bwd()
+        if self.chunks is not None:
+            self.rank.bwd_inner(self.chunks[1])
+            ex.wait()
+            self.rank.bwd_edges(self.chunks[1])
+        else:
+            ex.wait()
+            self.rank.bwd()
         if work is not None:
             work.wait()
 

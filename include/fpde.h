@@ -190,6 +190,51 @@ int fpde_fwd_rows(int op,
                   int64_t loss_rows);
 
 /*
+ * Launches over a range of x-planes, for overlapping the halo exchange of a grid split into slabs
+ * with the work that does not read the halo planes (Sections 2.1 and 2.2: rows are independent, so
+ * a launch may cover any subset of them).  Only FPDE_OP_NS_3D_T and FPDE_OP_NS_3D_T_XSLAB have
+ * them (FPDE_ERR_BAD_OP otherwise).
+ *
+ *   fpde_plane_chunk   planes per chunk for this operator and grid (0 = no ranged launches);
+ *                      chunk c covers planes [c * chunk, min((c + 1) * chunk, n_x)).  Host only.
+ *   fpde_fwd_chunks    fpde_fwd_rows restricted to the chunks [chunk_lo, chunk_hi): residuals are
+ *                      written on those planes only, their loss partial sums go to their own slots
+ *                      of the workspace.  `finish` != 0: the loss vector is formed from the partial
+ *                      sums of ALL chunks, so this must be the last of a set of calls that share
+ *                      workspace and stream and together cover every chunk.  loss_rows = 0: the
+ *                      array's own row count.
+ *   fpde_bwd_chunks    fpde_bwd restricted to the chunks [chunk_lo, chunk_hi): gradients are written
+ *                      on those planes only (they read the upstream arrays and fields one plane
+ *                      beyond the range at either end).
+ * FPDE_ERR_SHAPE for an empty or out-of-range chunk range.
+ */
+int fpde_plane_chunk(int op, int ndim, const int64_t* shape);
+int fpde_fwd_chunks(int op,
+                    const float* const* fields,
+                    const float* const* sources,
+                    float* const* residuals,
+                    double* loss_out,
+                    int ndim, const int64_t* shape,
+                    const double* spacing,
+                    const double* coeffs, int ncoeffs,
+                    const int* bc,
+                    void* workspace, size_t workspace_bytes,
+                    void* stream,
+                    int64_t loss_rows,
+                    int chunk_lo, int chunk_hi, int finish);
+int fpde_bwd_chunks(int op,
+                    const float* const* fields,
+                    const float* const* gres,
+                    const double* gscale,
+                    float* const* gfields,
+                    int ndim, const int64_t* shape,
+                    const double* spacing,
+                    const double* coeffs, int ncoeffs,
+                    const int* bc,
+                    void* stream,
+                    int chunk_lo, int chunk_hi);
+
+/*
  * Discrete adjoint in gather form with boundary-gradient correction (Sections 2.2 and 2.3):
  * gfields[f] = sum_e J_{e,f}^T G_e with G_e = gscale[e] * gres[e] on the rows of residual e
  * and 0 elsewhere (entries of gres at nodes without a row are ignored).

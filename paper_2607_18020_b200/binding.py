@@ -63,11 +63,20 @@ def lib():
                                ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         L.fpde_fwd_rows.restype = ctypes.c_int
         L.fpde_fwd_rows.argtypes = L.fpde_fwd.argtypes + [ctypes.c_int64]
+        L.fpde_plane_chunk.restype = ctypes.c_int
+        L.fpde_plane_chunk.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
+        L.fpde_fwd_chunks.restype = ctypes.c_int
+        L.fpde_fwd_chunks.argtypes = L.fpde_fwd.argtypes + [ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int]
         L.fpde_bwd.restype = ctypes.c_int
         L.fpde_bwd.argtypes = [ctypes.c_int, vpp, vpp, ctypes.POINTER(ctypes.c_double), vpp, ctypes.c_int,
                                ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fpde_bwd_chunks.restype = ctypes.c_int
+        L.fpde_bwd_chunks.argtypes = [ctypes.c_int, vpp, vpp, ctypes.POINTER(ctypes.c_double), vpp, ctypes.c_int,
+                                      ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                      ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                                      ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
         L.fpde_has_single_pass.restype = ctypes.c_int
         L.fpde_has_single_pass.argtypes = [ctypes.c_int]
         L.fpde_fwd_bwd_workspace_bytes.restype = ctypes.c_size_t
@@ -326,6 +335,39 @@ def fpde_fwd_bwd(op, fields, sources, residuals, gfields, loss_out, shape, spaci
                             wsb, _stream_handle(stream))
     if st != FPDE_OK:
         raise FpdeError(st, "fpde_fwd_bwd")
+
+
+def plane_chunk(op, shape) -> int:
+    """Planes per chunk of the ranged launches for this operator and grid (0: the operator has none)."""
+    return int(lib().fpde_plane_chunk(_opid(op), len(shape), _i64(shape)))
+
+
+def fpde_fwd_chunks(op, fields, sources, residuals, loss_out, shape, spacing, coeffs, bc, workspace, loss_rows,
+                    chunk_lo, chunk_hi, finish, stream=None):
+    """fpde_fwd_rows over the chunks [chunk_lo, chunk_hi) of x-planes only (chunk length: plane_chunk());
+    `finish`: form the loss vector from the partial sums of all chunks (the last call of a set that
+    covers every chunk).  loss_rows = 0: the array's own row count."""
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    with _on_device_of(fields, sources, residuals, loss_out, workspace):
+        st = lib().fpde_fwd_chunks(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(sources)),
+                                   _ptr_array(_dev_ptrs(residuals)),
+                                   _dev_ptrs([loss_out])[0] if loss_out is not None else None, len(shape), _i64(shape),
+                                   _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                                   _dev_ptrs([workspace])[0] if workspace is not None else None, int(wsb),
+                                   _stream_handle(stream), int(loss_rows), int(chunk_lo), int(chunk_hi), int(bool(finish)))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_fwd_chunks")
+
+
+def fpde_bwd_chunks(op, fields, gres, gscale, gfields, shape, spacing, coeffs, bc, chunk_lo, chunk_hi, stream=None):
+    """fpde_bwd over the chunks [chunk_lo, chunk_hi) of x-planes only."""
+    with _on_device_of(fields, gres, gfields):
+        st = lib().fpde_bwd_chunks(_opid(op), _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(gres)),
+                                   _f64(gscale) if gscale is not None else None, _ptr_array(_dev_ptrs(gfields)),
+                                   len(shape), _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc),
+                                   _stream_handle(stream), int(chunk_lo), int(chunk_hi))
+    if st != FPDE_OK:
+        raise FpdeError(st, "fpde_bwd_chunks")
 
 
 def workspace_bytes_f64(op, shape) -> int:

@@ -17,6 +17,7 @@ namespace fpde {
 int lap2d_items(const int* n);
 int star3d_items(const int* n);
 int ns_items(const int* n, bool xint, int planes_per_item = 0);
+int ns_plane_chunk(const int* n, bool xint);
 int burgers_items(const int* n);
 int ns2d_items(const int* n);
 int ns3d_items(const int* n);
@@ -219,10 +220,12 @@ size_t fpde_workspace_bytes(int op, int ndim, const int64_t* shape) {
     return ((need + 255) / 256) * 256 + 4096;
 }
 
+// chunk_hi > chunk_lo: only the work items of those chunks of x-planes are launched (operators whose
+// launcher can do that), and the loss vector is formed only if `finish`.
 static int fwd_impl(int op, const float* const* fields, const float* const* sources, float* const* residuals,
                     double* loss_out, int ndim, const int64_t* shape, const double* spacing,
                     const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
-                    void* stream, int64_t loss_rows);
+                    void* stream, int64_t loss_rows, int chunk_lo = 0, int chunk_hi = 0, int finish = 1);
 
 int fpde_fwd(int op, const float* const* fields, const float* const* sources, float* const* residuals,
              double* loss_out, int ndim, const int64_t* shape, const double* spacing,
@@ -241,10 +244,22 @@ int fpde_fwd_rows(int op, const float* const* fields, const float* const* source
                     workspace_bytes, stream, loss_rows);
 }
 
+static bool has_plane_chunks(int op) { return op == FPDE_OP_NS_3D_T || op == FPDE_OP_NS_3D_T_XSLAB; }
+
+// planes per chunk of the ranged launches: the launcher's own choice for this grid
+static int plane_chunk_of(int op, const int* n) {
+    if (!has_plane_chunks(op)) return 0;
+    // shortened on short arrays until there are at least four chunks (never below four planes), so
+    // that a slab of a grid split many ways still has chunks away from its halo planes
+    int P = ns_plane_chunk(n, op == FPDE_OP_NS_3D_T_XSLAB);
+    while (P > 4 && (n[0] + P - 1) / P < 4) P = std::max(4, P / 2);
+    return P;
+}
+
 static int fwd_impl(int op, const float* const* fields, const float* const* sources, float* const* residuals,
                     double* loss_out, int ndim, const int64_t* shape, const double* spacing,
                     const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
-                    void* stream, int64_t loss_rows) {
+                    void* stream, int64_t loss_rows, int chunk_lo, int chunk_hi, int finish) {
     Problem q;
     std::memset(&q, 0, sizeof(q));
     int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
@@ -272,6 +287,24 @@ static int fwd_impl(int op, const float* const* fields, const float* const* sour
     q.stream = static_cast<cudaStream_t>(stream);
     cudaError_t ce = cudaSuccess;
     int items = 0;
+    if (chunk_hi > chunk_lo) {
+        // a range of plane chunks: fixed chunk length, partial sums in their global slots
+        const int P = plane_chunk_of(op, q.n);
+        if (P <= 0) return FPDE_ERR_BAD_OP;
+        const int nchunks = (q.n[0] + P - 1) / P;
+        if (chunk_lo < 0 || chunk_hi > nchunks) return FPDE_ERR_SHAPE;
+        q.planes_per_item = P; q.chunk_lo = chunk_lo; q.chunk_hi = chunk_hi;
+        if (loss_out && workspace_bytes < (size_t)ns_items(q.n, q.bc0_interior, P) * e.ne * sizeof(float))
+            return FPDE_ERR_WORKSPACE;
+        ce = launch_ns_fwd(q);
+        if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+        if (loss_out && finish) {
+            ce = launch_loss_finalize(q.partials, ns_items(q.n, q.bc0_interior, P), e.ne, loss_rows > 0 ? loss_rows : q.rows,
+                                      loss_out, q.stream);
+            if (ce != cudaSuccess) return FPDE_ERR_CUDA;
+        }
+        return FPDE_OK;
+    }
     switch (op) {
     case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_fwd(q); items = burgers_items(q.n); break;
     case FPDE_OP_POISSON_2D:
@@ -293,7 +326,8 @@ static int fwd_impl(int op, const float* const* fields, const float* const* sour
 
 static int bwd_impl(int op, const float* const* fields, const float* const* gres, const double* gscale,
                     float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
-                    const double* coeffs, int ncoeffs, const int* bc, void* stream, bool gres_zero_off_rows);
+                    const double* coeffs, int ncoeffs, const int* bc, void* stream, bool gres_zero_off_rows,
+                    int chunk_lo = 0, int chunk_hi = 0);
 
 int fpde_bwd(int op, const float* const* fields, const float* const* gres, const double* gscale,
              float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
@@ -303,9 +337,35 @@ int fpde_bwd(int op, const float* const* fields, const float* const* gres, const
     return bwd_impl(op, fields, gres, gscale, gfields, ndim, shape, spacing, coeffs, ncoeffs, bc, stream, false);
 }
 
+int fpde_plane_chunk(int op, int ndim, const int64_t* shape) {
+    int n[MAX_D] = {0, 0, 0, 0};
+    if (check_shape(op, ndim, shape, n, nullptr, nullptr) != FPDE_OK) return 0;
+    return plane_chunk_of(op, n);
+}
+
+int fpde_fwd_chunks(int op, const float* const* fields, const float* const* sources, float* const* residuals,
+                    double* loss_out, int ndim, const int64_t* shape, const double* spacing,
+                    const double* coeffs, int ncoeffs, const int* bc, void* workspace, size_t workspace_bytes,
+                    void* stream, int64_t loss_rows, int chunk_lo, int chunk_hi, int finish) {
+    if (op < 0 || op >= FPDE_OP_COUNT || !has_plane_chunks(op)) return FPDE_ERR_BAD_OP;
+    if (chunk_hi <= chunk_lo || loss_rows < 0) return FPDE_ERR_SHAPE;
+    return fwd_impl(op, fields, sources, residuals, loss_out, ndim, shape, spacing, coeffs, ncoeffs, bc, workspace,
+                    workspace_bytes, stream, loss_rows, chunk_lo, chunk_hi, finish);
+}
+
+int fpde_bwd_chunks(int op, const float* const* fields, const float* const* gres, const double* gscale,
+                    float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
+                    const double* coeffs, int ncoeffs, const int* bc, void* stream, int chunk_lo, int chunk_hi) {
+    if (op < 0 || op >= FPDE_OP_COUNT || !has_plane_chunks(op)) return FPDE_ERR_BAD_OP;
+    if (chunk_hi <= chunk_lo) return FPDE_ERR_SHAPE;
+    return bwd_impl(op, fields, gres, gscale, gfields, ndim, shape, spacing, coeffs, ncoeffs, bc, stream, false,
+                    chunk_lo, chunk_hi);
+}
+
 static int bwd_impl(int op, const float* const* fields, const float* const* gres, const double* gscale,
                     float* const* gfields, int ndim, const int64_t* shape, const double* spacing,
-                    const double* coeffs, int ncoeffs, const int* bc, void* stream, bool gres_zero_off_rows) {
+                    const double* coeffs, int ncoeffs, const int* bc, void* stream, bool gres_zero_off_rows,
+                    int chunk_lo, int chunk_hi) {
     Problem q;
     std::memset(&q, 0, sizeof(q));
     int st = validate(op, fields, ndim, shape, spacing, coeffs, ncoeffs, bc, q);
@@ -327,6 +387,13 @@ static int bwd_impl(int op, const float* const* fields, const float* const* gres
     q.stream = static_cast<cudaStream_t>(stream);
     q.gres_zero_off_rows = gres_zero_off_rows;
     cudaError_t ce = cudaSuccess;
+    if (chunk_hi > chunk_lo) {
+        const int P = plane_chunk_of(op, q.n);
+        if (P <= 0) return FPDE_ERR_BAD_OP;
+        if (chunk_lo < 0 || chunk_hi > (q.n[0] + P - 1) / P) return FPDE_ERR_SHAPE;
+        q.planes_per_item = P; q.chunk_lo = chunk_lo; q.chunk_hi = chunk_hi;
+        return launch_ns_bwd(q) == cudaSuccess ? FPDE_OK : FPDE_ERR_CUDA;
+    }
     switch (op) {
     case FPDE_OP_BURGERS_1D_T: ce = launch_burgers_bwd(q); break;
     case FPDE_OP_POISSON_2D:

@@ -320,6 +320,16 @@ int ns_items(const int* n, bool xint, int planes_per_item) {
     return p.nitems;
 }
 
+// Planes per work item the launcher chooses for this grid when the caller names none.
+int ns_plane_chunk(const int* n, bool xint) {
+    Problem q{};
+    for (int a = 0; a < 4; ++a) { q.n[a] = n[a]; q.h[a] = 1.0; }
+    q.bc0_interior = xint;
+    NsParams p{}; dim3 block;
+    ns_geometry(q, p, block);
+    return p.planes_per_item;
+}
+
 cudaError_t launch_ns_fwd(const Problem& q) {
     if (!q.bc0_interior && q.planes_per_item == 0) {
         bool launched = false;

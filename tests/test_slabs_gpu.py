@@ -90,3 +90,50 @@ def test_step_dist_with_one_rank():
     assert abs(float(loss[-1]) - loss_ref[-1]) <= LOSS_TOL * abs(loss_ref[-1])
     for f, g in enumerate(rank.owned(rank.grads)):
         assert_close(g.cpu().numpy(), g_ref[f], "one-rank slab gradient %d" % f)
+
+
+@pytest.mark.parametrize("name,shape", [("ns_tgv_128x16", (23, 8, 8, 8)), ("ns_tgv_xslab_34", (30, 6, 8, 16))])
+def test_launches_over_plane_chunks_add_up_to_the_full_launch(name, shape):
+    """fpde_fwd_chunks / fpde_bwd_chunks over a partition of the chunks of x-planes, in any order, write
+    what one full launch writes, bit for bit, and the loss formed by the last call is the full launch's."""
+    w = W.make(name, seed=44, shape=shape, kind="randn")
+    fields, sources, res_w, loss_w = run_fwd(torch, w)
+    rows = B.row_count(w.op, w.shape)
+    grads_w = run_bwd(torch, w, fields, [r.view for r in res_w], [2.0 / rows] * len(res_w))
+    P = B.plane_chunk(w.op, w.shape)
+    assert P > 0
+    K = -(-shape[0] // P)
+    assert K >= 3
+    res = [torch.full(shape, 7.0, dtype=torch.float32, device="cuda") for _ in res_w]
+    grads = [torch.full(shape, 9.0, dtype=torch.float32, device="cuda") for _ in fields]
+    loss = torch.full((len(res) + 1,), -1.0, dtype=torch.float64, device="cuda")
+    ws = torch.empty(B.workspace_bytes(w.op, shape), dtype=torch.uint8, device="cuda")
+    parts = [(1, K - 1), (K - 1, K), (0, 1)]                    # inner chunks first, then the two ends
+    for i, (lo, hi) in enumerate(parts):
+        B.fpde_fwd_chunks(w.op, fields, sources, res, loss, shape, w.spacing, w.coeffs, w.bc, ws, 0, lo, hi,
+                          i == len(parts) - 1)
+    for lo, hi in parts:
+        B.fpde_bwd_chunks(w.op, fields, res, [2.0 / rows] * len(res), grads, shape, w.spacing, w.coeffs, w.bc, lo, hi)
+    torch.cuda.synchronize()
+    for a, b in zip(res, res_w):
+        assert torch.equal(a, b.view)
+    for a, b in zip(grads, grads_w):
+        assert torch.equal(a, b.view)
+    assert torch.equal(loss, loss_w)
+    assert B.plane_chunk(W.HELMHOLTZ_3D_O4, (32, 32, 32)) == 0
+
+
+def test_step_dist_overlap_plan_on_one_rank():
+    """One rank, a slab long enough to have chunks of planes away from its halos: the step that queues
+    those chunks before waiting for the halo planes gives the oracle's loss and gradients."""
+    w = W.make("ns_tgv_128x16", seed=45, shape=(26, 8, 8, 8), kind="randn")
+    rank = S.SlabRank(torch, B, S.plans(w.op, w.shape, 1)[0], w.spacing, w.coeffs)
+    rank.load_owned(w.fields, w.sources)
+    plan = rank.chunk_plan()
+    assert plan is not None and plan[0][1] >= 1 and plan[0][2] < plan[0][0] and plan[1][2] > plan[1][1]
+    loss = S.step_dist(rank, dist=None, overlap=True)
+    torch.cuda.synchronize()
+    _, loss_ref, g_ref, _ = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    assert np.all(np.abs(loss.cpu().numpy() - loss_ref) <= LOSS_TOL * np.abs(loss_ref))
+    for f, g in enumerate(rank.owned(rank.grads)):
+        assert_close(g.cpu().numpy(), g_ref[f], "overlapped one-rank slab gradient %d" % f)

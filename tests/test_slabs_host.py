@@ -8,6 +8,7 @@ import sys
 import numpy as np
 import pytest
 
+from paper_2607_18020_b200 import binding as B
 from paper_2607_18020_b200 import slabs as S
 from paper_2607_18020_b200 import workloads as W
 
@@ -128,3 +129,28 @@ def test_exchange_between_two_gloo_ranks(op, shape):
     import torch.multiprocessing as mp
     s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
     mp.spawn(_rank_main, args=(2, port, op, shape), nprocs=2, join=True)
+
+
+def test_chunk_plan_keeps_inner_launches_off_the_halo_planes():
+    """The launches queued while the halo planes are in flight must neither cover nor read a plane an
+    exchange fills: checked plane by plane from the chunk length the library reports."""
+    for shape, world in (((128, 128, 128, 16), 2), ((128, 128, 128, 16), 4), ((121, 16, 16, 16), 1), ((50, 8, 8, 8), 2)):
+        for plan in S.plans(W.NS_3D_T, shape, world):
+            rank = S.SlabRank(torch, B, plan, (0.1,) * 4, (0.01,), device="cpu")
+            cp = rank.chunk_plan()
+            assert cp is not None, (shape, world)
+            R = plan.radius
+            for (K, lo, hi), n, halo_lo in ((cp[0], plan.tight_shape[0], range(0, R)),
+                                            (cp[1], plan.local_shape[0], range(R, 2 * R))):
+                P = B.plane_chunk(plan.local_op, (n,) + tuple(shape[1:]))
+                assert K == -(-n // P) and 1 <= lo < hi < K
+                halo = set(halo_lo) | {n - 1 - h for h in halo_lo}
+                read = set()
+                for a in range(lo * P, min(hi * P, n)):
+                    read.update(range(a - R, a + R + 1))
+                assert not (read & halo), (shape, world, plan.rank, sorted(read & halo))
+    # an operator without launches over plane ranges, and a slab too short to have inner chunks
+    short = S.SlabRank(torch, B, S.plans(W.NS_3D_T, (8, 8, 8, 8), 2)[0], (0.1,) * 4, (0.01,), device="cpu")
+    assert short.chunk_plan() is None
+    hh = S.SlabRank(torch, B, S.plans(W.HELMHOLTZ_3D_O4, (64, 16, 16), 2)[0], (0.1,) * 3, (1.0,), device="cpu")
+    assert hh.chunk_plan() is None
