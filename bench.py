@@ -51,7 +51,7 @@ KERNEL_NAMES = {                    # op: (fwd kernel, bwd kernel)
     W.BURGERS_1D_T: ("burgers_fwd_kernel", "burgers_bwd_kernel"),
     W.POISSON_2D: ("lap2d_kernel<PoissonFwd>", "lap2d_kernel<PoissonBwd>"),
     W.GRAYSCOTT_2D: ("lap2d_kernel<GrayScottFwd>", "lap2d_kernel<GrayScottBwd>"),
-    W.HELMHOLTZ_3D_O4: ("star3d_kernel<fwd>", "star3d_kernel<bwd>"),
+    W.HELMHOLTZ_3D_O4: ("star3d_kernel<fwd>", "star3d_tma_kernel<bwd>"),
     W.NS_3D_T: ("ns_fwd_kernel", "ns_bwd_kernel"),
     W.NS_2D_STEADY: ("ns2d_kernel<fwd>", "ns2d_kernel<bwd>"),
     W.NS_3D_STEADY: ("ns3d_kernel<fwd>", "ns3d_kernel<bwd>"),
@@ -64,8 +64,8 @@ NCU_TRAFFIC_BYTES = {
     ("ns_tgv_128x16", "ns_bwd_kernel"): 2 * 762521088,
     ("grayscott_4096", "lap2d_kernel<GrayScottFwd>"): 222671616,
     ("grayscott_4096", "lap2d_kernel<GrayScottBwd>"): 366043648,
-    ("helmholtz_256", "star3d_kernel<fwd>"): 169988352,
-    ("helmholtz_256", "star3d_kernel<bwd>"): 97383424,
+    ("helmholtz_256", "star3d_kernel<fwd>"): 171900000,
+    ("helmholtz_256", "star3d_tma_kernel<bwd>"): 97610000,
     ("ns2d_steady_4096", "ns2d_kernel<fwd>"): 362135040,
     ("ns2d_steady_4096", "ns2d_kernel<bwd>"): 511582720,
     ("ns3d_steady_256", "ns3d_kernel<fwd>"): 516224256,
