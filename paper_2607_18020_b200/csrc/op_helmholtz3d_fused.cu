@@ -72,8 +72,8 @@ __device__ __forceinline__ void hf_star_step(const V4 (&L)[RY + 4], const float2
         V4 s1z, s2z;
         s1z.lo = make_float2(zl[j].y + c.lo.y, c.lo.x + c.hi.x);
         s1z.hi = make_float2(c.lo.y + c.hi.y, c.hi.x + zr[j].x);
-        s2z.lo = make_float2(zl[j].x + c.hi.x, zl[j].y + c.hi.y);
-        s2z.hi = make_float2(c.lo.x + zr[j].x, c.lo.y + zr[j].y);
+        s2z.lo = add2(zl[j], c.hi);                          // (z-2, z-1) + (z+2, z+3): both register pairs
+        s2z.hi = add2(c.lo, zr[j]);
         A2[j] = v4fma(s1y, w.w16y, A2[j]);
         A2[j] = v4fma(s2y, w.nwy, A2[j]);
         A2[j] = v4fma(c, w.kc, A2[j]);

@@ -192,8 +192,8 @@ star3d_tma_kernel(const __grid_constant__ Star3dTmaParams p) {
                     V4 s1z, s2z;
                     s1z.lo = make_float2(zl[j].y + c.lo.y, c.lo.x + c.hi.x);
                     s1z.hi = make_float2(c.lo.y + c.hi.y, c.hi.x + zr[j].x);
-                    s2z.lo = make_float2(zl[j].x + c.hi.x, zl[j].y + c.hi.y);
-                    s2z.hi = make_float2(c.lo.x + zr[j].x, c.lo.y + zr[j].y);
+                    s2z.lo = add2(zl[j], c.hi);                          // (z-2, z-1) + (z+2, z+3): both register pairs
+                    s2z.hi = add2(c.lo, zr[j]);
                     if (MODE == 1) {
                         // the y neighbours in the z band are zero too: their sum is formed apart and masked
                         V4 py = v4mul(s1y, w16y);

@@ -99,3 +99,34 @@ def test_random_shape_adjoint_of_arbitrary_upstream_arrays(name, shape, seed):
     for f, (g, gr) in enumerate(zip(out, ref64)):
         d = np.abs(g.cpu().numpy() - gr).max()
         assert d <= 1e-11 * max(1.0, np.abs(gr).max()), "%s%s fp64 adjoint %d: %g" % (name, shape, f, d)
+
+
+def _staged_helmholtz_shapes():
+    """Randomly drawn grids wide enough for the shared-memory staged Helmholtz engine (z lines of 136
+    floats and more, 40 rows and more), fixed seed: ragged tiles in y and z, few and many planes."""
+    rng = np.random.RandomState(20261125)
+    out = []
+    for _ in range(10):
+        out.append((int(rng.randint(8, 40)), int(rng.randint(40, 90)), 4 * int(rng.randint(34, 100))))
+    return out
+
+
+@pytest.mark.parametrize("shape", _staged_helmholtz_shapes())
+def test_fuzz_staged_helmholtz_engine(shape, monkeypatch):
+    """Forward on the staged engine too (FPDE_STAR3D_TMA_FWD=1), adjoint of the residuals and of an
+    arbitrary upstream array with entries off the rows, against the oracle."""
+    monkeypatch.setenv("FPDE_STAR3D_TMA", "1")
+    monkeypatch.setenv("FPDE_STAR3D_TMA_FWD", "1")
+    w = W.make("helmholtz_256", seed=50, shape=shape, kind="randn")
+    R_ref, loss_ref, g_ref, rows = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    fields, sources, res, loss = run_fwd(torch, w)
+    assert_close(res[0].view.cpu().numpy(), R_ref[0], "staged helmholtz %s residual" % (shape,))
+    assert np.all(np.abs(loss.cpu().numpy() - loss_ref) <= LOSS_TOL * np.abs(loss_ref))
+    grads = run_bwd(torch, w, fields, [res[0].view], [2.0 / rows])
+    assert_close(grads[0].view.cpu().numpy(), g_ref[0], "staged helmholtz %s gradient" % (shape,))
+    rng = np.random.default_rng(7)
+    G = rng.standard_normal(shape).astype(np.float32)
+    g2_ref = oracle.bwd(w.op, w.fields, [G.astype(np.float64) * 0.5], w.shape, w.spacing, w.coeffs)
+    grads2 = run_bwd(torch, w, fields, to_dev(torch, [G]), [0.5])
+    assert_close(grads2[0].view.cpu().numpy(), g2_ref[0], "staged helmholtz %s arbitrary upstream" % (shape,))
+    assert B.diag_tma_timeouts() == 0
