@@ -294,24 +294,23 @@ class DeviceProblem:
         self.loss = torch.zeros(ne + 1, dtype=torch.float64, device="cuda")
         self.ws = torch.empty(B.workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
         self.gscale = [2.0 / B.row_count(w.op, w.shape)] * ne
-        self.ws2 = None
+
+        # the C arguments of the three calls, marshalled once: on small grids the per-call marshalling
+        # costs more host time than the kernels take
+        self.ws2 = torch.empty(B.fwd_bwd_workspace_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+        self.step = B.PreparedStep(w.op, self.fields, self.sources, self.res, self.grads, self.loss, w.shape, w.spacing,
+                                   w.coeffs, w.bc, workspace=self.ws, gscale=self.gscale, fwd_bwd_workspace=self.ws2)
+        self._store_res = not B.has_single_pass(w.op)          # two-kernel operators need the intermediate
 
     def fwd(self):
-        w = self.w
-        self.B.fpde_fwd(w.op, self.fields, self.sources, self.res, self.loss, w.shape, w.spacing, w.coeffs, w.bc, self.ws)
+        self.step.fwd()
 
     def bwd(self):
-        w = self.w
-        self.B.fpde_bwd(w.op, self.fields, self.res, self.gscale, self.grads, w.shape, w.spacing, w.coeffs, w.bc)
+        self.step.bwd()
 
     def fwd_bwd(self):
         """The loss-specialised pass: loss + dL/dfield, residual arrays not stored."""
-        w = self.w
-        if self.ws2 is None:
-            self.ws2 = self.torch.empty(self.B.fwd_bwd_workspace_bytes(w.op, w.shape), dtype=self.torch.uint8, device="cuda")
-        res = None if self.B.has_single_pass(w.op) else self.res      # two-kernel operators need the intermediate
-        self.B.fpde_fwd_bwd(w.op, self.fields, self.sources, res, self.grads, self.loss, w.shape, w.spacing,
-                            w.coeffs, w.bc, self.ws2)
+        self.step.fwd_bwd(store_residuals=self._store_res)
 
 
 class SlabProblem:

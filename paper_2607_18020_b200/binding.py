@@ -370,6 +370,67 @@ def fpde_bwd_chunks(op, fields, gres, gscale, gfields, shape, spacing, coeffs, b
         raise FpdeError(st, "fpde_bwd_chunks")
 
 
+class PreparedStep:
+    """The arguments of fpde_fwd / fpde_bwd / fpde_fwd_bwd for one set of tensors, marshalled ONCE.
+
+    Turning tensors into pointer arrays costs more host time than a small grid's kernels take on the
+    GPU (tens of microseconds per call against a few); a training loop calls the same operator on the
+    same tensors every step, so this object builds the C arguments once and each `fwd()` / `bwd()` /
+    `fwd_bwd()` is then a single foreign call on torch's current stream.  Pure marshalling: every
+    step still runs in the library's kernels.  The tensors must stay alive and in place."""
+
+    def __init__(self, op, fields, sources, residuals, gfields, loss_out, shape, spacing, coeffs, bc,
+                 workspace=None, gscale=None, fwd_bwd_workspace=None):
+        self._keep = (fields, sources, residuals, gfields, loss_out, workspace, fwd_bwd_workspace)
+        _on_device_of(fields, sources, residuals, gfields, loss_out, workspace, fwd_bwd_workspace)   # one device?
+        self._idx = fields[0].device.index
+        L = lib()
+        self._op = _opid(op)
+        self._nd = len(shape)
+        self._f, self._s = _ptr_array(_dev_ptrs(fields)), _ptr_array(_dev_ptrs(sources))
+        self._r = _ptr_array(_dev_ptrs(residuals)) if residuals is not None else None
+        self._g = _ptr_array(_dev_ptrs(gfields)) if gfields is not None else None
+        self._loss = _dev_ptrs([loss_out])[0] if loss_out is not None else None
+        self._shape, self._h, self._c, self._nc, self._bc = _i64(shape), _f64(spacing), _f64(coeffs), len(coeffs), _bcs(bc)
+        self._ws = _dev_ptrs([workspace])[0] if workspace is not None else None
+        self._wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        self._ws2 = _dev_ptrs([fwd_bwd_workspace])[0] if fwd_bwd_workspace is not None else None
+        self._wsb2 = fwd_bwd_workspace.numel() * fwd_bwd_workspace.element_size() if fwd_bwd_workspace is not None else 0
+        if gscale is None and residuals is not None:
+            rows = L.fpde_row_count(self._op, self._nd, self._shape)
+            gscale = [2.0 / rows] * len(residuals)
+        self._gs = _f64(gscale) if gscale is not None else None
+        self._fwd, self._bwd, self._fb = L.fpde_fwd, L.fpde_bwd, L.fpde_fwd_bwd
+        import torch
+        self._torch = torch
+
+    def _call(self, fn, name, *args):
+        t = self._torch
+        if t.cuda.current_device() == self._idx:        # the usual case: no device switch needed
+            st = fn(*args, t.cuda.current_stream().cuda_stream)
+        else:
+            with t.cuda.device(self._idx):
+                st = fn(*args, t.cuda.current_stream().cuda_stream)
+        if st != FPDE_OK:
+            raise FpdeError(st, name)
+
+    def fwd(self):
+        """fpde_fwd(fields, sources -> residuals, loss) on the current stream."""
+        self._call(self._fwd, "fpde_fwd", self._op, self._f, self._s, self._r, self._loss, self._nd, self._shape,
+                   self._h, self._c, self._nc, self._bc, self._ws, self._wsb)
+
+    def bwd(self):
+        """fpde_bwd with the residual arrays as upstream arrays and the prepared scales (default 2/N_r:
+        the gradient of the fused loss) -> gfields."""
+        self._call(self._bwd, "fpde_bwd", self._op, self._f, self._r, self._gs, self._g, self._nd, self._shape,
+                   self._h, self._c, self._nc, self._bc, None, 0)
+
+    def fwd_bwd(self, store_residuals=True):
+        """fpde_fwd_bwd: loss and gradient from one call."""
+        self._call(self._fb, "fpde_fwd_bwd", self._op, self._f, self._s, self._r if store_residuals else None, self._g,
+                   self._loss, self._nd, self._shape, self._h, self._c, self._nc, self._bc, self._ws2, self._wsb2)
+
+
 def workspace_bytes_f64(op, shape) -> int:
     return int(lib().fpde_workspace_bytes_f64(_opid(op), len(shape), _i64(shape)))
 

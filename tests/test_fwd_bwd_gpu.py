@@ -159,3 +159,38 @@ def test_helmholtz_single_pass_prototype(shape, store_res, monkeypatch):
         res.check()
         assert_close(res.view.cpu().numpy(), R_ref[0], "helmholtz single pass %s residual" % (shape,))
     assert B.diag_tma_timeouts() == 0
+
+
+@pytest.mark.parametrize("name,shape", [("poisson_1024", (40, 48)), ("ns_tgv_128x16", (9, 8, 8, 8)), ("grayscott_4096", (48, 64))])
+def test_prepared_step_is_the_same_calls_with_the_arguments_marshalled_once(name, shape):
+    """PreparedStep.fwd / bwd / fwd_bwd give bit for bit what fpde_fwd / fpde_bwd / fpde_fwd_bwd give."""
+    w = W.make(name, seed=51, shape=shape, kind="randn")
+    fields, sources = to_dev(torch, w.fields), to_dev(torch, w.sources)
+    ne = len(W.OP_META[w.op]["residuals"])
+    mk = lambda n: [torch.full(shape, 3.0, dtype=torch.float32, device="cuda") for _ in range(n)]
+    res_a, res_b, g_a, g_b, g_c, g_d = mk(ne), mk(ne), mk(len(fields)), mk(len(fields)), mk(len(fields)), mk(len(fields))
+    loss_a = torch.zeros(ne + 1, dtype=torch.float64, device="cuda"); loss_b = loss_a.clone() - 1
+    loss_c = loss_a.clone() - 2; loss_d = loss_a.clone() - 3
+    ws = torch.empty(B.workspace_bytes(w.op, shape), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty(B.fwd_bwd_workspace_bytes(w.op, shape), dtype=torch.uint8, device="cuda")
+    rows = B.row_count(w.op, shape)
+    B.fpde_fwd(w.op, fields, sources, res_a, loss_a, shape, w.spacing, w.coeffs, w.bc, ws)
+    B.fpde_bwd(w.op, fields, res_a, [2.0 / rows] * ne, g_a, shape, w.spacing, w.coeffs, w.bc)
+    step = B.PreparedStep(w.op, fields, sources, res_b, g_b, loss_b, shape, w.spacing, w.coeffs, w.bc, workspace=ws,
+                          fwd_bwd_workspace=ws2)
+    step.fwd(); step.bwd()
+    torch.cuda.synchronize()
+    for a, b in zip(res_a + g_a, res_b + g_b):
+        assert torch.equal(a, b)
+    assert torch.equal(loss_a, loss_b)
+    # the one-call entry point, through the binding and through the prepared step
+    store = not B.has_single_pass(w.op)
+    res_c, res_d = mk(ne), mk(ne)
+    B.fpde_fwd_bwd(w.op, fields, sources, res_c if store else None, g_c, loss_c, shape, w.spacing, w.coeffs, w.bc, ws2)
+    step2 = B.PreparedStep(w.op, fields, sources, res_d, g_d, loss_d, shape, w.spacing, w.coeffs, w.bc, workspace=ws,
+                           fwd_bwd_workspace=ws2)
+    step2.fwd_bwd(store_residuals=store)
+    torch.cuda.synchronize()
+    for a, b in zip(g_c, g_d):
+        assert torch.equal(a, b)
+    assert torch.equal(loss_c, loss_d)
