@@ -279,16 +279,14 @@ static int env_int(const char* name, int dflt) {
 
 constexpr int S3T_MAX_CTAS = 2048;       // upper bound of the grid (= loss partial sums a launch may write)
 
-struct S3tShape { int tyb, ry, st; };
+struct S3tShape { int tyb, ry; };
+constexpr int S3T_STAGES = 6;            // ring depth (4, 6 and 8 measured within a microsecond of one another)
 
-// Launch shape: rows per block / per thread and ring depth.
-static S3tShape s3t_shape(bool fwd) {
+// Launch shape: rows per block / per thread.
+static S3tShape s3t_shape() {
     S3tShape g;
-    const int tyb = env_int("FPDE_STAR3D_TMA_TYB", 8);
-    g.tyb = tyb >= 32 ? 32 : (tyb >= 16 ? 16 : 8);
+    g.tyb = env_int("FPDE_STAR3D_TMA_TYB", 8) >= 16 ? 16 : 8;
     g.ry = env_int("FPDE_STAR3D_TMA_RY", 2) >= 4 ? 4 : 2;
-    const int st = env_int("FPDE_STAR3D_TMA_STAGES", 6);
-    g.st = st >= 8 ? 8 : (st >= 6 ? 6 : 4);
     return g;
 }
 
@@ -296,7 +294,7 @@ static S3tShape s3t_shape(bool fwd) {
 // full tile in z and y.  FPDE_STAR3D_TMA=0 selects the L1-staged engine everywhere.
 bool star3d_tma_wanted(const int* n) {
     if (env_int("FPDE_STAR3D_TMA", 1) == 0 || tma_encode_fn() == nullptr) return false;
-    return n[2] >= S3T_WP && n[1] >= 32 + 8 && n[0] >= 8;
+    return n[2] >= S3T_WP && n[1] >= 16 + 8 && n[0] >= 8;
 }
 
 int star3d_tma_items(const int*) { return S3T_MAX_CTAS; }
@@ -335,22 +333,13 @@ static cudaError_t s3t_launch(const Problem& q, Star3dTmaParams& p, int* items) 
     return launch_kernel_smem(kern, dim3((unsigned)G), dim3(threads, 1, 1), smem, q.stream, p);
 }
 
-template <int MODE, int TYB, int RY>
-static cudaError_t s3t_dispatch_st(const Problem& q, Star3dTmaParams& p, int st, int* items) {
-    constexpr int MINB = TYB == 8 ? 3 : (TYB == 16 ? 2 : 1);        // CTAs per SM the register budget is set for
-    if (st == 8) return s3t_launch<MODE, TYB, RY, 8, MINB>(q, p, items);
-    if (st == 6) return s3t_launch<MODE, TYB, RY, 6, MINB>(q, p, items);
-    return s3t_launch<MODE, TYB, RY, 4, MINB>(q, p, items);
-}
-
 template <int MODE>
 static cudaError_t s3t_dispatch(const Problem& q, Star3dTmaParams& p, const S3tShape& g, int* items) {
-    if (g.tyb == 32 && g.ry == 4) return s3t_dispatch_st<MODE, 32, 4>(q, p, g.st, items);
-    if (g.tyb == 32) return s3t_dispatch_st<MODE, 32, 2>(q, p, g.st, items);
-    if (g.tyb == 16 && g.ry == 4) return s3t_dispatch_st<MODE, 16, 4>(q, p, g.st, items);
-    if (g.tyb == 16) return s3t_dispatch_st<MODE, 16, 2>(q, p, g.st, items);
-    if (g.ry == 4) return s3t_dispatch_st<MODE, 8, 4>(q, p, g.st, items);
-    return s3t_dispatch_st<MODE, 8, 2>(q, p, g.st, items);
+    // CTAs per SM the register budget is set for: 3 with 8-row tiles, 2 with 16-row tiles
+    if (g.tyb == 16 && g.ry == 4) return s3t_launch<MODE, 16, 4, S3T_STAGES, 2>(q, p, items);
+    if (g.tyb == 16) return s3t_launch<MODE, 16, 2, S3T_STAGES, 2>(q, p, items);
+    if (g.ry == 4) return s3t_launch<MODE, 8, 4, S3T_STAGES, 3>(q, p, items);
+    return s3t_launch<MODE, 8, 2, S3T_STAGES, 3>(q, p, items);
 }
 
 // mode as in the kernel.  `launched` false (with cudaSuccess) = this grid runs on the other engine.
@@ -362,7 +351,7 @@ cudaError_t launch_star3d_tma(const Problem& q, int mode, int* items, bool& laun
     if (!star3d_tma_wanted(q.n)) return cudaSuccess;
     if (mode == 0 && env_int("FPDE_STAR3D_TMA_FWD", 0) == 0) return cudaSuccess;
     const bool fwd = mode == 0;
-    const S3tShape g = s3t_shape(fwd);
+    const S3tShape g = s3t_shape();
     Star3dTmaParams p{};
     p.n0 = q.n[0]; p.n1 = q.n[1]; p.n2 = q.n[2]; p.nc4 = q.n[2] / 4;
     p.ncb = (p.n2 + S3T_TZ - 1) / S3T_TZ;
