@@ -209,11 +209,11 @@ def cpu_baseline_all_cores(name: str, planes_per_worker: int, reps: int = 2):
     """P = os.cpu_count() processes, each running the single-thread oracle on its own sample at the
     same time; aggregate points per second over the window from the first start to the last end."""
     import multiprocessing as mp
-    P = os.cpu_count() or 1
+    P = min(os.cpu_count() or 1, 64)                # one process per host core (at most 64: each holds ~250 MB)
     n0 = W.CONFIGS[name]["shape"][0]
     planes = max(5, min(planes_per_worker, n0))
     ctx = mp.get_context("spawn")
-    t_go = time.time() + 8.0                        # imports, sample generation and the warm-up pass come first
+    t_go = time.time() + 8.0 + 0.1 * P                      # imports, sample generation and the warm-up pass come first
     with ctx.Pool(P) as pool:
         out = pool.map(_oracle_worker, [(name, planes, 1042 + i, reps, t_go) for i in range(P)], chunksize=1)
     t_first, t_last = min(o[0] for o in out), max(o[1] for o in out)
