@@ -61,6 +61,15 @@ static int check_shape(int op, int ndim, const int64_t* shape, int* n_out, int64
     return FPDE_OK;
 }
 
+// Planes per chunk of the launches over ranges of x-planes (unsteady NS): the launcher's own choice
+// for this grid, shortened on short arrays until there are at least four chunks (never below four
+// planes), so that a slab of a grid split many ways still has chunks away from its halo planes.
+static int ranged_plane_chunk(const int* n, bool xint) {
+    int P = ns_plane_chunk(n, xint);
+    while (P > 4 && (n[0] + P - 1) / P < 4) P = std::max(4, P / 2);
+    return P;
+}
+
 static size_t workspace_need(int op, const int* n) {
     int items = 0;
     switch (op) {
@@ -69,8 +78,9 @@ static size_t workspace_need(int op, const int* n) {
     case FPDE_OP_GRAYSCOTT_2D:
     case FPDE_OP_GRAYSCOTT_2D_XSLAB: items = lap2d_items(n); break;
     case FPDE_OP_HELMHOLTZ_3D_O4: items = star3d_items(n); break;
-    case FPDE_OP_NS_3D_T: items = ns_items(n, false); break;
-    case FPDE_OP_NS_3D_T_XSLAB: items = ns_items(n, true); break;
+    // (the launches over ranges of plane chunks may use a shorter chunk, i.e. more partial sums)
+    case FPDE_OP_NS_3D_T: items = std::max(ns_items(n, false), ns_items(n, false, ranged_plane_chunk(n, false))); break;
+    case FPDE_OP_NS_3D_T_XSLAB: items = std::max(ns_items(n, true), ns_items(n, true, ranged_plane_chunk(n, true))); break;
     case FPDE_OP_NS_2D_STEADY: items = ns2d_items(n); break;
     case FPDE_OP_NS_3D_STEADY: items = ns3d_items(n); break;
     }
@@ -249,11 +259,7 @@ static bool has_plane_chunks(int op) { return op == FPDE_OP_NS_3D_T || op == FPD
 // planes per chunk of the ranged launches: the launcher's own choice for this grid
 static int plane_chunk_of(int op, const int* n) {
     if (!has_plane_chunks(op)) return 0;
-    // shortened on short arrays until there are at least four chunks (never below four planes), so
-    // that a slab of a grid split many ways still has chunks away from its halo planes
-    int P = ns_plane_chunk(n, op == FPDE_OP_NS_3D_T_XSLAB);
-    while (P > 4 && (n[0] + P - 1) / P < 4) P = std::max(4, P / 2);
-    return P;
+    return ranged_plane_chunk(n, op == FPDE_OP_NS_3D_T_XSLAB);
 }
 
 static int fwd_impl(int op, const float* const* fields, const float* const* sources, float* const* residuals,
