@@ -25,7 +25,7 @@
 // in 30 us; the consumers alone, computing on whatever is in shared memory, take 21-23 us -- with
 // about 90 executed instructions per output float4 (a third of them the packed arithmetic) they
 // are bound by instruction issue at 0.4-0.5 per cycle and scheduler, as the L1-staged kernels
-// are.  Together: adjoint 26.7 us (L1-staged: 29.5), forward 39 us (L1-staged: 34, within a
+// are.  Together: adjoint 24.8 us (L1-staged: 29.5), forward 36 us (L1-staged: 34, within a
 // tenth of its DRAM time), so the adjoint runs here by default and the forward pass does not.
 //
 // Every wait is bounded (tma_common.cuh); star3d_tma_timeouts() reports waits that gave up.
@@ -343,9 +343,9 @@ static cudaError_t s3t_dispatch(const Problem& q, Star3dTmaParams& p, const S3tS
 }
 
 // mode as in the kernel.  `launched` false (with cudaSuccess) = this grid runs on the other engine.
-// The adjoint runs here by default (measured on 256^3: 26.7 us against 29.5 us for the L1-staged
+// The adjoint runs here by default (measured on 256^3: 24.8 us against 29.5 us for the L1-staged
 // engine); the forward pass, which streams a second input array and whose L1-staged kernel is
-// already within a tenth of its DRAM time, only with FPDE_STAR3D_TMA_FWD=1 (39 us against 34 us).
+// already within a tenth of its DRAM time, only with FPDE_STAR3D_TMA_FWD=1 (36 us against 34 us).
 cudaError_t launch_star3d_tma(const Problem& q, int mode, int* items, bool& launched) {
     launched = false;
     if (!star3d_tma_wanted(q.n)) return cudaSuccess;
