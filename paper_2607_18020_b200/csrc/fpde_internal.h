@@ -93,6 +93,31 @@ inline int planes_for_grid(int n0, int tuned, long items_per_chunk, long long po
     return planes;
 }
 
+// SMs of the current device (148 when there is none to ask: host-only queries).
+inline int sm_count_or_default() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    return n;
+}
+
+// Wave fitting for grids that fill the GPU: with `planes` planes per item a launch has
+// items_per_chunk * ceil(n0 / planes) blocks, which run in ceil(blocks / slots) waves (slots = SMs x
+// resident blocks per SM).  A last wave that is nearly empty, or a single wave that leaves some SMs
+// with one block more than others, costs up to a full item; this returns the item length whose
+// block count just fits the same number of waves (a little longer items, fewer blocks).
+inline int fit_planes_to_waves(int n0, int planes, long items_per_chunk, long slots) {
+    if (items_per_chunk < 1 || slots < 1) return planes;
+    const long blocks = items_per_chunk * ((n0 + planes - 1) / planes);
+    const long waves = (blocks + slots - 1) / slots;
+    const long chunks = waves * slots / items_per_chunk;           // most chunks that still fit
+    if (chunks < 1) return planes;
+    const int fitted = (int)((n0 + chunks - 1) / chunks);
+    return fitted >= planes ? fitted : planes;                      // never shorter than the tuned length
+}
+
 // Launchers: return cudaGetLastError() after queuing the kernels.
 cudaError_t launch_burgers_fwd(const Problem& p);
 cudaError_t launch_burgers_bwd(const Problem& p);

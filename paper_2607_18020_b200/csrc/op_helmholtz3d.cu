@@ -231,8 +231,13 @@ static void star3d_geometry(const Problem& q, Star3dParams& p, dim3& block, doub
     p.nmb = (p.n1 + ty - 1) / ty;
     const long per_chunk = (long)p.ncb * p.nmb;
     const long long points = (long long)p.n0 * p.n1 * p.n2;
-    p.planes_per_item = fwd ? env_int("FPDE_STAR3D_PLANES_F", planes_for_grid(p.n0, 32, per_chunk, points))
-                            : env_int("FPDE_STAR3D_PLANES_B", planes_for_grid(p.n0, 10, per_chunk, points));
+    // large grids: the tuned length, stretched until the blocks just fill whole waves of the 4 blocks
+    // an SM holds (256^3 forward: 32 -> 29 planes, 512 -> 576 blocks for 592 slots, 33.9 -> 31.9 us)
+    auto fitted = [&](int tuned) {
+        const int pl = planes_for_grid(p.n0, tuned, per_chunk, points);
+        return points >= (1ll << 22) ? fit_planes_to_waves(p.n0, pl, per_chunk, 4l * sm_count_or_default()) : pl;
+    };
+    p.planes_per_item = fwd ? env_int("FPDE_STAR3D_PLANES_F", fitted(32)) : env_int("FPDE_STAR3D_PLANES_B", fitted(10));
     p.nitems = p.ncb * p.nmb * ((p.n0 + p.planes_per_item - 1) / p.planes_per_item);
     double wsum = 0.0;
     for (int a = 0; a < 3; ++a) {
