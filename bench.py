@@ -383,9 +383,12 @@ def e2e_steps(torch, B, w, steps, warmup, barrier):
     """The same step from pinned HOST buffers through fpde_loss_grad_host: per step, H2D of every
     field/source, forward, adjoint, D2H of every gradient and of the loss, then a stream sync (the
     caller reads the loss)."""
-    hf = [torch.from_numpy(f).pin_memory() for f in w.fields]
+    # the fields (and the gradients) are slices of ONE pinned buffer each: evenly spaced arrays let the
+    # library move a range of planes of all of them in one strided copy
+    hf_all = torch.stack([torch.from_numpy(f) for f in w.fields]).pin_memory()
+    hg_all = torch.empty((len(w.fields),) + tuple(w.shape), dtype=torch.float32).pin_memory()
+    hf, hg = list(hf_all.unbind(0)), list(hg_all.unbind(0))
     hs = [torch.from_numpy(s).pin_memory() for s in w.sources]
-    hg = [torch.empty(w.shape, dtype=torch.float32).pin_memory() for _ in w.fields]
     ne = len(W.OP_META[w.op]["residuals"])
     hl = torch.zeros(ne + 1, dtype=torch.float64).pin_memory()
     arena = torch.empty(B.host_arena_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")

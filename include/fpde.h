@@ -360,7 +360,10 @@ int fpde_bwd_f64(int op,
  * on `stream`, and the gradients are copied down on a second internal stream, so the two copy
  * directions overlap; `stream` waits for both internal streams before the call's work counts as
  * done on it, so synchronising `stream` is still all a caller has to do.  (FPDE_HOST_PIPELINE=0
- * in the environment selects the plain one-stream form.)
+ * in the environment selects the plain one-stream form.)  If the host arrays of a kind are slices
+ * of ONE page-locked allocation at even spacing (e.g. h_fields[k] = base + k * stride), a range of
+ * planes of all of them moves in one strided copy instead of one copy per array, which is worth
+ * about 5 % of the step on a link busy in both directions; any other layout works as before.
  */
 size_t fpde_host_arena_bytes(int op, int ndim, const int64_t* shape);
 

@@ -1,6 +1,8 @@
 // C ABI of libfpde.so: operator registry, argument validation, conversion of host scalars to
 // kernel parameters, dispatch to the per-operator launchers, and the final loss reduction.
 // See include/fpde.h for the contract of every entry point.
+#include <cuda.h>
+
 #include "../../include/fpde.h"
 #include "fpde_common.cuh"
 #include "fpde_internal.h"
@@ -669,6 +671,31 @@ static std::vector<int> host_pipe_chunks(int n0) {
 // and destroying them on every call cost more than the launches they order).  Calls are queued
 // under the mutex, one at a time; an event recorded again by a later call does not disturb the
 // waits an earlier call queued on it (a stream wait captures the record that precedes it).
+// Is [lo, hi) inside ONE allocation the driver knows (pinned host memory or device memory)?  A
+// strided copy over several arrays is only valid when they are slices of one allocation; arrays that
+// merely happen to be evenly spaced are not.  (Driver entry point through the runtime, no -lcuda.)
+static bool one_allocation(const void* lo, const void* hi) {
+    typedef CUresult (*GetAttrFn)(void*, CUpointer_attribute, CUdeviceptr);
+    static GetAttrFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuPointerGetAttribute", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return (GetAttrFn) nullptr;
+        }
+        return reinterpret_cast<GetAttrFn>(f);
+    }();
+    if (fn == nullptr) return false;
+    CUdeviceptr start = 0;
+    size_t size = 0;
+    const CUdeviceptr p = reinterpret_cast<CUdeviceptr>(lo);
+    if (fn(&start, CU_POINTER_ATTRIBUTE_RANGE_START_ADDR, p) != CUDA_SUCCESS ||
+        fn(&size, CU_POINTER_ATTRIBUTE_RANGE_SIZE, p) != CUDA_SUCCESS)
+        return false;
+    return p >= start && reinterpret_cast<CUdeviceptr>(hi) <= start + size;
+}
+
 static std::mutex g_pipe_mutex;
 struct HostPipeState {
     cudaStream_t in = nullptr, out = nullptr;
@@ -761,9 +788,36 @@ static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, flo
     chk(cudaEventRecord(e_start, cs));
     chk(cudaStreamWaitEvent(s_in, e_start, 0));
     chk(cudaStreamWaitEvent(s_out, e_start, 0));
+    // When the caller's arrays of a kind are evenly spaced in host memory (slices of one buffer), the
+    // planes of all of them move in ONE strided copy per transfer instead of one copy per array: on a
+    // link busy in both directions every copy costs about 10 us of dead time.
+    auto even_stride = [&](const float* const* h, const float* const* d, ptrdiff_t* hs, ptrdiff_t* ds) {
+        if (nf < 2) return false;
+        const char* e = std::getenv("FPDE_HOST_STRIDED");
+        if (e && e[0] == '0') return false;
+        *hs = reinterpret_cast<const char*>(h[1]) - reinterpret_cast<const char*>(h[0]);
+        *ds = reinterpret_cast<const char*>(d[1]) - reinterpret_cast<const char*>(d[0]);
+        if (*hs <= 0 || *ds <= 0) return false;
+        for (int f = 2; f < nf; ++f)
+            if (reinterpret_cast<const char*>(h[f]) - reinterpret_cast<const char*>(h[f - 1]) != *hs ||
+                reinterpret_cast<const char*>(d[f]) - reinterpret_cast<const char*>(d[f - 1]) != *ds)
+                return false;
+        const size_t arr_bytes = (size_t)plane * n0 * sizeof(float);
+        if ((size_t)*hs < arr_bytes || (size_t)*ds < arr_bytes) return false;
+        return one_allocation(h[0], reinterpret_cast<const char*>(h[nf - 1]) + arr_bytes) &&
+               one_allocation(d[0], reinterpret_cast<const char*>(d[nf - 1]) + arr_bytes);
+    };
+    ptrdiff_t hs_in = 0, ds_in = 0, hs_out = 0, ds_out = 0;
+    const bool strided_in = even_stride(h_fields, d_f, &hs_in, &ds_in);
+    const bool strided_out = even_stride(h_gfields, d_g, &hs_out, &ds_out);
     auto up = [&](int64_t lo, int64_t hi) {
         if (hi <= lo) return;
         const size_t off = (size_t)(lo * plane), bytes = (size_t)((hi - lo) * plane) * sizeof(float);
+        if (strided_in) {
+            chk(cudaMemcpy2DAsync(d_f[0] + off, (size_t)ds_in, h_fields[0] + off, (size_t)hs_in, bytes, (size_t)nf,
+                                  cudaMemcpyHostToDevice, s_in));
+            return;
+        }
         for (int f = 0; f < nf; ++f)
             chk(cudaMemcpyAsync(d_f[f] + off, h_fields[f] + off, bytes, cudaMemcpyHostToDevice, s_in));
     };
@@ -796,6 +850,11 @@ static int loss_grad_host_pipelined(Problem q, const float* const* h_fields, flo
         chk(cudaEventRecord(e_bwd[c], cs));
         chk(cudaStreamWaitEvent(s_out, e_bwd[c], 0));
         const size_t off = (size_t)(first(c) * plane), bytes = (size_t)((end(c) - first(c)) * plane) * sizeof(float);
+        if (strided_out) {
+            chk(cudaMemcpy2DAsync(h_gfields[0] + off, (size_t)hs_out, d_g[0] + off, (size_t)ds_out, bytes, (size_t)nf,
+                                  cudaMemcpyDeviceToHost, s_out));
+            return;
+        }
         for (int f = 0; f < nf; ++f)
             chk(cudaMemcpyAsync(h_gfields[f] + off, d_g[f] + off, bytes, cudaMemcpyDeviceToHost, s_out));
     };

@@ -246,6 +246,36 @@ def test_pipelined_host_entry_for_navier_stokes(shape, monkeypatch):
         assert np.array_equal(a, b)
 
 
+@pytest.mark.parametrize("shape", [(48, 10, 8, 8), (33, 4, 8, 8)])
+def test_pipelined_host_entry_with_arrays_that_are_slices_of_one_buffer(shape, monkeypatch):
+    """When the host arrays of a kind are slices of ONE pinned buffer (evenly spaced, one allocation) the
+    pipelined host entry moves a range of planes of all of them in one strided copy; the results are bit
+    for bit those of separate buffers (which take one copy per array), and of FPDE_HOST_STRIDED=0."""
+    w = W.make("ns_tgv_128x16", seed=48, shape=shape, kind="randn")
+    arena = torch.empty(B.host_arena_bytes(w.op, w.shape), dtype=torch.uint8, device="cuda")
+    outs = []
+    for stacked, switch in ((True, "1"), (True, "0"), (False, "1")):
+        monkeypatch.setenv("FPDE_HOST_STRIDED", switch)
+        if stacked:
+            hf_all = torch.stack([torch.from_numpy(f) for f in w.fields]).pin_memory()
+            hg_all = torch.full((len(w.fields),) + tuple(shape), 7.0, dtype=torch.float32).pin_memory()
+            hf, hg = list(hf_all.unbind(0)), list(hg_all.unbind(0))
+        else:
+            hf = [torch.from_numpy(f).pin_memory() for f in w.fields]
+            hg = [torch.full(shape, 7.0, dtype=torch.float32).pin_memory() for _ in w.fields]
+        hl = torch.zeros(5, dtype=torch.float64).pin_memory()
+        B.fpde_loss_grad_host(w.op, hf, [], hg, hl, w.shape, w.spacing, w.coeffs, w.bc, arena)
+        torch.cuda.current_stream().synchronize()
+        outs.append(([g.numpy().copy() for g in hg], hl.numpy().copy()))
+    _, loss_ref, g_ref, _ = oracle.loss_and_grad(w.op, w.fields, w.sources, w.shape, w.spacing, w.coeffs)
+    for f, g in enumerate(outs[0][0]):
+        assert_close(g, g_ref[f], "host entry, stacked buffers, gradient %d" % f)
+    for gs, l in outs[1:]:
+        for a, b in zip(gs, outs[0][0]):
+            assert np.array_equal(a, b)
+        assert np.array_equal(l, outs[0][1])
+
+
 @pytest.mark.parametrize("shape", [(8, 12, 16, 8), (19, 8, 8, 16), (6, 4, 4, 32), (7, 16, 32, 16), (5, 12, 48, 8)])
 def test_ns_tma_and_l1_staged_kernels_agree_with_oracle(shape, monkeypatch):
     """FPDE_NS_TMA=1 runs grids that tile exactly on the TMA-staged kernels (one-box tiles away from
